@@ -1,0 +1,390 @@
+"""fp64 CPU oracle for the mHC-lite residual-mixing layer (and the mHC / SK path).
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, obviously-correct
+statement of what the CUDA library computes.  It shares no code with the CUDA
+path and must never be imported by it: only the tests, the smoke check and the
+benchmark's CPU-baseline leg may call it.
+
+Everything is evaluated in fp64, token by token (vectorised over the token
+axis with einsum / matmul as library steps; no blocking, fusion or reordering
+beyond what the equations state).
+
+What is computed, with the passage that defines it:
+
+* Eq. (1)   x_{l+1} = H_res x_l + H_post^T f(H_pre x_l)      -> premix_fwd, postres_fwd
+* Eq. (4)   RMSNorm of the flattened x_l, the three affine maps, sigmoid /
+            2*sigmoid / softmax                                -> coeffs_fwd
+* Eq. (5)   H_res = sum_k a_k P_k over all n! permutations     -> hres_from_weights
+            (Section 3.2 also states it as a product of a with a constant
+            0/1 matrix of shape n! x n^2                        -> hres_from_weights_matmul)
+* Eq. (2)   mHC: H_res = SK(exp(mat(.))), 20 iterations        -> sk_iterate, sk_coeffs_fwd
+* Section 3.1 footnote / Eq. (3): l1-error and relative range  -> l1_error, relative_range
+* the backward of all of the above is the exact gradient (the paper relies on
+  automatic differentiation)                                   -> *_bwd
+
+Readings of the paper taken here (each is a choice where the text is silent):
+  - RMSNorm: x' = x / sqrt(mean(x^2) + eps) * gain over the whole flattened
+    vector of length n*C; eps is an argument; gain is elementwise.
+  - flatten order: stream-major, m = j*C + c.
+  - permutations in lexicographic order of (sigma(0), ..., sigma(n-1)), index 0 the
+    identity; P_k[i, sigma_k(i)] = 1.
+  - H_post (1 x n) times f(.) (1 x C) is the outer product: row i of the update is
+    H_post[i] * y.
+  - projection columns ordered [res | pre | post]; alpha = (res, pre, post).
+  - SK: one iteration = normalise all columns, then all rows (the order that
+    reproduces the worked 3x3 example of Section 1); mat() is row-major; the
+    maximum logit is subtracted before exp (SK is invariant to a global scale).
+
+Pins (tests/test_oracle_*.py): permutation table vs brute force; exact double
+stochasticity; one-hot and uniform weights; the two routes to H_res; products
+over depth; the printed 3x3 SK example; closed forms of RMSNorm / softmax /
+sigmoid; n = 2 closed form; central finite differences for every gradient.
+Parity unpinned: the value of eps (a free argument) and the normalisation of the
+test tolerances, which are choices and not derivable from the paper.
+"""
+from __future__ import annotations
+
+import itertools
+import math
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------- #
+# permutations (Theorem 3.1 / Section 3.2)
+# --------------------------------------------------------------------------- #
+def perm_table(n: int) -> np.ndarray:
+    """All n! permutations of (0..n-1), lexicographic; row k is sigma_k. uint8 [n!, n]."""
+    return np.array(list(itertools.permutations(range(n))), dtype=np.uint8)
+
+
+def perm_matrices(n: int) -> np.ndarray:
+    """P[k, i, j] = 1 iff sigma_k(i) = j.  float64 [n!, n, n]."""
+    sig = perm_table(n)
+    P = np.zeros((sig.shape[0], n, n), dtype=F64)
+    for k in range(sig.shape[0]):
+        for i in range(n):
+            P[k, i, sig[k, i]] = 1.0
+    return P
+
+
+def hres_from_weights(a: np.ndarray, n: int) -> np.ndarray:
+    """Eq. (5): H_res[t] = sum_k a[t,k] P_k, by table look-up.  a [T, n!] -> [T, n, n]."""
+    sig = perm_table(n)
+    a = np.asarray(a, dtype=F64)
+    H = np.zeros((a.shape[0], n, n), dtype=F64)
+    for k in range(sig.shape[0]):
+        for i in range(n):
+            H[:, i, sig[k, i]] += a[:, k]
+    return H
+
+
+def hres_from_weights_matmul(a: np.ndarray, n: int) -> np.ndarray:
+    """Section 3.2: the same H_res as a @ M with M the constant 0/1 matrix [n!, n^2]."""
+    M = perm_matrices(n).reshape(-1, n * n)
+    return (np.asarray(a, dtype=F64) @ M).reshape(-1, n, n)
+
+
+# --------------------------------------------------------------------------- #
+# storage rounding (bf16 tensors between kernels)
+# --------------------------------------------------------------------------- #
+def round_bf16(a: np.ndarray) -> np.ndarray:
+    """Nearest-even rounding of fp64 values to the bf16 grid, returned as fp64."""
+    a = np.asarray(a, dtype=F64)
+    f32 = a.astype(np.float32)
+    bits = f32.view(np.uint32).astype(np.uint64)
+    low = bits & 0xFFFF
+    hi = bits >> 16
+    err = np.abs(a) - np.abs(f32.astype(F64))
+    up = (low > 0x8000) | ((low == 0x8000) & ((err > 0) | ((err == 0) & ((hi & 1) == 1))))
+    out = ((hi + up.astype(np.uint64)) << 16).astype(np.uint32)
+    return out.view(np.float32).astype(F64)
+
+
+# --------------------------------------------------------------------------- #
+# forward
+# --------------------------------------------------------------------------- #
+def _groups(n: int, n_res: int):
+    """Column slices (res, pre, post) of the concatenated projection."""
+    return slice(0, n_res), slice(n_res, n_res + n), slice(n_res + n, n_res + 2 * n)
+
+
+def _alpha_vec(alpha, n: int, n_res: int) -> np.ndarray:
+    alpha = np.asarray(alpha, dtype=F64).reshape(3)
+    return np.concatenate([np.full(n_res, alpha[0]), np.full(n, alpha[1]), np.full(n, alpha[2])])
+
+
+def rmsnorm_fwd(xh: np.ndarray, gain: np.ndarray, eps: float):
+    """x' = x * rstd * gain, rstd = (mean(x^2) + eps)^(-1/2), over the last axis."""
+    xh = np.asarray(xh, dtype=F64)
+    ms = np.mean(xh * xh, axis=-1)
+    rstd = 1.0 / np.sqrt(ms + eps)
+    return xh * rstd[..., None] * np.asarray(gain, dtype=F64), rstd
+
+
+def _logits(x, W, b, alpha, gain, eps, n_res):
+    x = np.asarray(x, dtype=F64)
+    T, n, C = x.shape
+    xh = x.reshape(T, n * C)                       # stream-major flatten
+    xn, rstd = rmsnorm_fwd(xh, gain, eps)
+    p = xn @ np.asarray(W, dtype=F64)              # [T, N]
+    z = _alpha_vec(alpha, n, n_res) * p + np.asarray(b, dtype=F64)
+    return xh, xn, rstd, p, z
+
+
+def _sigmoid(z):
+    return 1.0 / (1.0 + np.exp(-z))
+
+
+def _softmax(z):
+    m = np.max(z, axis=-1, keepdims=True)
+    e = np.exp(z - m)
+    return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def coeffs_fwd(x, W, b, alpha, gain, eps: float = 1e-6) -> dict:
+    """Eq. (4) and (5): the dynamic mappings of mHC-lite for every token.
+
+    x [T,n,C]; W [nC, n!+2n]; b [n!+2n]; alpha (res, pre, post); gain [nC].
+    Returns H_res [T,n,n], H_pre [T,n], H_post [T,n], a [T,n!], z, p, rstd.
+    """
+    n = np.asarray(x).shape[1]
+    n_res = math.factorial(n)
+    xh, xn, rstd, p, z = _logits(x, W, b, alpha, gain, eps, n_res)
+    gr, gp, go = _groups(n, n_res)
+    a = _softmax(z[:, gr])
+    return dict(H_res=hres_from_weights(a, n), H_pre=_sigmoid(z[:, gp]),
+                H_post=2.0 * _sigmoid(z[:, go]), a=a, z=z, p=p, rstd=rstd)
+
+
+def premix_fwd(x, H_pre) -> np.ndarray:
+    """Eq. (1), inner term: u = H_pre x_l.   [T,n,C],[T,n] -> [T,C]."""
+    return np.einsum("tj,tjc->tc", np.asarray(H_pre, dtype=F64), np.asarray(x, dtype=F64))
+
+
+def postres_fwd(x, y, H_res, H_post) -> np.ndarray:
+    """Eq. (1): x_{l+1}[i] = sum_j H_res[i,j] x_l[j] + H_post[i] y.  -> [T,n,C]."""
+    x = np.asarray(x, dtype=F64)
+    y = np.asarray(y, dtype=F64)
+    return (np.einsum("tij,tjc->tic", np.asarray(H_res, dtype=F64), x)
+            + np.asarray(H_post, dtype=F64)[:, :, None] * y[:, None, :])
+
+
+# --------------------------------------------------------------------------- #
+# backward (exact gradient of Eq. (1), (4), (5))
+# --------------------------------------------------------------------------- #
+def postres_bwd(x, y, H_res, H_post, g) -> dict:
+    """Gradient of postres_fwd w.r.t. y, H_res, H_post and x, given g = dL/dx_{l+1}."""
+    x = np.asarray(x, dtype=F64); y = np.asarray(y, dtype=F64); g = np.asarray(g, dtype=F64)
+    H_res = np.asarray(H_res, dtype=F64); H_post = np.asarray(H_post, dtype=F64)
+    return dict(dy=np.einsum("ti,tic->tc", H_post, g),
+                dH_post=np.einsum("tic,tc->ti", g, y),
+                dH_res=np.einsum("tic,tjc->tij", g, x),
+                dx=np.einsum("tij,tic->tjc", H_res, g))
+
+
+def premix_bwd(x, H_pre, du) -> dict:
+    """Gradient of premix_fwd given du = dL/du."""
+    x = np.asarray(x, dtype=F64); du = np.asarray(du, dtype=F64)
+    H_pre = np.asarray(H_pre, dtype=F64)
+    return dict(dH_pre=np.einsum("tc,tjc->tj", du, x),
+                dx=H_pre[:, :, None] * du[:, None, :])
+
+
+def _proj_bwd(xh, xn, rstd, p, W, alpha, gain, dz, n, n_res):
+    """Gradient through z = alpha*(RMSNorm(x) W) + b, shared by the lite and SK paths."""
+    T, nC = xh.shape
+    W = np.asarray(W, dtype=F64); gain = np.asarray(gain, dtype=F64)
+    gr, gp, go = _groups(n, n_res)
+    db = dz.sum(axis=0)
+    dalpha = np.array([np.sum(dz[:, s] * p[:, s]) for s in (gr, gp, go)])
+    e = _alpha_vec(alpha, n, n_res) * dz
+    dW = xn.T @ e
+    dxn = e @ W.T
+    dgain = np.sum(dxn * xh * rstd[:, None], axis=0)
+    s = np.sum(xh * gain * dxn, axis=1)
+    dxh = rstd[:, None] * gain * dxn - xh * (rstd ** 3 * s / nC)[:, None]
+    return dict(dx=dxh.reshape(T, n, nC // n), dW=dW, db=db, dalpha=dalpha, dgain=dgain, dz=dz)
+
+
+def coeffs_bwd(x, W, b, alpha, gain, eps, dH_res, dH_pre, dH_post) -> dict:
+    """Gradient of coeffs_fwd: from (dH_res, dH_pre, dH_post) to dx, dW, db, dalpha, dgain."""
+    x = np.asarray(x, dtype=F64)
+    n = x.shape[1]
+    n_res = math.factorial(n)
+    xh, xn, rstd, p, z = _logits(x, W, b, alpha, gain, eps, n_res)
+    gr, gp, go = _groups(n, n_res)
+    a = _softmax(z[:, gr]); H_pre = _sigmoid(z[:, gp]); H_post = 2.0 * _sigmoid(z[:, go])
+    # Eq. (5): dL/da_k = sum_i dH_res[i, sigma_k(i)]
+    da = np.einsum("tij,kij->tk", np.asarray(dH_res, dtype=F64), perm_matrices(n))
+    dz = np.empty_like(z)
+    dz[:, gr] = a * (da - np.sum(a * da, axis=1, keepdims=True))
+    dz[:, gp] = np.asarray(dH_pre, dtype=F64) * H_pre * (1.0 - H_pre)
+    dz[:, go] = np.asarray(dH_post, dtype=F64) * H_post * (1.0 - H_post / 2.0)
+    return _proj_bwd(xh, xn, rstd, p, W, alpha, gain, dz, n, n_res)
+
+
+def layer_fwd(x, y, W, b, alpha, gain, eps: float = 1e-6, kind: str = "lite", iters: int = 20) -> dict:
+    """One Hyper-Connections layer with the sublayer output y given (Eq. (1))."""
+    co = coeffs_fwd(x, W, b, alpha, gain, eps) if kind == "lite" else sk_coeffs_fwd(x, W, b, alpha, gain, eps, iters)
+    co["u"] = premix_fwd(x, co["H_pre"])
+    co["x_next"] = postres_fwd(x, y, co["H_res"], co["H_post"])
+    return co
+
+
+def layer_bwd(x, y, W, b, alpha, gain, eps, g, du, kind: str = "lite", iters: int = 20) -> dict:
+    """Backward of layer_fwd for L(x_next, u) with g = dL/dx_next, du = dL/du; y is an input."""
+    co = coeffs_fwd(x, W, b, alpha, gain, eps) if kind == "lite" else sk_coeffs_fwd(x, W, b, alpha, gain, eps, iters)
+    b1 = postres_bwd(x, y, co["H_res"], co["H_post"], g)
+    b2 = premix_bwd(x, co["H_pre"], du)
+    if kind == "lite":
+        b3 = coeffs_bwd(x, W, b, alpha, gain, eps, b1["dH_res"], b2["dH_pre"], b1["dH_post"])
+    else:
+        b3 = sk_coeffs_bwd(x, W, b, alpha, gain, eps, b1["dH_res"], b2["dH_pre"], b1["dH_post"], iters)
+    return dict(dx=b1["dx"] + b2["dx"] + b3["dx"], dy=b1["dy"], dW=b3["dW"], db=b3["db"],
+                dalpha=b3["dalpha"], dgain=b3["dgain"], dH_res=b1["dH_res"], dH_post=b1["dH_post"],
+                dH_pre=b2["dH_pre"], dx_coeffs=b3["dx"], dz=b3["dz"])
+
+
+# --------------------------------------------------------------------------- #
+# mHC comparison path: Sinkhorn-Knopp (Eq. (2))
+# --------------------------------------------------------------------------- #
+def sk_iterate(M0, iters: int = 20, keep: bool = False):
+    """SK on a batch of positive matrices [T,n,n]: `iters` x (all columns, then all rows)."""
+    M = np.array(M0, dtype=F64, copy=True)
+    hist = []
+    for _ in range(iters):
+        cs = M.sum(axis=1, keepdims=True)          # column sums (over rows i)
+        M = M / cs
+        if keep:
+            hist.append(("col", M.copy(), cs))
+        rs = M.sum(axis=2, keepdims=True)          # row sums (over columns j)
+        M = M / rs
+        if keep:
+            hist.append(("row", M.copy(), rs))
+    return (M, hist) if keep else M
+
+
+def sk_iterate_bwd(hist, dM):
+    """Reverse-mode through the normalisations recorded by sk_iterate(keep=True).
+
+    For Y = X / s with s the column (row) sum of X: dX = (dY - sum(dY*Y)) / s,
+    the sum taken within each column (row).
+    """
+    d = np.array(dM, dtype=F64, copy=True)
+    for kind, Y, s in reversed(hist):
+        ax = 1 if kind == "col" else 2
+        d = (d - np.sum(d * Y, axis=ax, keepdims=True)) / s
+    return d
+
+
+def sk_coeffs_fwd(x, W, b, alpha, gain, eps: float = 1e-6, iters: int = 20) -> dict:
+    """Eq. (2): mHC's mappings; W [nC, n^2+2n], columns [res (row-major n x n) | pre | post]."""
+    x = np.asarray(x, dtype=F64)
+    T, n, _ = x.shape
+    n_res = n * n
+    xh, xn, rstd, p, z = _logits(x, W, b, alpha, gain, eps, n_res)
+    gr, gp, go = _groups(n, n_res)
+    Z = z[:, gr].reshape(T, n, n)
+    M0 = np.exp(Z - Z.max(axis=(1, 2), keepdims=True))
+    return dict(H_res=sk_iterate(M0, iters), H_pre=_sigmoid(z[:, gp]), H_post=2.0 * _sigmoid(z[:, go]),
+                z=z, p=p, rstd=rstd, M0=M0)
+
+
+def sk_coeffs_bwd(x, W, b, alpha, gain, eps, dH_res, dH_pre, dH_post, iters: int = 20) -> dict:
+    x = np.asarray(x, dtype=F64)
+    T, n, _ = x.shape
+    n_res = n * n
+    xh, xn, rstd, p, z = _logits(x, W, b, alpha, gain, eps, n_res)
+    gr, gp, go = _groups(n, n_res)
+    Z = z[:, gr].reshape(T, n, n)
+    M0 = np.exp(Z - Z.max(axis=(1, 2), keepdims=True))
+    _, hist = sk_iterate(M0, iters, keep=True)
+    dM0 = sk_iterate_bwd(hist, np.asarray(dH_res, dtype=F64))
+    H_pre = _sigmoid(z[:, gp]); H_post = 2.0 * _sigmoid(z[:, go])
+    dz = np.empty_like(z)
+    dz[:, gr] = (dM0 * M0).reshape(T, n_res)       # through exp; the max shift carries no gradient
+    dz[:, gp] = np.asarray(dH_pre, dtype=F64) * H_pre * (1.0 - H_pre)
+    dz[:, go] = np.asarray(dH_post, dtype=F64) * H_post * (1.0 - H_post / 2.0)
+    return _proj_bwd(xh, xn, rstd, p, W, alpha, gain, dz, n, n_res)
+
+
+# --------------------------------------------------------------------------- #
+# doubly-stochastic diagnostics (Section 3.1)
+# --------------------------------------------------------------------------- #
+def l1_error(X) -> np.ndarray:
+    """||X 1 - 1||_1 + ||X^T 1 - 1||_1 per matrix (footnote of Section 3.1)."""
+    X = np.asarray(X, dtype=F64)
+    return np.abs(X.sum(axis=-1) - 1.0).sum(axis=-1) + np.abs(X.sum(axis=-2) - 1.0).sum(axis=-1)
+
+
+def relative_range(X) -> np.ndarray:
+    """Eq. (3): nu = (smallest positive entry) / (largest entry), per matrix."""
+    X = np.asarray(X, dtype=F64)
+    flat = X.reshape(X.shape[:-2] + (-1,))
+    pos = np.where(flat > 0, flat, np.inf)
+    return pos.min(axis=-1) / flat.max(axis=-1)
+
+
+def column_sums(X) -> np.ndarray:
+    return np.asarray(X, dtype=F64).sum(axis=-2)
+
+
+def depth_product(H_list) -> np.ndarray:
+    """prod_l H_res_l per token, later layers multiplying on the left (x_{l+1} = H_l x_l)."""
+    P = np.array(H_list[0], dtype=F64, copy=True)
+    for H in H_list[1:]:
+        P = np.einsum("tij,tjk->tik", np.asarray(H, dtype=F64), P)
+    return P
+
+
+# --------------------------------------------------------------------------- #
+# layer stack with a stand-in sublayer (used for the 24-layer workload)
+# --------------------------------------------------------------------------- #
+def standin_sublayer_fwd(u, eps: float = 1e-6):
+    """Stand-in for f: y = u / sqrt(mean(u^2) + eps) (no gain)."""
+    u = np.asarray(u, dtype=F64)
+    r = 1.0 / np.sqrt(np.mean(u * u, axis=-1, keepdims=True) + eps)
+    return u * r
+
+
+def standin_sublayer_bwd(u, dy, eps: float = 1e-6):
+    u = np.asarray(u, dtype=F64); dy = np.asarray(dy, dtype=F64)
+    C = u.shape[-1]
+    r = 1.0 / np.sqrt(np.mean(u * u, axis=-1, keepdims=True) + eps)
+    return r * dy - u * (r ** 3) * np.sum(u * dy, axis=-1, keepdims=True) / C
+
+
+def stack_fwd_bwd(x0, params, g_top, eps: float = 1e-6, bf16_storage: bool = True) -> dict:
+    """Forward and backward through len(params) layers with y = standin(u).
+
+    With bf16_storage, the tensors that live in bf16 between kernels (u, y,
+    x_{l+1}, dy, du, dx) are rounded to bf16 where they are stored; all arithmetic
+    stays fp64.
+    """
+    rnd = round_bf16 if bf16_storage else (lambda v: np.asarray(v, dtype=F64))
+    xs = [np.asarray(x0, dtype=F64)]
+    saved = []
+    for (W, b, alpha, gain) in params:
+        x = xs[-1]
+        co = coeffs_fwd(x, W, b, alpha, gain, eps)
+        u = rnd(premix_fwd(x, co["H_pre"]))
+        y = rnd(standin_sublayer_fwd(u, eps))
+        xs.append(rnd(postres_fwd(x, y, co["H_res"], co["H_post"])))
+        saved.append((co, u, y))
+    g = np.asarray(g_top, dtype=F64)
+    grads = []
+    for l in reversed(range(len(params))):
+        W, b, alpha, gain = params[l]
+        x = xs[l]; co, u, y = saved[l]
+        b1 = postres_bwd(x, y, co["H_res"], co["H_post"], g)
+        dy = rnd(b1["dy"])
+        du = rnd(standin_sublayer_bwd(u, dy, eps))
+        b2 = premix_bwd(x, co["H_pre"], du)
+        b3 = coeffs_bwd(x, W, b, alpha, gain, eps, b1["dH_res"], b2["dH_pre"], b1["dH_post"])
+        g = rnd(b1["dx"] + b2["dx"] + b3["dx"])
+        grads.append(dict(dW=b3["dW"], db=b3["db"], dalpha=b3["dalpha"], dgain=b3["dgain"]))
+    grads.reverse()
+    return dict(xs=xs, H_res=[s[0]["H_res"] for s in saved], dx0=g, grads=grads)
