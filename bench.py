@@ -1,0 +1,316 @@
+#!/usr/bin/env python
+"""Benchmark of the mHC-lite mixing hot path (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2]
+
+One "step" is one pass of the whole path over one batch of synthetic tokens: mappings + stream
+pre-mix, post/residual merge, the merge's backward, and the fused backward tail (the sublayer's
+output y and its backward's du are inputs).  Rank r of an N-GPU run processes its own shard of
+tokens (weak scaling, no data-path collective).  Prints one JSON line on rank 0.
+
+--impl reference times the fp64 CPU oracle on the host cores (rank 0 only) on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "mhclite_mixing_fwd_bwd_tokens_per_sec"
+UNIT = "tokens/s"
+
+
+def algorithmic_bytes_per_token(n: int, C: int) -> dict:
+    """bf16 bytes each stage must move per token when x_l is read once per pass."""
+    return {
+        "pre_fwd": (2 * n + 2) * C,          # read x_l, write u
+        "post_fwd": (4 * n + 2) * C,         # read x_l, y; write x_next
+        "post_bwd": (4 * n + 4) * C,         # read g, x_l, y; write dy
+        "tail_bwd": (6 * n + 2) * C,         # read du, x_l, g; write dx
+    }
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [s.strip() for s in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------
+def oracle_sample_tokens_per_sec(wl, sample_tokens: int, repeats: int = 1):
+    """Times the fp64 oracle (as it stands) on `sample_tokens` tokens of the workload, fwd+bwd."""
+    from oracle import mhclite_oracle as O
+    from paper_2601_05732_b200 import synth
+    inp = synth.make_layer_inputs(wl.n, wl.C, sample_tokens, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std)
+    f = synth.bf16_bits_to_f64
+    x, y, g, du = f(inp["x"]), f(inp["y"]), f(inp["g"]), f(inp["du"])
+    W, b, al, ga = (inp[k].astype(np.float64) for k in ("W", "b", "alpha", "gain"))
+    best = float("inf")
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        O.layer_fwd(x, y, W, b, al, ga, 1e-6)
+        if wl.backward:
+            O.layer_bwd(x, y, W, b, al, ga, 1e-6, g, du)
+        best = min(best, time.perf_counter() - t0)
+    return sample_tokens / best, best
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [d.get("num_threads", 1) for d in threadpool_info() if d.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, wl, rank):
+    """The oracle arm: each step is a bounded sample of the workload on the host cores."""
+    if rank != 0:
+        return
+    sample = min(wl.T, 2048)
+    for _ in range(args.warmup):
+        oracle_sample_tokens_per_sec(wl, sample)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample_tokens_per_sec(wl, sample)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    cores = blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "n": wl.n, "C": wl.C, "T": wl.T, "note": wl.note,
+                   "sample": f"{sample} tokens per step (input generation included)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{sample} tokens of {wl.name} per step, fwd+bwd, numpy fp64"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------
+def run_ours(args, wl, rank, world):
+    import torch
+    import torch.distributed as dist
+    from paper_2601_05732_b200 import synth
+    from paper_2601_05732_b200 import layer as L
+    from paper_2601_05732_b200.binding import MhcLite
+
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    # CPU baseline first (rank 0, single-GPU run only), before the first GPU call
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        sample = min(wl.T, args.cpu_sample)
+        v, secs = oracle_sample_tokens_per_sec(wl, sample)
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                        "sample": f"{sample} tokens of {wl.name}, fwd+bwd, numpy fp64, {secs:.1f} s"}
+
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    n, C, T = wl.n, wl.C, wl.T
+    inp = synth.make_layer_inputs(n, C, T, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std, shard=rank)
+    ctx = MhcLite(n, C, local)
+    P = L.LayerParams(inp["W"], inp["b"], inp["alpha"], inp["gain"], dev)
+    B = L.LayerBuffers(ctx, T, "lite")
+    x, y, g, du = (L.to_device_bf16(inp[k], dev) for k in ("x", "y", "g", "du"))
+    eps = 1e-6
+
+    def step():
+        L.pre_fwd(ctx, P, B, x, eps, True)
+        L.post_fwd(ctx, B, x, y)
+        if wl.backward:
+            L.post_bwd(ctx, B, x, y, g, True)
+            L.tail_bwd(ctx, P, B, x, g, du, eps, True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    # ---- timed region: K steps, device time, max over ranks ------------------------------------
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = ctx.kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = ctx.kernel_launches() - launches0
+    # keep the GPU busy a little longer so that the sampler sees the loaded clocks even for short runs
+    t_end = time.time() + 0.6
+    while rank == 0 and time.time() < t_end:
+        step()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    if world > 1:
+        tt = torch.tensor([ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+
+    # ---- per-stage device time (same launch configuration), for the roofline of the dominant stage
+    stages = [("pre_fwd", lambda: L.pre_fwd(ctx, P, B, x, eps, True)), ("post_fwd", lambda: L.post_fwd(ctx, B, x, y))]
+    if wl.backward:
+        stages += [("post_bwd", lambda: L.post_bwd(ctx, B, x, y, g, True)),
+                   ("tail_bwd", lambda: L.tail_bwd(ctx, P, B, x, g, du, eps, True))]
+    ev = {k: [] for k, _ in stages}
+    for _ in range(args.steps):
+        for k, fn in stages:
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b_.record()
+            ev[k].append((a, b_))
+    torch.cuda.synchronize()
+    stage_ms = {k: sum(a.elapsed_time(b_) for a, b_ in v) / len(v) for k, v in ev.items()}
+
+    # ---- end to end through the C ABI with host buffers ----------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda t: t.cpu().pin_memory()
+        hx, hy, hg, hdu = pin(x), pin(y), pin(g), pin(du)
+        hu, hxn, hdy, hdx = (torch.empty_like(t, device="cpu").pin_memory() for t in (B.u, B.x_next, B.dy, B.dx))
+        run = lambda: ctx.step_host(hx, hy, hg, hdu, P.W, P.b, P.alpha, P.gain, eps, hu, hxn, hdy, hdx,
+                                    B.dW, B.db, B.dalpha, B.dgain)
+        k_e2e = max(3, min(args.steps, 10))
+        for _ in range(2):
+            run()
+        barrier()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(k_e2e):
+            run()
+        b_.record()
+        barrier()
+        ms_e2e = a.elapsed_time(b_)
+        if world > 1:
+            tt = torch.tensor([ms_e2e], device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms_e2e = float(tt.item())
+        h2d = sum(t.numel() * 2 for t in (hx, hy, hg, hdu))
+        d2h = sum(t.numel() * 2 for t in (hu, hxn, hdy, hdx))
+        e2e = {"value": world * T * k_e2e / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / k_e2e}
+
+    if rank == 0:
+        peak, peak_kind = load_peaks()
+        bpt = algorithmic_bytes_per_token(n, C)
+        dom = max(stage_ms, key=stage_ms.get)
+        achieved = bpt[dom] * T / (stage_ms[dom] * 1e-3) / 1e9
+        total_bytes = sum(bpt[k] for k in stage_ms) * T
+        roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
+                    "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                    "whole_step_gbs": total_bytes / (ms / args.steps * 1e-3) / 1e9,
+                    "whole_step_frac_of_8TBs": total_bytes / (ms / args.steps * 1e-3) / 8e12,
+                    "stage_ms": stage_ms,
+                    "stage_gbs": {k: bpt[k] * T / (v * 1e-3) / 1e9 for k, v in stage_ms.items()}}
+        line = {
+            "metric": METRIC, "value": world * T * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, f32 accumulate",
+            "data": "synthetic",
+            "config": {"workload": wl.name, "n": n, "C": C, "T_per_gpu": T, "passes": "fwd+bwd" if wl.backward else "fwd",
+                       "note": wl.note, "l2": "inputs larger than L2 (working set %.0f MB)" % (total_bytes / 1e6)},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+            "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--T", type=int, default=0, help="override the token count of the workload")
+    ap.add_argument("--cpu-sample", type=int, default=16384, help="tokens of the oracle's timed sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2601_05732_b200 import synth
+    import dataclasses
+    wl = synth.WORKLOADS[args.workload]
+    if args.T:
+        wl = dataclasses.replace(wl, T=args.T)
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        run_reference(args, wl, rank)
+        return
+    if world != args.gpus:
+        if args.gpus != 1 or world != 1:
+            print(f"bench.py: --gpus {args.gpus} needs torchrun with {args.gpus} ranks (WORLD_SIZE={world})", file=sys.stderr)
+            sys.exit(2)
+    run_ours(args, wl, rank, world)
+
+
+if __name__ == "__main__":
+    main()

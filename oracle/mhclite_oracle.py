@@ -245,7 +245,7 @@ def layer_bwd(x, y, W, b, alpha, gain, eps, g, du, kind: str = "lite", iters: in
         b3 = sk_coeffs_bwd(x, W, b, alpha, gain, eps, b1["dH_res"], b2["dH_pre"], b1["dH_post"], iters)
     return dict(dx=b1["dx"] + b2["dx"] + b3["dx"], dy=b1["dy"], dW=b3["dW"], db=b3["db"],
                 dalpha=b3["dalpha"], dgain=b3["dgain"], dH_res=b1["dH_res"], dH_post=b1["dH_post"],
-                dH_pre=b2["dH_pre"], dx_coeffs=b3["dx"], dz=b3["dz"])
+                dH_pre=b2["dH_pre"], dx_coeffs=b3["dx"], dx_premix=b2["dx"], dz=b3["dz"])
 
 
 # --------------------------------------------------------------------------- #

@@ -1,0 +1,117 @@
+// Shared device/host helpers of the mHC-lite library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/mhclite.h"
+
+namespace mhcl {
+
+constexpr int kMaxN = 5;          // residual streams supported: 2..5
+constexpr int kMaxFact = 120;     // 5!
+constexpr int kWarp = 32;
+
+// ---- context -------------------------------------------------------------------------------------
+}  // namespace mhcl
+
+struct mhclite_ctx {
+    int n, C, device;
+    int nfact;                    // n!
+    int sm_count;
+    void* ws;
+    size_t ws_bytes;
+    mutable int64_t launches;     // kernels launched through this context
+    char err[256];
+};
+
+namespace mhcl {
+
+inline int ipow_fact(int n) { int f = 1; for (int i = 2; i <= n; ++i) f *= i; return f; }
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+inline int64_t round_up64(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+
+// Number of projection columns. kind 0: n!+2n (mHC-lite); kind 1: n*n+2n (SK path).
+inline int n_res_cols(int n, int kind) { return kind == 0 ? ipow_fact(n) : n * n; }
+inline int n_cols(int n, int kind) { return n_res_cols(n, kind) + 2 * n; }
+
+int fail(mhclite_ctx* ctx, int status, const char* fmt, ...);
+int check_cuda(mhclite_ctx* ctx, cudaError_t e, const char* what);
+
+// Workspace layout (all offsets 256-byte aligned). See workspace.cu.
+struct Workspace {
+    float* e;        // [T][Npad]   rstd * alpha (.) dz, fp32
+    float* kappa;    // [T]         rstd^2 * sum_c (alpha dz)_c p_c / (nC)
+    float* G;        // [nC][Npad]  sum_t x[t,m] e[t,c] (before the gain factor)
+    float* dH_pre;   // [T][n]      <du, x_j> of the fused backward tail
+    size_t bytes;
+    int Npad;
+};
+Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base);
+
+// Permutation tables in constant memory (perm_table.cu).
+struct PermTables {
+    uint8_t sigma[kMaxFact * kMaxN];         // sigma[k*n + i] = sigma_k(i)
+    uint8_t klist[kMaxN * kMaxN * 24];       // klist[(i*n+j)*(n-1)! + r] = r-th k with sigma_k(i) = j
+};
+void host_perm_tables(int n, PermTables* out);
+cudaError_t upload_perm_tables(int n);       // to the current device
+cudaError_t download_perm_sigma(int n, uint8_t* sigma_host);
+
+// Instantiates a statement for the compile-time stream count N_ = n (2..5).
+#define MHCL_DISPATCH_N(n, ...)                               \
+    switch (n) {                                              \
+        case 2: { constexpr int N_ = 2; __VA_ARGS__; } break; \
+        case 3: { constexpr int N_ = 3; __VA_ARGS__; } break; \
+        case 4: { constexpr int N_ = 4; __VA_ARGS__; } break; \
+        case 5: { constexpr int N_ = 5; __VA_ARGS__; } break; \
+        default: break;                                       \
+    }
+
+// ---- device helpers ------------------------------------------------------------------------------
+#ifdef __CUDACC__
+extern __constant__ PermTables c_perm[kMaxN + 1];   // indexed by n
+
+__device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+
+// 8 bf16 (one 16-byte vector) -> 8 floats
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+    f[0] = bf16lo(v.x); f[1] = bf16hi(v.x); f[2] = bf16lo(v.y); f[3] = bf16hi(v.y);
+    f[4] = bf16lo(v.z); f[5] = bf16hi(v.z); f[6] = bf16lo(v.w); f[7] = bf16hi(v.w);
+}
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);      // .x = a (low half), .y = b
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+    uint4 v;
+    v.x = pack2(f[0], f[1]); v.y = pack2(f[2], f[3]); v.z = pack2(f[4], f[5]); v.w = pack2(f[6], f[7]);
+    return v;
+}
+// streaming 16-byte accesses: activations are touched once per kernel
+__device__ __forceinline__ uint4 ld_stream(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(void* p, const uint4& v) {
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+#endif
+
+}  // namespace mhcl

@@ -1,0 +1,46 @@
+// Launchers of the library's kernels (host side). Each enqueues on the given stream and returns.
+#pragma once
+#include "common.cuh"
+
+namespace mhcl {
+
+// stream_kernels.cu
+void launch_premix_fwd(const mhclite_ctx* c, int64_t T, const void* x, const float* H_pre, void* u, cudaStream_t s);
+void launch_postres_fwd(const mhclite_ctx* c, int64_t T, const void* x, const void* y, const float* H_res,
+                        const float* H_post, void* x_next, cudaStream_t s);
+void launch_postres_bwd(const mhclite_ctx* c, int64_t T, const void* x, const void* y, const float* H_res,
+                        const float* H_post, const void* g, void* dy, float* dH_res, float* dH_post, void* dx,
+                        int acc, cudaStream_t s);
+void launch_premix_bwd(const mhclite_ctx* c, int64_t T, const void* x, const float* H_pre, const void* du,
+                       float* dH_pre, void* dx, int acc, cudaStream_t s);
+void launch_tail_mix(const mhclite_ctx* c, int64_t T, const void* x, const void* g, const void* du, const float* H_res,
+                     const float* H_pre, float* dH_pre, void* dx, cudaStream_t s);
+void launch_ds_gap(const mhclite_ctx* c, int64_t T, const float* H_res, float* l1, float* cdev, cudaStream_t s);
+
+// proj_kernels.cu : RMSNorm statistics + the skinny projection and its gradient
+// p[t,c] = rstd_t * sum_m x[t,m] gain[m] W[m,c] (c < N), rstd[t]
+void launch_proj_fwd(const mhclite_ctx* c, int64_t T, int N, const void* x, const float* W, const float* gain,
+                     float eps, float* p, float* rstd, cudaStream_t s);
+// dx[t,m] (+)= sum_c e[t,c] gain[m] W[m,c] - x[t,m] kappa[t]   (e = rstd*alpha*dz)
+void launch_proj_bwd_dx(const mhclite_ctx* c, int64_t T, int N, int Npad, const void* x, const float* W,
+                        const float* gain, const float* e, const float* kappa, void* dx, int acc, cudaStream_t s);
+// G[m,c] = sum_t x[t,m] e[t,c];  dW (+)= gain (.) G ;  dgain[m] (+)= sum_c W[m,c] G[m,c]
+void launch_proj_bwd_dw(const mhclite_ctx* c, int64_t T, int N, int Npad, const void* x, const float* W,
+                        const float* gain, const float* e, float* G, float* dW, float* dgain, int acc,
+                        cudaStream_t s);
+
+// act_kernels.cu : per-token activations, H_res assembly and their gradients
+void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const float* p, const float* b, const float* alpha,
+                         float* H_res, float* H_pre, float* H_post, float* a_saved, cudaStream_t s);
+void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float* a, const float* p, const float* rstd,
+                         const float* alpha, const float* H_pre, const float* H_post, const float* dH_res,
+                         const float* dH_pre, const float* dH_post, float* e, float* kappa, float* db,
+                         float* dalpha, cudaStream_t s);
+void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const float* p, const float* b, const float* alpha,
+                       float* H_res, float* H_pre, float* H_post, cudaStream_t s);
+void launch_sk_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, int iters, const float* p, const float* b,
+                       const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
+                       const float* dH_res, const float* dH_pre, const float* dH_post, float* e, float* kappa,
+                       float* db, float* dalpha, cudaStream_t s);
+
+}  // namespace mhcl

@@ -1,0 +1,432 @@
+// C ABI of the library: argument validation, workspace planning and kernel sequencing.
+#include <stdarg.h>
+#include <new>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace mhcl {
+
+int fail(mhclite_ctx* ctx, int status, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+        va_end(ap);
+    }
+    return status;
+}
+
+int check_cuda(mhclite_ctx* ctx, cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return MHCLITE_OK;
+    return fail(ctx, MHCLITE_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base) {
+    Workspace w;
+    const int N = n_cols(n, kind);
+    w.Npad = round_up(N, 8);
+    char* p = (char*)base;
+    size_t off = 0;
+    w.e = (float*)(p + off);     off += align256((size_t)T * w.Npad * sizeof(float));
+    w.kappa = (float*)(p + off); off += align256((size_t)T * sizeof(float));
+    w.G = (float*)(p + off);     off += align256((size_t)n * C * w.Npad * sizeof(float));
+    w.dH_pre = (float*)(p + off); off += align256((size_t)T * n * sizeof(float));
+    w.bytes = off;
+    return w;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+// Makes the context's device current for the duration of a call.
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int dev) {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != dev) { err = cudaSetDevice(dev); switched = (err == cudaSuccess); }
+    }
+    ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+};
+
+}  // namespace mhcl
+
+using namespace mhcl;
+
+#define MHCL_REQUIRE_CTX(ctx)  do { if (!(ctx)) return MHCLITE_ERR_BAD_ARG; (ctx)->err[0] = 0; } while (0)
+#define MHCL_REQUIRE_T(ctx, T) do { if ((T) < 0) return fail(ctx, MHCLITE_ERR_BAD_ARG, "T < 0"); } while (0)
+#define MHCL_PTR(ctx, p)                                                                            \
+    do {                                                                                            \
+        if (!(p)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "null pointer: %s", #p);                    \
+        if (!aligned16(p)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "pointer not 16-byte aligned: %s", #p); \
+    } while (0)
+#define MHCL_OPT_PTR(ctx, p)                                                                        \
+    do {                                                                                            \
+        if ((p) && !aligned16(p)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "pointer not 16-byte aligned: %s", #p); \
+    } while (0)
+#define MHCL_DEVICE(ctx)                                                                            \
+    DeviceGuard guard_((ctx)->device);                                                              \
+    if (guard_.err != cudaSuccess) return check_cuda(ctx, guard_.err, "cudaSetDevice")
+#define MHCL_LAUNCH_CHECK(ctx, what) do { int rc_ = check_cuda(ctx, cudaGetLastError(), what); if (rc_) return rc_; } while (0)
+
+static int need_workspace(mhclite_ctx* ctx, int64_t T, int kind, Workspace* w) {
+    const size_t need = mhclite_workspace_bytes(ctx->n, ctx->C, T, kind);
+    if (!ctx->ws || ctx->ws_bytes < need)
+        return fail(ctx, MHCLITE_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu attached", need, ctx->ws ? ctx->ws_bytes : (size_t)0);
+    *w = plan_workspace(ctx->n, ctx->C, T, kind, ctx->ws);
+    return MHCLITE_OK;
+}
+
+extern "C" {
+
+const char* mhclite_status_string(int status) {
+    switch (status) {
+        case MHCLITE_OK: return "ok";
+        case MHCLITE_ERR_BAD_ARG: return "bad argument";
+        case MHCLITE_ERR_CUDA: return "CUDA error";
+        case MHCLITE_ERR_WORKSPACE: return "workspace missing or too small";
+        case MHCLITE_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+const char* mhclite_last_error(const mhclite_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+int mhclite_create(mhclite_ctx** out, int n, int C, int device) {
+    if (!out) return MHCLITE_ERR_BAD_ARG;
+    *out = nullptr;
+    if (n < 2 || n > kMaxN || C <= 0 || (C % 8) != 0 || device < 0) return MHCLITE_ERR_BAD_ARG;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device >= count) return MHCLITE_ERR_CUDA;
+    mhclite_ctx* ctx = new (std::nothrow) mhclite_ctx();
+    if (!ctx) return MHCLITE_ERR_CUDA;
+    ctx->n = n; ctx->C = C; ctx->device = device; ctx->nfact = ipow_fact(n);
+    ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->err[0] = 0; ctx->launches = 0;
+    {
+        DeviceGuard g(device);
+        cudaError_t e = g.err;
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+        for (int k = 2; k <= kMaxN && e == cudaSuccess; ++k) e = upload_perm_tables(k);
+        if (e != cudaSuccess) { delete ctx; return MHCLITE_ERR_CUDA; }
+    }
+    *out = ctx;
+    return MHCLITE_OK;
+}
+
+int mhclite_destroy(mhclite_ctx* ctx) {
+    if (!ctx) return MHCLITE_ERR_BAD_ARG;
+    delete ctx;
+    return MHCLITE_OK;
+}
+
+int mhclite_perm_table(int n, uint8_t* sigma_host) {
+    if (n < 2 || n > kMaxN || !sigma_host) return MHCLITE_ERR_BAD_ARG;
+    PermTables t;
+    host_perm_tables(n, &t);
+    memcpy(sigma_host, t.sigma, (size_t)ipow_fact(n) * n);
+    return MHCLITE_OK;
+}
+
+int mhclite_perm_table_device(mhclite_ctx* ctx, uint8_t* sigma_host) {
+    MHCL_REQUIRE_CTX(ctx);
+    if (!sigma_host) return fail(ctx, MHCLITE_ERR_BAD_ARG, "null pointer: sigma_host");
+    MHCL_DEVICE(ctx);
+    return check_cuda(ctx, download_perm_sigma(ctx->n, sigma_host), "read permutation table");
+}
+
+size_t mhclite_workspace_bytes(int n, int C, int64_t T, int kind) {
+    if (n < 2 || n > kMaxN || C <= 0 || T < 0 || kind < 0 || kind > 1) return 0;
+    return plan_workspace(n, C, T, kind, nullptr).bytes;
+}
+
+int mhclite_set_workspace(mhclite_ctx* ctx, void* workspace, size_t bytes) {
+    MHCL_REQUIRE_CTX(ctx);
+    if (workspace && ((uintptr_t)workspace & 255)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "workspace not 256-byte aligned");
+    ctx->ws = workspace;
+    ctx->ws_bytes = workspace ? bytes : 0;
+    return MHCLITE_OK;
+}
+
+// ---- forward -------------------------------------------------------------------------------------
+int mhclite_coeffs_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W, const float* b,
+                       const float* alpha, const float* gain, float eps, float* H_res, float* H_pre, float* H_post,
+                       float* a_saved, float* p_saved, float* rstd, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, W); MHCL_PTR(ctx, b); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain);
+    MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, a_saved);
+    MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd);
+    if (!(eps >= 0.f)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "eps must be >= 0");
+    MHCL_DEVICE(ctx);
+    cudaStream_t s = (cudaStream_t)stream;
+    launch_proj_fwd(ctx, T, n_cols(ctx->n, 0), x, W, gain, eps, p_saved, rstd, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_fwd");
+    launch_lite_act_fwd(ctx, T, p_saved, b, alpha, H_res, H_pre, H_post, a_saved, s);
+    MHCL_LAUNCH_CHECK(ctx, "lite_act_fwd");
+    return MHCLITE_OK;
+}
+
+int mhclite_premix_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* H_pre, mhclite_bf16* u,
+                       void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, u);
+    MHCL_DEVICE(ctx);
+    launch_premix_fwd(ctx, T, x, H_pre, u, (cudaStream_t)stream);
+    MHCL_LAUNCH_CHECK(ctx, "premix_fwd");
+    return MHCLITE_OK;
+}
+
+int mhclite_postres_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const mhclite_bf16* y, const float* H_res,
+                        const float* H_post, mhclite_bf16* x_next, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, y); MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, x_next);
+    MHCL_DEVICE(ctx);
+    launch_postres_fwd(ctx, T, x, y, H_res, H_post, x_next, (cudaStream_t)stream);
+    MHCL_LAUNCH_CHECK(ctx, "postres_fwd");
+    return MHCLITE_OK;
+}
+
+int mhclite_pre_fwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W, const float* b,
+                          const float* alpha, const float* gain, float eps, float* H_res, float* H_pre, float* H_post,
+                          float* a_saved, float* p_saved, float* rstd, mhclite_bf16* u, void* stream) {
+    MHCL_REQUIRE_CTX(ctx);
+    if (T > 0) MHCL_PTR(ctx, u);
+    int rc = mhclite_coeffs_fwd(ctx, T, x, W, b, alpha, gain, eps, H_res, H_pre, H_post, a_saved, p_saved, rstd, stream);
+    if (rc) return rc;
+    return mhclite_premix_fwd(ctx, T, x, H_pre, u, stream);
+}
+
+// ---- backward ------------------------------------------------------------------------------------
+int mhclite_postres_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const mhclite_bf16* y, const float* H_res,
+                        const float* H_post, const mhclite_bf16* g, mhclite_bf16* dy, float* dH_res, float* dH_post,
+                        mhclite_bf16* dx, int accumulate_dx, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, y); MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, g);
+    MHCL_PTR(ctx, dy); MHCL_PTR(ctx, dH_res); MHCL_PTR(ctx, dH_post); MHCL_OPT_PTR(ctx, dx);
+    MHCL_DEVICE(ctx);
+    launch_postres_bwd(ctx, T, x, y, H_res, H_post, g, dy, dH_res, dH_post, dx, accumulate_dx, (cudaStream_t)stream);
+    MHCL_LAUNCH_CHECK(ctx, "postres_bwd");
+    return MHCLITE_OK;
+}
+
+int mhclite_premix_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* H_pre, const mhclite_bf16* du,
+                       float* dH_pre, mhclite_bf16* dx, int accumulate_dx, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, du); MHCL_PTR(ctx, dH_pre); MHCL_OPT_PTR(ctx, dx);
+    MHCL_DEVICE(ctx);
+    launch_premix_bwd(ctx, T, x, H_pre, du, dH_pre, dx, accumulate_dx, (cudaStream_t)stream);
+    MHCL_LAUNCH_CHECK(ctx, "premix_bwd");
+    return MHCLITE_OK;
+}
+
+// Zeroes the parameter-gradient accumulators that the kernels add into, unless the caller accumulates.
+static int prep_param_grads(mhclite_ctx* ctx, int N, float* db, float* dalpha, int accumulate, cudaStream_t s) {
+    if (accumulate) return MHCLITE_OK;
+    int rc = check_cuda(ctx, cudaMemsetAsync(db, 0, (size_t)N * sizeof(float), s), "memset db");
+    if (rc) return rc;
+    return check_cuda(ctx, cudaMemsetAsync(dalpha, 0, 3 * sizeof(float), s), "memset dalpha");
+}
+
+int mhclite_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W, const float* alpha,
+                       const float* gain, float eps, const float* a_saved, const float* p_saved, const float* rstd,
+                       const float* H_pre, const float* H_post, const float* dH_res, const float* dH_pre,
+                       const float* dH_post, mhclite_bf16* dx, int accumulate_dx, float* dW, float* db, float* dalpha,
+                       float* dgain, int accumulate_params, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    (void)eps;
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, W); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain); MHCL_PTR(ctx, a_saved);
+    MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, dH_res);
+    MHCL_PTR(ctx, dH_pre); MHCL_PTR(ctx, dH_post); MHCL_PTR(ctx, dx); MHCL_PTR(ctx, dW); MHCL_PTR(ctx, db);
+    MHCL_PTR(ctx, dalpha); MHCL_PTR(ctx, dgain);
+    Workspace w;
+    int rc = need_workspace(ctx, T, 0, &w);
+    if (rc) return rc;
+    MHCL_DEVICE(ctx);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int N = n_cols(ctx->n, 0);
+    rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
+    if (rc) return rc;
+    launch_lite_act_bwd(ctx, T, w.Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post, w.e,
+                        w.kappa, db, dalpha, s);
+    MHCL_LAUNCH_CHECK(ctx, "lite_act_bwd");
+    launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W, gain, w.e, w.kappa, dx, accumulate_dx, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dx");
+    launch_proj_bwd_dw(ctx, T, N, w.Npad, x, W, gain, w.e, w.G, dW, dgain, accumulate_params, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dw");
+    return MHCLITE_OK;
+}
+
+int mhclite_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W, const float* alpha,
+                           const float* gain, float eps, const float* a_saved, const float* p_saved, const float* rstd,
+                           const float* H_res, const float* H_pre, const float* H_post, const mhclite_bf16* g,
+                           const mhclite_bf16* du, const float* dH_res, const float* dH_post, mhclite_bf16* dx,
+                           float* dW, float* db, float* dalpha, float* dgain, int accumulate_params, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    (void)eps; (void)H_post;
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, W); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain); MHCL_PTR(ctx, a_saved);
+    MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd); MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post);
+    MHCL_PTR(ctx, g); MHCL_PTR(ctx, du); MHCL_PTR(ctx, dH_res); MHCL_PTR(ctx, dH_post); MHCL_PTR(ctx, dx);
+    MHCL_PTR(ctx, dW); MHCL_PTR(ctx, db); MHCL_PTR(ctx, dalpha); MHCL_PTR(ctx, dgain);
+    Workspace w;
+    int rc = need_workspace(ctx, T, 0, &w);
+    if (rc) return rc;
+    MHCL_DEVICE(ctx);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int N = n_cols(ctx->n, 0);
+    rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
+    if (rc) return rc;
+    launch_tail_mix(ctx, T, x, g, du, H_res, H_pre, w.dH_pre, dx, s);
+    MHCL_LAUNCH_CHECK(ctx, "tail_mix");
+    launch_lite_act_bwd(ctx, T, w.Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, w.dH_pre, dH_post, w.e,
+                        w.kappa, db, dalpha, s);
+    MHCL_LAUNCH_CHECK(ctx, "lite_act_bwd");
+    launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W, gain, w.e, w.kappa, dx, 1, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dx");
+    launch_proj_bwd_dw(ctx, T, N, w.Npad, x, W, gain, w.e, w.G, dW, dgain, accumulate_params, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dw");
+    return MHCLITE_OK;
+}
+
+// ---- SK comparison path --------------------------------------------------------------------------
+int mhc_sk20_coeffs_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W_sk, const float* b_sk,
+                        const float* alpha, const float* gain, float eps, int iters, float* H_res, float* H_pre,
+                        float* H_post, float* p_saved, float* rstd, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (iters < 1 || iters > 64) return fail(ctx, MHCLITE_ERR_BAD_ARG, "iters must be in [1,64]");
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, W_sk); MHCL_PTR(ctx, b_sk); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain);
+    MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd);
+    if (!(eps >= 0.f)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "eps must be >= 0");
+    MHCL_DEVICE(ctx);
+    cudaStream_t s = (cudaStream_t)stream;
+    launch_proj_fwd(ctx, T, n_cols(ctx->n, 1), x, W_sk, gain, eps, p_saved, rstd, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_fwd");
+    launch_sk_act_fwd(ctx, T, iters, p_saved, b_sk, alpha, H_res, H_pre, H_post, s);
+    MHCL_LAUNCH_CHECK(ctx, "sk_act_fwd");
+    return MHCLITE_OK;
+}
+
+int mhc_sk20_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W_sk, const float* b_sk,
+                        const float* alpha, const float* gain, float eps, int iters, const float* p_saved,
+                        const float* rstd, const float* H_pre, const float* H_post, const float* dH_res,
+                        const float* dH_pre, const float* dH_post, mhclite_bf16* dx, int accumulate_dx, float* dW,
+                        float* db, float* dalpha, float* dgain, int accumulate_params, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    (void)eps;
+    if (iters < 1 || iters > 64) return fail(ctx, MHCLITE_ERR_BAD_ARG, "iters must be in [1,64]");
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, W_sk); MHCL_PTR(ctx, b_sk); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain);
+    MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, dH_res);
+    MHCL_PTR(ctx, dH_pre); MHCL_PTR(ctx, dH_post); MHCL_PTR(ctx, dx); MHCL_PTR(ctx, dW); MHCL_PTR(ctx, db);
+    MHCL_PTR(ctx, dalpha); MHCL_PTR(ctx, dgain);
+    Workspace w;
+    int rc = need_workspace(ctx, T, 1, &w);
+    if (rc) return rc;
+    MHCL_DEVICE(ctx);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int N = n_cols(ctx->n, 1);
+    rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
+    if (rc) return rc;
+    launch_sk_act_bwd(ctx, T, w.Npad, iters, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post, w.e,
+                      w.kappa, db, dalpha, s);
+    MHCL_LAUNCH_CHECK(ctx, "sk_act_bwd");
+    launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W_sk, gain, w.e, w.kappa, dx, accumulate_dx, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dx");
+    launch_proj_bwd_dw(ctx, T, N, w.Npad, x, W_sk, gain, w.e, w.G, dW, dgain, accumulate_params, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dw");
+    return MHCLITE_OK;
+}
+
+int mhclite_ds_gap(mhclite_ctx* ctx, int64_t T, const float* H_res, float* l1_err, float* colsum_dev, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, H_res); MHCL_OPT_PTR(ctx, l1_err); MHCL_OPT_PTR(ctx, colsum_dev);
+    MHCL_DEVICE(ctx);
+    launch_ds_gap(ctx, T, H_res, l1_err, colsum_dev, (cudaStream_t)stream);
+    MHCL_LAUNCH_CHECK(ctx, "ds_gap");
+    return MHCLITE_OK;
+}
+
+// ---- whole step from host buffers ----------------------------------------------------------------
+namespace {
+struct StepStaging {
+    mhclite_bf16 *x, *y, *g, *du, *u, *x_next, *dy, *dx;
+    float *H_res, *H_pre, *H_post, *a, *p, *rstd, *dH_res, *dH_post;
+    size_t bytes;
+};
+StepStaging plan_step(int n, int C, int64_t T, void* base) {
+    StepStaging s;
+    char* p = (char*)base;
+    size_t off = 0;
+    const size_t big = (size_t)T * n * C * sizeof(mhclite_bf16), small = (size_t)T * C * sizeof(mhclite_bf16);
+    const int nf = ipow_fact(n), N = n_cols(n, 0);
+    auto take = [&](size_t b) { void* q = p + off; off += align256(b); return q; };
+    s.x = (mhclite_bf16*)take(big); s.y = (mhclite_bf16*)take(small); s.g = (mhclite_bf16*)take(big);
+    s.du = (mhclite_bf16*)take(small); s.u = (mhclite_bf16*)take(small); s.x_next = (mhclite_bf16*)take(big);
+    s.dy = (mhclite_bf16*)take(small); s.dx = (mhclite_bf16*)take(big);
+    s.H_res = (float*)take((size_t)T * n * n * 4); s.H_pre = (float*)take((size_t)T * n * 4);
+    s.H_post = (float*)take((size_t)T * n * 4); s.a = (float*)take((size_t)T * nf * 4);
+    s.p = (float*)take((size_t)T * N * 4); s.rstd = (float*)take((size_t)T * 4);
+    s.dH_res = (float*)take((size_t)T * n * n * 4); s.dH_post = (float*)take((size_t)T * n * 4);
+    s.bytes = off;
+    return s;
+}
+}  // namespace
+
+size_t mhclite_step_host_bytes(int n, int C, int64_t T) {
+    if (n < 2 || n > kMaxN || C <= 0 || T < 0) return 0;
+    return plan_step(n, C, T, nullptr).bytes;
+}
+
+int mhclite_step_host(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x_host, const mhclite_bf16* y_host,
+                      const mhclite_bf16* g_host, const mhclite_bf16* du_host, const float* W, const float* b,
+                      const float* alpha, const float* gain, float eps, mhclite_bf16* u_host,
+                      mhclite_bf16* x_next_host, mhclite_bf16* dy_host, mhclite_bf16* dx_host, float* dW, float* db,
+                      float* dalpha, float* dgain, int accumulate_params, void* staging, size_t staging_bytes,
+                      void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    if (!x_host || !y_host || !g_host || !du_host || !u_host || !x_next_host || !dy_host || !dx_host)
+        return fail(ctx, MHCLITE_ERR_BAD_ARG, "null host pointer");
+    if (!staging || ((uintptr_t)staging & 255)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "staging null or not 256-byte aligned");
+    const StepStaging s = plan_step(ctx->n, ctx->C, T, staging);
+    if (staging_bytes < s.bytes)
+        return fail(ctx, MHCLITE_ERR_WORKSPACE, "staging of %zu bytes needed, %zu given", s.bytes, staging_bytes);
+    MHCL_DEVICE(ctx);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t big = (size_t)T * ctx->n * ctx->C * sizeof(mhclite_bf16), small = (size_t)T * ctx->C * sizeof(mhclite_bf16);
+    int rc;
+#define MHCL_COPY(dst, src, bytes, kind) \
+    if ((rc = check_cuda(ctx, cudaMemcpyAsync(dst, src, bytes, kind, st), "cudaMemcpyAsync " #dst))) return rc
+    MHCL_COPY(s.x, x_host, big, cudaMemcpyHostToDevice);
+    if ((rc = mhclite_pre_fwd_fused(ctx, T, s.x, W, b, alpha, gain, eps, s.H_res, s.H_pre, s.H_post, s.a, s.p, s.rstd,
+                                    s.u, stream))) return rc;
+    MHCL_COPY(u_host, s.u, small, cudaMemcpyDeviceToHost);
+    MHCL_COPY(s.y, y_host, small, cudaMemcpyHostToDevice);
+    if ((rc = mhclite_postres_fwd(ctx, T, s.x, s.y, s.H_res, s.H_post, s.x_next, stream))) return rc;
+    MHCL_COPY(x_next_host, s.x_next, big, cudaMemcpyDeviceToHost);
+    MHCL_COPY(s.g, g_host, big, cudaMemcpyHostToDevice);
+    if ((rc = mhclite_postres_bwd(ctx, T, s.x, s.y, s.H_res, s.H_post, s.g, s.dy, s.dH_res, s.dH_post, nullptr, 0,
+                                  stream))) return rc;
+    MHCL_COPY(dy_host, s.dy, small, cudaMemcpyDeviceToHost);
+    MHCL_COPY(s.du, du_host, small, cudaMemcpyHostToDevice);
+    if ((rc = mhclite_tail_bwd_fused(ctx, T, s.x, W, alpha, gain, eps, s.a, s.p, s.rstd, s.H_res, s.H_pre, s.H_post,
+                                     s.g, s.du, s.dH_res, s.dH_post, s.dx, dW, db, dalpha, dgain, accumulate_params,
+                                     stream))) return rc;
+    MHCL_COPY(dx_host, s.dx, big, cudaMemcpyDeviceToHost);
+#undef MHCL_COPY
+    return MHCLITE_OK;
+}
+
+int64_t mhclite_kernel_launches(const mhclite_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

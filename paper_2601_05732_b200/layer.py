@@ -1,0 +1,90 @@
+"""Device buffers of one Hyper-Connections layer and the call sequences around the caller's sublayer.
+
+Plumbing only: tensors are allocated with PyTorch and handed to the C ABI through
+:class:`~paper_2601_05732_b200.binding.MhcLite`; every step of the path runs in the
+library's kernels.
+
+Forward (paper Eq. (1), (4), (5)):   pre  -> [sublayer f: the caller's] -> post
+Backward:                            post_bwd -> [f's backward]        -> tail
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from .binding import MhcLite
+
+
+def to_device_bf16(bits: np.ndarray, device) -> torch.Tensor:
+    """uint16 bf16 bit patterns -> bf16 tensor on the device (no value conversion)."""
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+def bf16_to_host_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+class LayerParams:
+    def __init__(self, W, b, alpha, gain, device):
+        f = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device)
+        self.W, self.b, self.alpha, self.gain = f(W), f(b), f(alpha), f(gain)
+
+
+class LayerBuffers:
+    """Outputs and saved tensors of one layer for T tokens (kind 'lite' or 'sk')."""
+
+    def __init__(self, ctx: MhcLite, T: int, kind: str = "lite"):
+        n, C, dev = ctx.n, ctx.C, f"cuda:{ctx.device}"
+        self.kind = kind
+        N = ctx.n_cols(0 if kind == "lite" else 1)
+        f32 = lambda *s: torch.empty(*s, dtype=torch.float32, device=dev)
+        bf = lambda *s: torch.empty(*s, dtype=torch.bfloat16, device=dev)
+        self.H_res, self.H_pre, self.H_post = f32(T, n, n), f32(T, n), f32(T, n)
+        self.a_saved = f32(T, ctx.nfact) if kind == "lite" else None
+        self.p_saved, self.rstd = f32(T, N), f32(T)
+        self.u, self.x_next = bf(T, C), bf(T, n, C)
+        self.dy, self.dx = bf(T, C), bf(T, n, C)
+        self.dH_res, self.dH_post, self.dH_pre = f32(T, n, n), f32(T, n), f32(T, n)
+        self.dW, self.db, self.dalpha, self.dgain = f32(n * C, N), f32(N), f32(4)[:3], f32(n * C)
+        ctx.ensure_workspace(T, 0 if kind == "lite" else 1)
+
+
+def pre_fwd(ctx: MhcLite, P: LayerParams, B: LayerBuffers, x, eps=1e-6, fused=True, iters=20):
+    """Mappings + stream pre-mix: everything before the sublayer. Result: B.u (and the coefficients)."""
+    if B.kind == "sk":
+        ctx.sk20_coeffs_fwd(x, P.W, P.b, P.alpha, P.gain, eps, iters, B.H_res, B.H_pre, B.H_post, B.p_saved, B.rstd)
+        ctx.premix_fwd(x, B.H_pre, B.u)
+    elif fused:
+        ctx.pre_fwd_fused(x, P.W, P.b, P.alpha, P.gain, eps, B.H_res, B.H_pre, B.H_post, B.a_saved, B.p_saved,
+                          B.rstd, B.u)
+    else:
+        ctx.coeffs_fwd(x, P.W, P.b, P.alpha, P.gain, eps, B.H_res, B.H_pre, B.H_post, B.a_saved, B.p_saved, B.rstd)
+        ctx.premix_fwd(x, B.H_pre, B.u)
+
+
+def post_fwd(ctx: MhcLite, B: LayerBuffers, x, y):
+    """Residual mixing + merge of the sublayer output: B.x_next."""
+    ctx.postres_fwd(x, y, B.H_res, B.H_post, B.x_next)
+
+
+def post_bwd(ctx: MhcLite, B: LayerBuffers, x, y, g, fused=True):
+    """Backward of the merge: B.dy, B.dH_res, B.dH_post (and, unfused, the H_res^T g part of B.dx)."""
+    skip_dx = fused and B.kind == "lite"          # the fused tail recomputes H_res^T g from g
+    ctx.postres_bwd(x, y, B.H_res, B.H_post, g, B.dy, B.dH_res, B.dH_post, None if skip_dx else B.dx, False)
+
+
+def tail_bwd(ctx: MhcLite, P: LayerParams, B: LayerBuffers, x, g, du, eps=1e-6, fused=True, iters=20,
+             accumulate_params=False):
+    """Everything after the sublayer's backward: B.dx and the parameter gradients."""
+    if B.kind == "sk":
+        ctx.premix_bwd(x, B.H_pre, du, B.dH_pre, B.dx, True)
+        ctx.sk20_coeffs_bwd(x, P.W, P.b, P.alpha, P.gain, eps, iters, B.p_saved, B.rstd, B.H_pre, B.H_post,
+                            B.dH_res, B.dH_pre, B.dH_post, B.dx, True, B.dW, B.db, B.dalpha, B.dgain,
+                            accumulate_params)
+    elif fused:
+        ctx.tail_bwd_fused(x, P.W, P.alpha, P.gain, eps, B.a_saved, B.p_saved, B.rstd, B.H_res, B.H_pre, B.H_post,
+                           g, du, B.dH_res, B.dH_post, B.dx, B.dW, B.db, B.dalpha, B.dgain, accumulate_params)
+    else:
+        ctx.premix_bwd(x, B.H_pre, du, B.dH_pre, B.dx, True)
+        ctx.coeffs_bwd(x, P.W, P.alpha, P.gain, eps, B.a_saved, B.p_saved, B.rstd, B.H_pre, B.H_post,
+                       B.dH_res, B.dH_pre, B.dH_post, B.dx, True, B.dW, B.db, B.dalpha, B.dgain, accumulate_params)

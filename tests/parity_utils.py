@@ -1,0 +1,120 @@
+"""Helpers of the GPU parity tests: run the CUDA path through the C ABI, run the oracle on the same host
+inputs, and compare element by element with the stated tolerances.
+
+Tolerances (they follow the arithmetic: bf16 storage rounds to 2^-9 relative, fp32 accumulation over
+n*C <= 2^15 terms leaves ~1e-6 relative):
+  bf16 tensors : |gpu - ref| <= 2e-2 |ref| + 1e-3 rms(ref)          for every element
+  fp32 mappings: |gpu - ref| <= 1e-5 max(|ref|, rms(ref))           (H_res, H_pre, H_post, a, p, rstd)
+  fp32 parameter gradients: |gpu - ref| <= 1e-3 max(|ref|, rms(ref)) (the binding tolerance is 2e-2)
+"""
+import numpy as np
+import torch
+
+from oracle import mhclite_oracle as O
+from paper_2601_05732_b200 import synth
+from paper_2601_05732_b200.binding import MhcLite
+from paper_2601_05732_b200 import layer as L
+
+DEV = "cuda:0"
+
+
+def rms(a):
+    a = np.asarray(a, dtype=np.float64)
+    return float(np.sqrt(np.mean(a * a))) if a.size else 0.0
+
+
+def check_bf16(name, got, ref, rel=2e-2, floor=1e-3, extra=0.0):
+    """`extra` (per element) allows for a tensor that was stored in bf16 on the way: one rounding of
+    an intermediate v moves the result by up to 2^-8 |v|, whatever the size of the final value."""
+    got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (name, got.shape, ref.shape)
+    tol = rel * np.abs(ref) + floor * rms(ref) + extra
+    bad = np.abs(got - ref) > tol
+    assert not bad.any(), f"{name}: {bad.sum()} of {bad.size} elements off; worst {np.abs(got - ref).max():.3e} (rms {rms(ref):.3e})"
+
+
+def check_f32(name, got, ref, rel=1e-5):
+    got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (name, got.shape, ref.shape)
+    tol = rel * np.maximum(np.abs(ref), rms(ref)) + 1e-30
+    err = np.abs(got - ref)
+    assert (err <= tol).all(), f"{name}: worst err/tol {np.max(err / tol):.2f}, max abs err {err.max():.3e}, rms {rms(ref):.3e}"
+
+
+def host(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+class GpuLayer:
+    """Uploads one layer's host inputs and runs the library's call sequence on them."""
+
+    def __init__(self, inp, eps=1e-6, kind="lite", iters=20):
+        self.inp, self.eps, self.kind, self.iters = inp, eps, kind, iters
+        n, C, T = inp["n"], inp["C"], inp["T"]
+        self.ctx = MhcLite(n, C, 0)
+        self.P = L.LayerParams(inp["W"], inp["b"], inp["alpha"], inp["gain"], DEV)
+        self.B = L.LayerBuffers(self.ctx, T, kind)
+        self.x = L.to_device_bf16(inp["x"], DEV); self.y = L.to_device_bf16(inp["y"], DEV)
+        self.g = L.to_device_bf16(inp["g"], DEV); self.du = L.to_device_bf16(inp["du"], DEV)
+
+    def forward(self, fused=True):
+        L.pre_fwd(self.ctx, self.P, self.B, self.x, self.eps, fused, self.iters)
+        L.post_fwd(self.ctx, self.B, self.x, self.y)
+        torch.cuda.synchronize()
+
+    def backward(self, fused=True, accumulate_params=False):
+        L.post_bwd(self.ctx, self.B, self.x, self.y, self.g, fused)
+        L.tail_bwd(self.ctx, self.P, self.B, self.x, self.g, self.du, self.eps, fused, self.iters, accumulate_params)
+        torch.cuda.synchronize()
+
+
+def oracle_inputs(inp):
+    f = synth.bf16_bits_to_f64
+    return dict(x=f(inp["x"]), y=f(inp["y"]), g=f(inp["g"]), du=f(inp["du"]),
+                W=inp["W"].astype(np.float64), b=inp["b"].astype(np.float64),
+                alpha=inp["alpha"].astype(np.float64), gain=inp["gain"].astype(np.float64))
+
+
+def oracle_fwd(inp, eps=1e-6, kind="lite", iters=20):
+    o = oracle_inputs(inp)
+    return O.layer_fwd(o["x"], o["y"], o["W"], o["b"], o["alpha"], o["gain"], eps, kind=kind, iters=iters)
+
+
+def oracle_bwd(inp, eps=1e-6, kind="lite", iters=20):
+    o = oracle_inputs(inp)
+    return O.layer_bwd(o["x"], o["y"], o["W"], o["b"], o["alpha"], o["gain"], eps, o["g"], o["du"], kind=kind, iters=iters)
+
+
+def compare_forward(G, ref, coeff_rel=1e-5):
+    B = G.B
+    check_f32("rstd", host(B.rstd), ref["rstd"], coeff_rel)
+    check_f32("p_saved", host(B.p_saved), ref["p"], coeff_rel)
+    if G.kind == "lite":
+        check_f32("a_saved", host(B.a_saved), ref["a"], coeff_rel)
+    check_f32("H_res", host(B.H_res), ref["H_res"], coeff_rel)
+    check_f32("H_pre", host(B.H_pre), ref["H_pre"], coeff_rel)
+    check_f32("H_post", host(B.H_post), ref["H_post"], coeff_rel)
+    check_bf16("u", host(B.u), ref["u"])
+    check_bf16("x_next", host(B.x_next), ref["x_next"])
+
+
+def staged_dx_allowance(ref, fused):
+    """dx is stored in bf16 between the calls that add to it: each stored intermediate v may round
+    the other way on the GPU (fp32 sums) than in fp64, which moves dx by up to 2^-8 |v|."""
+    d2 = ref["dx"] - ref["dx_coeffs"]                     # after H_res^T g + H_pre du
+    if fused:
+        return 2.0 ** -8 * np.abs(d2)
+    d1 = d2 - ref["dx_premix"]                            # after H_res^T g
+    return 2.0 ** -8 * (np.abs(d1) + np.abs(d2))
+
+
+def compare_backward(G, ref, grad_rel=1e-3, fused=True):
+    B = G.B
+    check_bf16("dy", host(B.dy), ref["dy"])
+    check_f32("dH_res", host(B.dH_res), ref["dH_res"], 2e-5)
+    check_f32("dH_post", host(B.dH_post), ref["dH_post"], 2e-5)
+    check_bf16("dx", host(B.dx), ref["dx"], extra=staged_dx_allowance(ref, fused))
+    check_f32("dW", host(B.dW), ref["dW"], grad_rel)
+    check_f32("db", host(B.db), ref["db"], grad_rel)
+    check_f32("dalpha", host(B.dalpha), ref["dalpha"], grad_rel)
+    check_f32("dgain", host(B.dgain), ref["dgain"], grad_rel)

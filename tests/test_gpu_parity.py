@@ -1,0 +1,183 @@
+"""Element-by-element parity of the CUDA path (through the C ABI) with the fp64 oracle on the same
+seeded inputs: sizes that span several tiles with ragged tails, every n, both call sequences."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mhclite_oracle as O
+from paper_2601_05732_b200 import synth
+from paper_2601_05732_b200 import layer as L
+from parity_utils import (DEV, GpuLayer, check_bf16, check_f32, compare_backward, compare_forward, host,
+                          oracle_bwd, oracle_fwd, oracle_inputs)
+
+pytestmark = pytest.mark.gpu
+
+CASES = [  # (n, C, T): ragged token tails (T not a multiple of 32/64/128) and ragged channel tails
+    (4, 256, 333), (4, 264, 130), (2, 8, 77), (3, 72, 200), (5, 136, 161), (4, 1024, 257), (3, 1536, 65),
+]
+
+
+@pytest.mark.parametrize("n,C,T", CASES)
+@pytest.mark.parametrize("fused", [True, False])
+def test_layer_parity(n, C, T, fused):
+    inp = synth.make_layer_inputs(n, C, T, seed=10 + n, bias_std=0.1, gain_std=0.1)
+    G = GpuLayer(inp)
+    G.forward(fused)
+    compare_forward(G, oracle_fwd(inp))
+    G.backward(fused)
+    compare_backward(G, oracle_bwd(inp), fused=fused)
+
+
+@pytest.mark.parametrize("n", [2, 3, 4, 5])
+def test_permutation_table_on_device_bit_exact(n):
+    from paper_2601_05732_b200.binding import MhcLite
+    got = MhcLite(n, 8).perm_table_device()
+    assert (got == O.perm_table(n)).all()
+
+
+@pytest.mark.parametrize("n", [2, 3, 4])
+def test_one_hot_weight_selects_each_permutation(n):
+    # W = 0, b_res = 0 at k and -200 elsewhere: a = e_k and H_res = P_k exactly (fp32 exp underflows to 0)
+    C, T = 64, 5
+    nf = math.factorial(n)
+    tab = O.perm_table(n)
+    for k in range(nf):
+        inp = synth.make_layer_inputs(n, C, T, seed=3)
+        inp["W"][:] = 0
+        inp["b"][:nf] = -200.0
+        inp["b"][k] = 0.0
+        G = GpuLayer(inp)
+        G.forward()
+        H = host(G.B.H_res)
+        expect = np.zeros((n, n)); expect[np.arange(n), tab[k]] = 1.0
+        assert (H == expect[None]).all(), k
+        # x_next = P_k x + H_post y with H_post = 1 (b_post = 0): row i takes stream sigma_k(i)
+        ref = oracle_fwd(inp)
+        check_bf16("x_next", host(G.B.x_next), ref["x_next"])
+
+
+def test_paper_initialisation_is_near_identity():
+    n, C, T = 4, 128, 64
+    inp = synth.make_layer_inputs(n, C, T, seed=4)
+    inp["W"][:] = 0
+    inp["b"][:] = synth.paper_init_bias(n)
+    G = GpuLayer(inp); G.forward()
+    ref = oracle_fwd(inp)
+    compare_forward(G, ref)
+    H = host(G.B.H_res)
+    assert np.abs(H - np.eye(4)).max() < 24 * math.exp(-8.0)
+
+
+@pytest.mark.parametrize("n", [3, 4, 5])
+def test_sharp_logits(n):
+    # alpha = 1 and a wide bias: the softmax is far from uniform, so a wrong permutation mapping or
+    # a wrong column group shows at first order.  fp32 accumulation over n*C terms of |p| ~ 5 leaves
+    # ~1e-5 absolute in the logits, hence the looser coefficient tolerance here.
+    C, T = 256, 150
+    inp = synth.make_layer_inputs(n, C, T, seed=20 + n, bias_std=2.0, alpha=[1.0, 0.7, 1.3], w_std=0.05, gain_std=0.2)
+    G = GpuLayer(inp)
+    G.forward(); compare_forward(G, oracle_fwd(inp), coeff_rel=2e-4)
+    G.backward(); compare_backward(G, oracle_bwd(inp), grad_rel=2e-3)
+    Hr = host(G.B.H_res)
+    assert np.abs(Hr.sum(1) - 1).max() < 1e-6 and np.abs(Hr.sum(2) - 1).max() < 1e-6 and Hr.min() >= 0
+    assert Hr.std() > 0.05     # genuinely non-uniform
+
+
+def test_coeffs_bwd_in_isolation():
+    # the gradient through the mappings is ~0.5 % of dx at the benchmark's distributions: check it alone
+    n, C, T = 4, 256, 200
+    inp = synth.make_layer_inputs(n, C, T, seed=31, bias_std=0.5, alpha=[1.0, 1.0, 1.0], w_std=0.05)
+    G = GpuLayer(inp); G.forward(False)
+    ref = oracle_bwd(inp)
+    B, P = G.B, G.P
+    f = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(DEV)
+    dHr, dHp, dHo = f(ref["dH_res"]), f(ref["dH_pre"]), f(ref["dH_post"])
+    G.ctx.coeffs_bwd(G.x, P.W, P.alpha, P.gain, 1e-6, B.a_saved, B.p_saved, B.rstd, B.H_pre, B.H_post,
+                     dHr, dHp, dHo, B.dx, False, B.dW, B.db, B.dalpha, B.dgain, False)
+    torch.cuda.synchronize()
+    check_bf16("dx_coeffs", host(B.dx), ref["dx_coeffs"])
+    check_f32("dW", host(B.dW), ref["dW"], 1e-3)
+    check_f32("dgain", host(B.dgain), ref["dgain"], 1e-3)
+    check_f32("db", host(B.db), ref["db"], 1e-3)
+    check_f32("dalpha", host(B.dalpha), ref["dalpha"], 1e-3)
+    # accumulate_params adds to what is there
+    G.ctx.coeffs_bwd(G.x, P.W, P.alpha, P.gain, 1e-6, B.a_saved, B.p_saved, B.rstd, B.H_pre, B.H_post,
+                     dHr, dHp, dHo, B.dx, True, B.dW, B.db, B.dalpha, B.dgain, True)
+    torch.cuda.synchronize()
+    check_f32("dW x2", host(B.dW), 2 * ref["dW"], 1e-3)
+    check_f32("db x2", host(B.db), 2 * ref["db"], 1e-3)
+    check_f32("dalpha x2", host(B.dalpha), 2 * ref["dalpha"], 1e-3)
+    check_f32("dgain x2", host(B.dgain), 2 * ref["dgain"], 1e-3)
+    check_bf16("dx x2", host(B.dx), 2 * ref["dx_coeffs"], rel=3e-2)
+
+
+@pytest.mark.parametrize("T", [0, 1, 2, 31, 33])
+def test_tiny_and_empty_token_counts(T):
+    n, C = 4, 64
+    inp = synth.make_layer_inputs(n, C, max(T, 1), seed=5, bias_std=0.1)
+    if T == 0:
+        from paper_2601_05732_b200.binding import MhcLite
+        ctx = MhcLite(n, C)
+        e = torch.empty(0, device=DEV)
+        # T = 0 is a valid no-op: pointers are not even inspected
+        assert ctx.lib.mhclite_premix_fwd(ctx._h, 0, None, None, None, None) == 0
+        assert ctx.lib.mhclite_postres_fwd(ctx._h, 0, None, None, None, None, None, None) == 0
+        return
+    G = GpuLayer(inp)
+    G.forward(); compare_forward(G, oracle_fwd(inp))
+    G.backward(); compare_backward(G, oracle_bwd(inp))
+
+
+def test_bad_arguments_are_rejected_without_launch():
+    from paper_2601_05732_b200.binding import MhcLite, MhcLiteError, ERR_BAD_ARG, ERR_WORKSPACE
+    n, C, T = 4, 64, 16
+    inp = synth.make_layer_inputs(n, C, T, seed=5)
+    G = GpuLayer(inp)
+    lib, h = G.ctx.lib, G.ctx._h
+    x = G.x.data_ptr()
+    assert lib.mhclite_premix_fwd(h, -1, x, G.B.H_pre.data_ptr(), G.B.u.data_ptr(), None) == ERR_BAD_ARG
+    assert lib.mhclite_premix_fwd(h, T, None, G.B.H_pre.data_ptr(), G.B.u.data_ptr(), None) == ERR_BAD_ARG
+    assert lib.mhclite_premix_fwd(h, T, x + 2, G.B.H_pre.data_ptr(), G.B.u.data_ptr(), None) == ERR_BAD_ARG
+    assert b"aligned" in lib.mhclite_last_error(h)
+    # a context without workspace refuses the calls that need one
+    ctx2 = MhcLite(n, C)
+    B = G.B
+    with pytest.raises(MhcLiteError) as ei:
+        ctx2._check(ctx2.lib.mhclite_coeffs_bwd(
+            ctx2._h, T, x, G.P.W.data_ptr(), G.P.alpha.data_ptr(), G.P.gain.data_ptr(), 1e-6, B.a_saved.data_ptr(),
+            B.p_saved.data_ptr(), B.rstd.data_ptr(), B.H_pre.data_ptr(), B.H_post.data_ptr(), B.dH_res.data_ptr(),
+            B.dH_pre.data_ptr(), B.dH_post.data_ptr(), B.dx.data_ptr(), 0, B.dW.data_ptr(), B.db.data_ptr(),
+            B.dalpha.data_ptr(), B.dgain.data_ptr(), 0, None), "coeffs_bwd")
+    assert ei.value.status == ERR_WORKSPACE
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ SK comparison path (Eq. (2))
+@pytest.mark.parametrize("n,C,T", [(4, 256, 300), (3, 72, 100), (2, 64, 50), (5, 40, 70)])
+def test_sk_path_parity(n, C, T):
+    inp = synth.make_layer_inputs(n, C, T, seed=40 + n, bias_std=0.5, alpha=[1.0, 1.0, 1.0], w_std=0.05, kind="sk")
+    G = GpuLayer(inp, kind="sk")
+    G.forward(); compare_forward(G, oracle_fwd(inp, kind="sk"), coeff_rel=1e-4)
+    G.backward(); compare_backward(G, oracle_bwd(inp, kind="sk"), grad_rel=2e-3, fused=False)
+
+
+def test_sk_gap_vs_lite_on_ill_conditioned_logits():
+    # paper Section 3.1: with a large relative range 1/nu, 20 iterations leave a visible gap; mHC-lite none
+    n, C, T = 4, 256, 4096
+    sk = synth.make_layer_inputs(n, C, T, seed=6, kind="sk")
+    sk["b"][:16] = synth.normal(6, 99, (16,), 10.0).astype(np.float32)
+    G = GpuLayer(sk, kind="sk"); G.forward()
+    ref = oracle_fwd(sk, kind="sk")
+    l1 = torch.empty(T, device=DEV); cd = torch.empty(T, device=DEV)
+    G.ctx.ds_gap(G.B.H_res, l1, cd); torch.cuda.synchronize()
+    gap_ref = O.l1_error(ref["H_res"])
+    assert gap_ref.max() > 1e-3                                   # the oracle sees the gap ...
+    check_f32("l1 gap", host(l1), gap_ref, 1e-2)                  # ... and the GPU path reproduces it
+    check_f32("colsum dev", host(cd), np.abs(O.column_sums(ref["H_res"]) - 1).max(axis=1), 1e-2)
+    lite = synth.make_layer_inputs(n, C, T, seed=6)
+    lite["b"][:24] = synth.normal(6, 98, (24,), 10.0).astype(np.float32)
+    GL = GpuLayer(lite); GL.forward()
+    GL.ctx.ds_gap(GL.B.H_res, l1, cd); torch.cuda.synchronize()
+    assert float(l1.max()) < 4e-6 and float(cd.max()) < 1e-6
