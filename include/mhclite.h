@@ -145,6 +145,30 @@ MHCLITE_API int mhclite_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf
                        float* dW, float* db, float* dalpha, float* dgain, int accumulate_params,
                        void* stream);
 
+/* Allocation-free variant of mhclite_coeffs_bwd (the paper has no counterpart: this is a property of
+ * the library, not of the method).  It is for callers that cannot hand the library a workspace because
+ * they cannot allocate device memory where the call is made: code running inside an allocator or
+ * memory-pool callback, a process with a memory budget fixed at start-up, a plug-in that only ever
+ * sees its inputs and outputs.  Same arguments, same results as mhclite_coeffs_bwd, but the scratch is
+ * a fixed array of mhclite_static_scratch_bytes() bytes inside the library's device image (every GPU
+ * that loads the library holds it until the process exits) and no workspace needs to be attached.
+ *   - Problem sizes whose mhclite_workspace_bytes(n, C, T, 0) exceeds that array are rejected with
+ *     MHCLITE_ERR_WORKSPACE and nothing is launched.
+ *   - The call allocates and frees nothing.  The first call on each device looks up the array's
+ *     device address (a synchronous, one-time set-up): make that first call before any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents; each call
+ *     rewrites or clears every part it reads, so back-to-back calls on one stream are fine, but two
+ *     calls that overlap on the GPU (different streams, different contexts) race on it. */
+MHCLITE_API size_t mhclite_static_scratch_bytes(void);
+MHCLITE_API int mhclite_coeffs_bwd_static(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x,
+                       const float* W, const float* alpha, const float* gain, float eps,
+                       const float* a_saved, const float* p_saved, const float* rstd,
+                       const float* H_pre, const float* H_post,
+                       const float* dH_res, const float* dH_pre, const float* dH_post,
+                       mhclite_bf16* dx, int accumulate_dx,
+                       float* dW, float* db, float* dalpha, float* dgain, int accumulate_params,
+                       void* stream);
+
 /* premix_bwd + coeffs_bwd + the H_res^T g term of postres_bwd, writing the complete dx once:
  *   dx[t,j,c] = sum_i H_res[t,i,j] g[t,i,c] + H_pre[t,j] du[t,c] + (gradient through the mappings).
  * dH_res and dH_post come from a preceding mhclite_postres_bwd call made with dx = NULL. */

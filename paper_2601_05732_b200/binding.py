@@ -45,6 +45,9 @@ SIGNATURES = {
     "mhclite_premix_bwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _i, _p]),
     "mhclite_coeffs_bwd": (_i, [_p, _i64, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p, _p, _i,
                                 _p, _p, _p, _p, _i, _p]),
+    "mhclite_static_scratch_bytes": (_sz, []),
+    "mhclite_coeffs_bwd_static": (_i, [_p, _i64, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p, _p, _i,
+                                       _p, _p, _p, _p, _i, _p]),
     "mhclite_tail_bwd_fused": (_i, [_p, _i64, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p, _p, _p,
                                     _p, _p, _p, _p, _p, _i, _p]),
     "mhc_sk20_coeffs_fwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _i, _p, _p, _p, _p, _p, _p]),
@@ -206,6 +209,18 @@ class MhcLite:
             self._ptr(dH_res, f), self._ptr(dH_pre, f), self._ptr(dH_post, f), self._ptr(dx, h), int(accumulate_dx),
             self._ptr(dW, f), self._ptr(db, f), self._ptr(dalpha, f), self._ptr(dgain, f), int(accumulate_params),
             self._stream()), "mhclite_coeffs_bwd")
+
+    def coeffs_bwd_static(self, x, W, alpha, gain, eps, a_saved, p_saved, rstd, H_pre, H_post, dH_res, dH_pre,
+                          dH_post, dx, accumulate_dx, dW, db, dalpha, dgain, accumulate_params=False):
+        """coeffs_bwd for callers that cannot allocate: scratch is the library's built-in device array
+        (no workspace is attached or touched; sizes beyond the array raise)."""
+        f, h = self._torch.float32, self._torch.bfloat16
+        self._check(self.lib.mhclite_coeffs_bwd_static(
+            self._h, x.shape[0], self._ptr(x, h), self._ptr(W, f), self._ptr(alpha, f), self._ptr(gain, f), float(eps),
+            self._ptr(a_saved, f), self._ptr(p_saved, f), self._ptr(rstd, f), self._ptr(H_pre, f), self._ptr(H_post, f),
+            self._ptr(dH_res, f), self._ptr(dH_pre, f), self._ptr(dH_post, f), self._ptr(dx, h), int(accumulate_dx),
+            self._ptr(dW, f), self._ptr(db, f), self._ptr(dalpha, f), self._ptr(dgain, f), int(accumulate_params),
+            self._stream()), "mhclite_coeffs_bwd_static")
 
     def tail_bwd_fused(self, x, W, alpha, gain, eps, a_saved, p_saved, rstd, H_res, H_pre, H_post, g, du,
                        dH_res, dH_post, dx, dW, db, dalpha, dgain, accumulate_params=False):
