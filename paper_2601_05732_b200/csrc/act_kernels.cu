@@ -20,18 +20,50 @@ constexpr int kMaxCols = kMaxFact + 2 * kMaxN;   // 130
 __device__ __forceinline__ float sigmoidf_(float z) { return 1.f / (1.f + expf(-z)); }
 
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kActThreads) lite_act_fwd_k(int64_t T, int n, int nf, const float* __restrict__ p,
+// Adds the K-slice partials of the projection, applies rstd and stores p_saved / rstd for one token.
+// Returns p for the columns this lane owns: col = lane + 32 s.
+__device__ __forceinline__ void finish_projection(int64_t t, int64_t T, int N, int Npad, int ksplit, float inv_nC,
+                                                  float eps, const float* __restrict__ qpart,
+                                                  const float* __restrict__ ssq, float* __restrict__ p_saved,
+                                                  float* __restrict__ rstd, int lane, float (&pv)[5]) {
+    float ss = 0.f;
+    for (int s = 0; s < ksplit; ++s) ss += __ldg(ssq + (int64_t)s * T + t);
+    const float r = 1.f / sqrtf(ss * inv_nC + eps);
+    if (lane == 0) rstd[t] = r;
+#pragma unroll
+    for (int k = 0; k < 5; ++k) {
+        const int c = lane + 32 * k;
+        pv[k] = 0.f;
+        if (c < N) {
+            float q = 0.f;
+            for (int s = 0; s < ksplit; ++s) q += __ldg(qpart + ((int64_t)s * T + t) * Npad + c);
+            pv[k] = r * q;
+            p_saved[t * N + c] = pv[k];
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kActThreads) lite_act_fwd_k(int64_t T, int n, int nf, int Npad, int ksplit,
+                                                             float inv_nC, float eps, const float* __restrict__ qpart,
+                                                             const float* __restrict__ ssq,
                                                              const float* __restrict__ b, const float* __restrict__ alpha,
                                                              float* __restrict__ H_res, float* __restrict__ H_pre,
-                                                             float* __restrict__ H_post, float* __restrict__ a_saved) {
+                                                             float* __restrict__ H_post, float* __restrict__ a_saved,
+                                                             float* __restrict__ p_saved, float* __restrict__ rstd) {
     __shared__ float a_s[kActWarps][kMaxFact + 8];
+    __shared__ float p_s[kActWarps][kMaxCols + 6];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int N = nf + 2 * n, per = nf / n, nn = n * n;
     const PermTables& tab = c_perm[n];
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
     const int64_t nwarps = (int64_t)gridDim.x * kActWarps;
     for (int64_t t = (int64_t)blockIdx.x * kActWarps + w; t < T; t += nwarps) {
-        const float* pt = p + t * N;
+        float pv[5];
+        finish_projection(t, T, N, Npad, ksplit, inv_nC, eps, qpart, ssq, p_saved, rstd, lane, pv);
+#pragma unroll
+        for (int k = 0; k < 5; ++k) if (lane + 32 * k < N) p_s[w][lane + 32 * k] = pv[k];
+        __syncwarp();
+        const float* pt = p_s[w];
         float z[4], m = -INFINITY;
 #pragma unroll
         for (int s = 0; s < 4; ++s) {
@@ -195,14 +227,27 @@ __device__ __forceinline__ void sk_load_m0(const float* pt, const float* b, floa
 }
 
 template <int N_>
-__global__ void __launch_bounds__(128) sk_act_fwd_k(int64_t T, int iters, const float* __restrict__ p,
+__global__ void __launch_bounds__(128) sk_act_fwd_k(int64_t T, int iters, int Npad, int ksplit, float inv_nC, float eps,
+                                                    const float* __restrict__ qpart, const float* __restrict__ ssq,
                                                     const float* __restrict__ b, const float* __restrict__ alpha,
                                                     float* __restrict__ H_res, float* __restrict__ H_pre,
-                                                    float* __restrict__ H_post) {
+                                                    float* __restrict__ H_post, float* __restrict__ p_saved,
+                                                    float* __restrict__ rstd) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= T) return;
     constexpr int N = N_ * N_ + 2 * N_;
-    const float* pt = p + t * N;
+    float ss = 0.f;
+    for (int s = 0; s < ksplit; ++s) ss += __ldg(ssq + (int64_t)s * T + t);
+    const float r = 1.f / sqrtf(ss * inv_nC + eps);
+    rstd[t] = r;
+    float pt[N];
+#pragma unroll
+    for (int c = 0; c < N; ++c) {
+        float q = 0.f;
+        for (int s = 0; s < ksplit; ++s) q += __ldg(qpart + ((int64_t)s * T + t) * Npad + c);
+        pt[c] = r * q;
+        p_saved[t * N + c] = pt[c];
+    }
     float M[N_][N_];
     sk_load_m0<N_>(pt, b, __ldg(alpha), M);
     sk_forward<N_>(M, iters, nullptr, nullptr);
@@ -316,11 +361,13 @@ static int warp_grid(int64_t T, int sm_count) {
     return (int)(blocks < 1 ? 1 : blocks);
 }
 
-void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const float* p, const float* b, const float* alpha,
-                         float* H_res, float* H_pre, float* H_post, float* a_saved, cudaStream_t s) {
+void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, const float* qpart, const float* ssq,
+                         float eps, const float* b, const float* alpha, float* H_res, float* H_pre, float* H_post,
+                         float* a_saved, float* p_saved, float* rstd, cudaStream_t s) {
     c->launches += 1;
-    lite_act_fwd_k<<<warp_grid(T, c->sm_count), kActThreads, 0, s>>>(T, c->n, c->nfact, p, b, alpha, H_res, H_pre,
-                                                                      H_post, a_saved);
+    lite_act_fwd_k<<<warp_grid(T, c->sm_count), kActThreads, 0, s>>>(
+        T, c->n, c->nfact, pp.Npad, pp.ksplit, 1.f / (float)(c->n * c->C), eps, qpart, ssq, b, alpha, H_res, H_pre,
+        H_post, a_saved, p_saved, rstd);
 }
 
 void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float* a, const float* p, const float* rstd,
@@ -337,11 +384,14 @@ void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float*
                                                         dalpha);
 }
 
-void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const float* p, const float* b, const float* alpha,
-                       float* H_res, float* H_pre, float* H_post, cudaStream_t s) {
+void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,
+                       const float* ssq, float eps, const float* b, const float* alpha, float* H_res, float* H_pre,
+                       float* H_post, float* p_saved, float* rstd, cudaStream_t s) {
     c->launches += 1;
     const int grid = (int)((T + 127) / 128);
-    MHCL_DISPATCH_N(c->n, sk_act_fwd_k<N_><<<grid, 128, 0, s>>>(T, iters, p, b, alpha, H_res, H_pre, H_post));
+    const float inv = 1.f / (float)(c->n * c->C);
+    MHCL_DISPATCH_N(c->n, sk_act_fwd_k<N_><<<grid, 128, 0, s>>>(T, iters, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b,
+                                                                 alpha, H_res, H_pre, H_post, p_saved, rstd));
 }
 
 void launch_sk_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, int iters, const float* p, const float* b,

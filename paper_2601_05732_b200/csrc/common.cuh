@@ -40,12 +40,27 @@ inline int n_cols(int n, int kind) { return n_res_cols(n, kind) + 2 * n; }
 int fail(mhclite_ctx* ctx, int status, const char* fmt, ...);
 int check_cuda(mhclite_ctx* ctx, cudaError_t e, const char* what);
 
-// Workspace layout (all offsets 256-byte aligned). See workspace.cu.
+// Launch plan of the tensor-core projection for one problem size (proj_mma.cu).
+constexpr int kMaxKSplit = 4;
+struct ProjPlan {
+    int NT;                 // 8-column tiles of the padded projection (1..5, or 20)
+    int Npad;               // NT * 8: row length of qpart
+    int nchunks;            // 64-wide K chunks covering nC
+    int ksteps;             // 16-wide MMA k-steps in the packed weights (4 per chunk)
+    int ksplit;             // K slices whose partial results the activation kernel adds
+    int chunks_per_split;
+};
+ProjPlan plan_proj(int n, int C, int64_t T, int N, int sm_count);
+
+// Workspace layout (all offsets 256-byte aligned), see plan_workspace.
 struct Workspace {
     float* e;        // [T][Npad]   rstd * alpha (.) dz, fp32
     float* kappa;    // [T]         rstd^2 * sum_c (alpha dz)_c p_c / (nC)
     float* G;        // [nC][Npad]  sum_t x[t,m] e[t,c] (before the gain factor)
     float* dH_pre;   // [T][n]      <du, x_j> of the fused backward tail
+    void* Wp;        // packed bf16 hi/lo weights in MMA fragment order
+    float* qpart;    // [kMaxKSplit][T][NTpad*8] partial x W' of each K slice
+    float* ssq;      // [kMaxKSplit][T]          partial sums of squares
     size_t bytes;
     int Npad;
 };

@@ -18,9 +18,12 @@ void launch_tail_mix(const mhclite_ctx* c, int64_t T, const void* x, const void*
 void launch_ds_gap(const mhclite_ctx* c, int64_t T, const float* H_res, float* l1, float* cdev, cudaStream_t s);
 
 // proj_kernels.cu : RMSNorm statistics + the skinny projection and its gradient
-// p[t,c] = rstd_t * sum_m x[t,m] gain[m] W[m,c] (c < N), rstd[t]
-void launch_proj_fwd(const mhclite_ctx* c, int64_t T, int N, const void* x, const float* W, const float* gain,
-                     float eps, float* p, float* rstd, cudaStream_t s);
+// proj_mma.cu: W' = diag(gain) W packed as bf16 hi/lo MMA fragments; qpart[s][t][c] = partial x W' of K slice s,
+// ssq[s][t] = partial sum of squares (the activation kernels add the slices and apply rstd)
+void launch_pack_w(const mhclite_ctx* c, const ProjPlan& p, int N, const float* W, const float* gain, void* Wp,
+                   cudaStream_t s);
+void launch_proj_fwd_mma(const mhclite_ctx* c, int64_t T, const ProjPlan& p, const void* x, const void* Wp,
+                         float* qpart, float* ssq, cudaStream_t s);
 // dx[t,m] (+)= sum_c e[t,c] gain[m] W[m,c] - x[t,m] kappa[t]   (e = rstd*alpha*dz)
 void launch_proj_bwd_dx(const mhclite_ctx* c, int64_t T, int N, int Npad, const void* x, const float* W,
                         const float* gain, const float* e, const float* kappa, void* dx, int acc, cudaStream_t s);
@@ -30,14 +33,16 @@ void launch_proj_bwd_dw(const mhclite_ctx* c, int64_t T, int N, int Npad, const 
                         cudaStream_t s);
 
 // act_kernels.cu : per-token activations, H_res assembly and their gradients
-void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const float* p, const float* b, const float* alpha,
-                         float* H_res, float* H_pre, float* H_post, float* a_saved, cudaStream_t s);
+void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, const float* qpart, const float* ssq,
+                         float eps, const float* b, const float* alpha, float* H_res, float* H_pre, float* H_post,
+                         float* a_saved, float* p_saved, float* rstd, cudaStream_t s);
 void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float* a, const float* p, const float* rstd,
                          const float* alpha, const float* H_pre, const float* H_post, const float* dH_res,
                          const float* dH_pre, const float* dH_post, float* e, float* kappa, float* db,
                          float* dalpha, cudaStream_t s);
-void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const float* p, const float* b, const float* alpha,
-                       float* H_res, float* H_pre, float* H_post, cudaStream_t s);
+void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,
+                       const float* ssq, float eps, const float* b, const float* alpha, float* H_res, float* H_pre,
+                       float* H_post, float* p_saved, float* rstd, cudaStream_t s);
 void launch_sk_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, int iters, const float* p, const float* b,
                        const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
                        const float* dH_res, const float* dH_pre, const float* dH_post, float* e, float* kappa,

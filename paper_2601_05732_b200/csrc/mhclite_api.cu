@@ -34,6 +34,10 @@ Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base) {
     w.kappa = (float*)(p + off); off += align256((size_t)T * sizeof(float));
     w.G = (float*)(p + off);     off += align256((size_t)n * C * w.Npad * sizeof(float));
     w.dH_pre = (float*)(p + off); off += align256((size_t)T * n * sizeof(float));
+    const ProjPlan pp = plan_proj(n, C, T, N, 148);          // sizes do not depend on the SM count
+    w.Wp = p + off;              off += align256((size_t)pp.ksteps * pp.NT * 32 * 16);
+    w.qpart = (float*)(p + off); off += align256((size_t)kMaxKSplit * T * pp.Npad * sizeof(float));
+    w.ssq = (float*)(p + off);   off += align256((size_t)kMaxKSplit * T * sizeof(float));
     w.bytes = off;
     return w;
 }
@@ -160,11 +164,18 @@ int mhclite_coeffs_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, a_saved);
     MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd);
     if (!(eps >= 0.f)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "eps must be >= 0");
+    Workspace w;
+    int rc = need_workspace(ctx, T, 0, &w);
+    if (rc) return rc;
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
-    launch_proj_fwd(ctx, T, n_cols(ctx->n, 0), x, W, gain, eps, p_saved, rstd, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_fwd");
-    launch_lite_act_fwd(ctx, T, p_saved, b, alpha, H_res, H_pre, H_post, a_saved, s);
+    const int N = n_cols(ctx->n, 0);
+    const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
+    launch_pack_w(ctx, pp, N, W, gain, w.Wp, s);
+    MHCL_LAUNCH_CHECK(ctx, "pack_w");
+    launch_proj_fwd_mma(ctx, T, pp, x, w.Wp, w.qpart, w.ssq, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_fwd_mma");
+    launch_lite_act_fwd(ctx, T, pp, w.qpart, w.ssq, eps, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_act_fwd");
     return MHCLITE_OK;
 }
@@ -306,11 +317,18 @@ int mhc_sk20_coeffs_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
     MHCL_PTR(ctx, x); MHCL_PTR(ctx, W_sk); MHCL_PTR(ctx, b_sk); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain);
     MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd);
     if (!(eps >= 0.f)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "eps must be >= 0");
+    Workspace w;
+    int rc = need_workspace(ctx, T, 1, &w);
+    if (rc) return rc;
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
-    launch_proj_fwd(ctx, T, n_cols(ctx->n, 1), x, W_sk, gain, eps, p_saved, rstd, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_fwd");
-    launch_sk_act_fwd(ctx, T, iters, p_saved, b_sk, alpha, H_res, H_pre, H_post, s);
+    const int N = n_cols(ctx->n, 1);
+    const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
+    launch_pack_w(ctx, pp, N, W_sk, gain, w.Wp, s);
+    MHCL_LAUNCH_CHECK(ctx, "pack_w");
+    launch_proj_fwd_mma(ctx, T, pp, x, w.Wp, w.qpart, w.ssq, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_fwd_mma");
+    launch_sk_act_fwd(ctx, T, iters, pp, w.qpart, w.ssq, eps, b_sk, alpha, H_res, H_pre, H_post, p_saved, rstd, s);
     MHCL_LAUNCH_CHECK(ctx, "sk_act_fwd");
     return MHCLITE_OK;
 }

@@ -1,83 +1,11 @@
-// RMSNorm statistics and the skinny projection of paper Eq. (4), with its gradient -- CUDA-core
-// (fp32 FMA) version.  The flattened token x[t, 0..nC) is contracted with W' = diag(gain) W:
-//   p[t,c]  = rstd_t * sum_m x[t,m] W'[m,c]                 rstd_t = (mean_m x^2 + eps)^(-1/2)
+// Gradient of the skinny projection of paper Eq. (4) and of RMSNorm -- CUDA-core (fp32 FMA) version.
+// With W' = diag(gain) W:
 //   dx[t,m] (+)= sum_c e[t,c] W'[m,c] - x[t,m] kappa_t       (e, kappa from the activation backward)
 //   G[m,c]  = sum_t x[t,m] e[t,c] ; dW = gain (.) G ; dgain[m] = sum_c W[m,c] G[m,c]
 #include "common.cuh"
 #include "kernels.h"
 
 namespace mhcl {
-
-// ------------------------------------------------------------------------------------------------
-// forward: 32 tokens per block, k-chunks of 32 staged in shared memory
-// ------------------------------------------------------------------------------------------------
-constexpr int kPfTok = 32, kPfK = 32, kPfThreads = 256, kPfSlots = 5;   // 5*32 >= 130 columns
-
-__global__ void __launch_bounds__(kPfThreads) proj_fwd_k(int64_t T, int nC, int N, float eps,
-                                                         const __nv_bfloat16* __restrict__ x, const float* __restrict__ W,
-                                                         const float* __restrict__ gain, float* __restrict__ p,
-                                                         float* __restrict__ rstd) {
-    __shared__ float xs[kPfTok][kPfK + 1];
-    __shared__ float ws[kPfK][kPfSlots * 32];
-    __shared__ float ssq[kPfTok];
-    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    const int64_t t0 = (int64_t)blockIdx.x * kPfTok;
-    const int slots = (N + 31) / 32;
-    float acc[4][kPfSlots];
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int s = 0; s < kPfSlots; ++s) acc[a][s] = 0.f;
-    float sq = 0.f;
-    const int lt = tid >> 2, lp = tid & 3;        // loader: token lt, 16-byte piece lp (threads 0..127)
-    for (int k0 = 0; k0 < nC; k0 += kPfK) {
-        if (tid < 128) {
-            float f[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-            const int64_t t = t0 + lt;
-            const int m = k0 + lp * 8;
-            if (t < T && m < nC) unpack8(*reinterpret_cast<const uint4*>(x + t * nC + m), f);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) { xs[lt][lp * 8 + e] = f[e]; sq = fmaf(f[e], f[e], sq); }
-        }
-        for (int i = tid; i < kPfK * slots * 32; i += kPfThreads) {
-            const int k = i / (slots * 32), c = i - k * (slots * 32);
-            const int m = k0 + k;
-            ws[k][c] = (m < nC && c < N) ? __ldg(W + (int64_t)m * N + c) * __ldg(gain + m) : 0.f;
-        }
-        __syncthreads();
-#pragma unroll 4
-        for (int k = 0; k < kPfK; ++k) {
-            float wv[kPfSlots];
-#pragma unroll
-            for (int s = 0; s < kPfSlots; ++s) wv[s] = (s < slots) ? ws[k][lane + 32 * s] : 0.f;
-#pragma unroll
-            for (int a = 0; a < 4; ++a) {
-                const float xv = xs[4 * w + a][k];
-#pragma unroll
-                for (int s = 0; s < kPfSlots; ++s) acc[a][s] = fmaf(xv, wv[s], acc[a][s]);
-            }
-        }
-        __syncthreads();
-    }
-    if (tid < 128) {
-        sq += __shfl_xor_sync(0xffffffffu, sq, 1);
-        sq += __shfl_xor_sync(0xffffffffu, sq, 2);
-        if (lp == 0) ssq[lt] = sq;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int a = 0; a < 4; ++a) {
-        const int64_t t = t0 + 4 * w + a;
-        if (t >= T) continue;
-        const float r = 1.f / sqrtf(ssq[4 * w + a] / (float)nC + eps);
-        if (lane == 0) rstd[t] = r;
-#pragma unroll
-        for (int s = 0; s < kPfSlots; ++s) {
-            const int c = lane + 32 * s;
-            if (c < N) p[t * N + c] = r * acc[a][s];
-        }
-    }
-}
 
 // ------------------------------------------------------------------------------------------------
 // backward w.r.t. x: tile of 64 tokens x 64 flattened channels, columns in chunks of 32
@@ -214,13 +142,6 @@ __global__ void __launch_bounds__(256) proj_bwd_finish_k(int nC, int N, int Npad
 }
 
 // ---- launchers -----------------------------------------------------------------------------------
-void launch_proj_fwd(const mhclite_ctx* c, int64_t T, int N, const void* x, const float* W, const float* gain,
-                     float eps, float* p, float* rstd, cudaStream_t s) {
-    c->launches += 1;
-    const int grid = (int)((T + kPfTok - 1) / kPfTok);
-    proj_fwd_k<<<grid, kPfThreads, 0, s>>>(T, c->n * c->C, N, eps, (const __nv_bfloat16*)x, W, gain, p, rstd);
-}
-
 void launch_proj_bwd_dx(const mhclite_ctx* c, int64_t T, int N, int Npad, const void* x, const float* W,
                         const float* gain, const float* e, const float* kappa, void* dx, int acc, cudaStream_t s) {
     c->launches += 1;

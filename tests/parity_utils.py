@@ -4,7 +4,10 @@ inputs, and compare element by element with the stated tolerances.
 Tolerances (they follow the arithmetic: bf16 storage rounds to 2^-9 relative, fp32 accumulation over
 n*C <= 2^15 terms leaves ~1e-6 relative):
   bf16 tensors : |gpu - ref| <= 2e-2 |ref| + 1e-3 rms(ref)          for every element
-  fp32 mappings: |gpu - ref| <= 1e-5 max(|ref|, rms(ref))           (H_res, H_pre, H_post, a, p, rstd)
+  fp32 mappings: |gpu - ref| <= 1e-5 max(|ref|, rms(ref))           (H_res, H_pre, H_post, a, rstd)
+  saved projection p = x' W: 4e-5 max(|ref|, rms(ref)) -- W' enters the tensor cores as a bf16 pair
+                hi + lo, which leaves up to 2^-18 relative error per weight (about 1e-5 of rms(p) in the
+                tails); alpha scales it down by 100x before it reaches the mappings
   fp32 parameter gradients: |gpu - ref| <= 1e-3 max(|ref|, rms(ref)) (the binding tolerance is 2e-2)
 """
 import numpy as np
@@ -88,7 +91,7 @@ def oracle_bwd(inp, eps=1e-6, kind="lite", iters=20):
 def compare_forward(G, ref, coeff_rel=1e-5):
     B = G.B
     check_f32("rstd", host(B.rstd), ref["rstd"], coeff_rel)
-    check_f32("p_saved", host(B.p_saved), ref["p"], coeff_rel)
+    check_f32("p_saved", host(B.p_saved), ref["p"], max(coeff_rel, 4e-5))
     if G.kind == "lite":
         check_f32("a_saved", host(B.a_saved), ref["a"], coeff_rel)
     check_f32("H_res", host(B.H_res), ref["H_res"], coeff_rel)
