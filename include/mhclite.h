@@ -152,8 +152,9 @@ MHCLITE_API int mhclite_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf
  * sees its inputs and outputs.  Same arguments, same results as mhclite_coeffs_bwd, but the scratch is
  * a fixed array of mhclite_static_scratch_bytes() bytes inside the library's device image (every GPU
  * that loads the library holds it until the process exits) and no workspace needs to be attached.
- *   - Problem sizes whose mhclite_workspace_bytes(n, C, T, 0) exceeds that array are rejected with
- *     MHCLITE_ERR_WORKSPACE and nothing is launched.
+ *   - The call needs about 4 * (T * Np + T + n * C * Np) bytes of it, Np = n!+2n rounded up to 8;
+ *     problem sizes that need more than the array holds are rejected with MHCLITE_ERR_WORKSPACE
+ *     and nothing is launched.
  *   - The call allocates and frees nothing.  The first call on each device looks up the array's
  *     device address (a synchronous, one-time set-up): make that first call before any stream capture.
  *   - All calls on a device share the one array and it keeps the previous call's contents; each call

@@ -10,8 +10,32 @@
 // normalisers and walks the iterates back (X = Y * s), instead of keeping every iterate.
 #include "common.cuh"
 #include "kernels.h"
+#include "mma.cuh"
 
 namespace mhcl {
+
+// Where the activation backward leaves e = rstd * alpha (.) dz for the projection backward: as fp32 rows
+// (CUDA-core kernels) and / or as a bf16 pair hi + lo (tensor-core kernel).  Null pointers are skipped.
+struct EOut {
+    float* e; int Npad;
+    __nv_bfloat16 *ehi, *elo; int Kp;
+};
+__device__ __forceinline__ void store_e(const EOut& o, int64_t t, int c, float v) {
+    if (o.e) o.e[t * o.Npad + c] = v;
+    if (o.ehi) {
+        __nv_bfloat16 h, l;
+        split_bf16(v, h, l);
+        o.ehi[t * o.Kp + c] = h;
+        o.elo[t * o.Kp + c] = l;
+    }
+}
+__device__ __forceinline__ void pad_e(const EOut& o, int64_t t, int N, int first, int step) {
+    if (o.e) for (int c = N + first; c < o.Npad; c += step) o.e[t * o.Npad + c] = 0.f;
+    if (o.ehi) for (int c = N + first; c < o.Kp; c += step) {
+        o.ehi[t * o.Kp + c] = __float2bfloat16_rn(0.f);
+        o.elo[t * o.Kp + c] = __float2bfloat16_rn(0.f);
+    }
+}
 
 constexpr int kActThreads = 256;
 constexpr int kActWarps = kActThreads / 32;
@@ -107,10 +131,10 @@ __global__ void __launch_bounds__(kActThreads) lite_act_fwd_k(int64_t T, int n, 
 // Shared tail of both backward kernels: from dz of one column to e, kappa, db, dalpha partials.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kActThreads) lite_act_bwd_k(
-    int64_t T, int n, int nf, int Npad, float inv_nC, const float* __restrict__ a_saved, const float* __restrict__ p,
+    int64_t T, int n, int nf, float inv_nC, const float* __restrict__ a_saved, const float* __restrict__ p,
     const float* __restrict__ rstd, const float* __restrict__ alpha, const float* __restrict__ H_pre,
     const float* __restrict__ H_post, const float* __restrict__ dH_res, const float* __restrict__ dH_pre,
-    const float* __restrict__ dH_post, float* __restrict__ e, float* __restrict__ kappa, float* db, float* dalpha) {
+    const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa, float* db, float* dalpha) {
     __shared__ float dh_s[kActWarps][32];
     __shared__ float red[kActWarps][kMaxCols + 3];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -139,14 +163,13 @@ __global__ void __launch_bounds__(kActThreads) lite_act_bwd_k(
         }
         dot = warp_sum(dot);
         float kap = 0.f;
-        float* et = e + t * Npad;
 #pragma unroll
         for (int s = 0; s < 4; ++s) {
             const int k = lane + 32 * s;
             if (k < nf) {
                 const float dz = a[s] * (da[s] - dot);
                 const float ed = a_res * dz, pv = pt[k];
-                et[k] = rs * ed;
+                store_e(eo, t, k, rs * ed);
                 kap = fmaf(ed, pv, kap);
                 db_res[s] += dz;
                 dal_res = fmaf(dz, pv, dal_res);
@@ -158,12 +181,12 @@ __global__ void __launch_bounds__(kActThreads) lite_act_bwd_k(
             if (lane < n) { const float h = H_pre[t * n + lane]; dz = dH_pre[t * n + lane] * h * (1.f - h); }
             else { const float h = H_post[t * n + lane - n]; dz = dH_post[t * n + lane - n] * h * (1.f - 0.5f * h); }
             const float ed = (lane < n ? a_pre : a_post) * dz, pv = pt[c];
-            et[c] = rs * ed;
+            store_e(eo, t, c, rs * ed);
             kap = fmaf(ed, pv, kap);
             db_gate += dz;
             dal_gate = fmaf(dz, pv, dal_gate);
         }
-        for (int c = N + lane; c < Npad; c += 32) et[c] = 0.f;
+        pad_e(eo, t, N, lane, 32);
         kap = warp_sum(kap);
         if (lane == 0) kappa[t] = rs * rs * kap * inv_nC;
         __syncwarp();
@@ -267,10 +290,10 @@ constexpr int kSkMaxIters = 64;
 
 template <int N_>
 __global__ void __launch_bounds__(128) sk_act_bwd_k(
-    int64_t T, int Npad, int iters, float inv_nC, const float* __restrict__ p, const float* __restrict__ b,
+    int64_t T, int iters, float inv_nC, const float* __restrict__ p, const float* __restrict__ b,
     const float* __restrict__ rstd, const float* __restrict__ alpha, const float* __restrict__ H_pre,
     const float* __restrict__ H_post, const float* __restrict__ dH_res, const float* __restrict__ dH_pre,
-    const float* __restrict__ dH_post, float* __restrict__ e, float* __restrict__ kappa, float* db, float* dalpha) {
+    const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa, float* db, float* dalpha) {
     constexpr int N = N_ * N_ + 2 * N_;
     __shared__ float red[N + 3];
     for (int c = threadIdx.x; c < N + 3; c += blockDim.x) red[c] = 0.f;
@@ -314,14 +337,13 @@ __global__ void __launch_bounds__(128) sk_act_bwd_k(
         sk_load_m0<N_>(pt, b, a_res, Y);
         const float r = __ldg(rstd + t);
         float kap = 0.f, dal0 = 0.f, dal1 = 0.f, dal2 = 0.f;
-        float* et = e + t * Npad;
 #pragma unroll
         for (int i = 0; i < N_; ++i)
 #pragma unroll
             for (int j = 0; j < N_; ++j) {
                 const int c = i * N_ + j;
                 const float dz = d[i][j] * Y[i][j], pv = pt[c], ed = a_res * dz;
-                et[c] = r * ed;
+                store_e(eo, t, c, r * ed);
                 kap = fmaf(ed, pv, kap);
                 dal0 = fmaf(dz, pv, dal0);
                 atomicAdd(&red[c], dz);
@@ -332,18 +354,18 @@ __global__ void __launch_bounds__(128) sk_act_bwd_k(
                 const int c = N_ * N_ + j;
                 const float h = H_pre[t * N_ + j];
                 const float dz = dH_pre[t * N_ + j] * h * (1.f - h), pv = pt[c], ed = a_pre * dz;
-                et[c] = r * ed; kap = fmaf(ed, pv, kap); dal1 = fmaf(dz, pv, dal1);
+                store_e(eo, t, c, r * ed); kap = fmaf(ed, pv, kap); dal1 = fmaf(dz, pv, dal1);
                 atomicAdd(&red[c], dz);
             }
             {
                 const int c = N_ * N_ + N_ + j;
                 const float h = H_post[t * N_ + j];
                 const float dz = dH_post[t * N_ + j] * h * (1.f - 0.5f * h), pv = pt[c], ed = a_post * dz;
-                et[c] = r * ed; kap = fmaf(ed, pv, kap); dal2 = fmaf(dz, pv, dal2);
+                store_e(eo, t, c, r * ed); kap = fmaf(ed, pv, kap); dal2 = fmaf(dz, pv, dal2);
                 atomicAdd(&red[c], dz);
             }
         }
-        for (int c = N; c < Npad; ++c) et[c] = 0.f;
+        pad_e(eo, t, N, 0, 1);
         kappa[t] = r * r * kap * inv_nC;
         atomicAdd(&red[N], dal0); atomicAdd(&red[N + 1], dal1); atomicAdd(&red[N + 2], dal2);
     }
@@ -372,15 +394,16 @@ void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, co
 
 void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float* a, const float* p, const float* rstd,
                          const float* alpha, const float* H_pre, const float* H_post, const float* dH_res,
-                         const float* dH_pre, const float* dH_post, float* e, float* kappa, float* db,
-                         float* dalpha, cudaStream_t s) {
+                         const float* dH_pre, const float* dH_post, float* e, void* ehi, void* elo, int Kp,
+                         float* kappa, float* db, float* dalpha, cudaStream_t s) {
+    const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
     c->launches += 1;
     // fewer, longer-lived blocks: the parameter-gradient partials are reduced once per block
     int64_t blocks = (T + kActWarps * 8 - 1) / (kActWarps * 8);
     if (blocks > c->sm_count * 4) blocks = c->sm_count * 4;
     if (blocks < 1) blocks = 1;
-    lite_act_bwd_k<<<(int)blocks, kActThreads, 0, s>>>(T, c->n, c->nfact, Npad, 1.f / (float)(c->n * c->C), a, p, rstd,
-                                                        alpha, H_pre, H_post, dH_res, dH_pre, dH_post, e, kappa, db,
+    lite_act_bwd_k<<<(int)blocks, kActThreads, 0, s>>>(T, c->n, c->nfact, 1.f / (float)(c->n * c->C), a, p, rstd,
+                                                        alpha, H_pre, H_post, dH_res, dH_pre, dH_post, eo, kappa, db,
                                                         dalpha);
 }
 
@@ -396,13 +419,14 @@ void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const ProjPla
 
 void launch_sk_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, int iters, const float* p, const float* b,
                        const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
-                       const float* dH_res, const float* dH_pre, const float* dH_post, float* e, float* kappa,
-                       float* db, float* dalpha, cudaStream_t s) {
+                       const float* dH_res, const float* dH_pre, const float* dH_post, float* e, void* ehi, void* elo,
+                       int Kp, float* kappa, float* db, float* dalpha, cudaStream_t s) {
+    const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
     c->launches += 1;
     const int grid = (int)((T + 127) / 128);
     const float inv = 1.f / (float)(c->n * c->C);
-    MHCL_DISPATCH_N(c->n, sk_act_bwd_k<N_><<<grid, 128, 0, s>>>(T, Npad, iters, inv, p, b, rstd, alpha, H_pre, H_post,
-                                                                  dH_res, dH_pre, dH_post, e, kappa, db, dalpha));
+    MHCL_DISPATCH_N(c->n, sk_act_bwd_k<N_><<<grid, 128, 0, s>>>(T, iters, inv, p, b, rstd, alpha, H_pre, H_post,
+                                                                  dH_res, dH_pre, dH_post, eo, kappa, db, dalpha));
 }
 
 }  // namespace mhcl

@@ -52,6 +52,15 @@ struct ProjPlan {
 };
 ProjPlan plan_proj(int n, int C, int64_t T, int N, int sm_count);
 
+// Launch plan of the tensor-core backward tail (tail_mma.cu).
+struct TailPlan {
+    int Kp, KS;             // projection columns padded to 16, and Kp / 16
+    int slices, splits;     // 64-channel slices x token ranges = the grid
+    int64_t tok_per_split;  // multiple of 32
+    bool supported;         // KS <= 3 (N <= 48); wider projections use the CUDA-core kernels
+};
+TailPlan plan_tail(int n, int C, int64_t T, int N, int sm_count);
+
 // Workspace layout (all offsets 256-byte aligned), see plan_workspace.
 struct Workspace {
     float* e;        // [T][Npad]   rstd * alpha (.) dz, fp32
@@ -61,6 +70,8 @@ struct Workspace {
     void* Wp;        // packed bf16 hi/lo weights in MMA fragment order
     float* qpart;    // [kMaxKSplit][T][NTpad*8] partial x W' of each K slice
     float* ssq;      // [kMaxKSplit][T]          partial sums of squares
+    void *ehi, *elo; // [T rounded up to 32][Kp] bf16 pair hi + lo = e
+    float* Gpart;    // [splits][nC][Kp] partial G of each token range
     size_t bytes;
     int Npad;
 };

@@ -38,14 +38,20 @@ void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, co
                          float* a_saved, float* p_saved, float* rstd, cudaStream_t s);
 void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float* a, const float* p, const float* rstd,
                          const float* alpha, const float* H_pre, const float* H_post, const float* dH_res,
-                         const float* dH_pre, const float* dH_post, float* e, float* kappa, float* db,
-                         float* dalpha, cudaStream_t s);
+                         const float* dH_pre, const float* dH_post, float* e, void* ehi, void* elo, int Kp,
+                         float* kappa, float* db, float* dalpha, cudaStream_t s);
 void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,
                        const float* ssq, float eps, const float* b, const float* alpha, float* H_res, float* H_pre,
                        float* H_post, float* p_saved, float* rstd, cudaStream_t s);
 void launch_sk_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, int iters, const float* p, const float* b,
                        const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
-                       const float* dH_res, const float* dH_pre, const float* dH_post, float* e, float* kappa,
-                       float* db, float* dalpha, cudaStream_t s);
+                       const float* dH_res, const float* dH_pre, const float* dH_post, float* e, void* ehi, void* elo,
+                       int Kp, float* kappa, float* db, float* dalpha, cudaStream_t s);
+
+// tail_mma.cu : tensor-core projection / RMSNorm backward, optionally fused with the rest of dx (g != NULL)
+void launch_tail_mma(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, const void* x, const void* g,
+                     const void* du, const void* ehi, const void* elo, const float* kappa, const float* H_res,
+                     const float* H_pre, const float* W, const float* gain, void* dx, int acc_dx, float* Gpart,
+                     float* dW, float* dgain, int acc_params, cudaStream_t s);
 
 }  // namespace mhcl

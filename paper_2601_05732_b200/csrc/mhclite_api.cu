@@ -38,6 +38,11 @@ Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base) {
     w.Wp = p + off;              off += align256((size_t)pp.ksteps * pp.NT * 32 * 16);
     w.qpart = (float*)(p + off); off += align256((size_t)kMaxKSplit * T * pp.Npad * sizeof(float));
     w.ssq = (float*)(p + off);   off += align256((size_t)kMaxKSplit * T * sizeof(float));
+    const TailPlan tp = plan_tail(n, C, T, N, 148);
+    const size_t erows = (size_t)round_up64(T, 32);
+    w.ehi = p + off;             off += align256(erows * tp.Kp * 2);
+    w.elo = p + off;             off += align256(erows * tp.Kp * 2);
+    w.Gpart = (float*)(p + off); off += align256(tp.supported ? (size_t)tp.splits * n * C * tp.Kp * sizeof(float) : 0);
     w.bytes = off;
     return w;
 }
@@ -81,6 +86,31 @@ static int need_workspace(mhclite_ctx* ctx, int64_t T, int kind, Workspace* w) {
     if (!ctx->ws || ctx->ws_bytes < need)
         return fail(ctx, MHCLITE_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu attached", need, ctx->ws ? ctx->ws_bytes : (size_t)0);
     *w = plan_workspace(ctx->n, ctx->C, T, kind, ctx->ws);
+    return MHCLITE_OK;
+}
+
+// The part of the backward shared by every entry point, after the activation backward has produced e and
+// kappa: projection / RMSNorm backward into dx (fused with H_res^T g + H_pre du when g is given) and the
+// parameter gradients dW, dgain.  Tensor cores when the projection is narrow enough, CUDA cores otherwise.
+static int proj_backward(mhclite_ctx* ctx, int64_t T, int N, const Workspace& w, const TailPlan& tp,
+                         const mhclite_bf16* x, const mhclite_bf16* g, const mhclite_bf16* du, const float* H_res,
+                         const float* H_pre, const float* W, const float* gain, mhclite_bf16* dx, int accumulate_dx,
+                         float* dW, float* dgain, int accumulate_params, cudaStream_t s) {
+    if (tp.supported) {
+        launch_tail_mma(ctx, T, N, tp, x, g, du, w.ehi, w.elo, w.kappa, H_res, H_pre, W, gain, dx, accumulate_dx,
+                        w.Gpart, dW, dgain, accumulate_params, s);
+        MHCL_LAUNCH_CHECK(ctx, "tail_mma");
+        return MHCLITE_OK;
+    }
+    if (g) {
+        launch_tail_mix(ctx, T, x, g, du, H_res, H_pre, nullptr, dx, s);
+        MHCL_LAUNCH_CHECK(ctx, "tail_mix");
+        accumulate_dx = 1;
+    }
+    launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W, gain, w.e, w.kappa, dx, accumulate_dx, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dx");
+    launch_proj_bwd_dw(ctx, T, N, w.Npad, x, W, gain, w.e, w.G, dW, dgain, accumulate_params, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dw");
     return MHCLITE_OK;
 }
 
@@ -265,14 +295,12 @@ int mhclite_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     const int N = n_cols(ctx->n, 0);
     rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
     if (rc) return rc;
-    launch_lite_act_bwd(ctx, T, w.Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post, w.e,
-                        w.kappa, db, dalpha, s);
+    const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
+    launch_lite_act_bwd(ctx, T, w.Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post,
+                        tp.supported ? nullptr : w.e, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_act_bwd");
-    launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W, gain, w.e, w.kappa, dx, accumulate_dx, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dx");
-    launch_proj_bwd_dw(ctx, T, N, w.Npad, x, W, gain, w.e, w.G, dW, dgain, accumulate_params, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dw");
-    return MHCLITE_OK;
+    return proj_backward(ctx, T, N, w, tp, x, nullptr, nullptr, nullptr, nullptr, W, gain, dx, accumulate_dx, dW, dgain,
+                         accumulate_params, s);
 }
 
 int mhclite_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W, const float* alpha,
@@ -295,16 +323,13 @@ int mhclite_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, c
     const int N = n_cols(ctx->n, 0);
     rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
     if (rc) return rc;
-    launch_tail_mix(ctx, T, x, g, du, H_res, H_pre, w.dH_pre, dx, s);
-    MHCL_LAUNCH_CHECK(ctx, "tail_mix");
-    launch_lite_act_bwd(ctx, T, w.Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, w.dH_pre, dH_post, w.e,
-                        w.kappa, db, dalpha, s);
+    const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
+    launch_premix_bwd(ctx, T, x, H_pre, du, w.dH_pre, nullptr, 0, s);
+    MHCL_LAUNCH_CHECK(ctx, "premix_bwd");
+    launch_lite_act_bwd(ctx, T, w.Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, w.dH_pre, dH_post,
+                        tp.supported ? nullptr : w.e, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_act_bwd");
-    launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W, gain, w.e, w.kappa, dx, 1, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dx");
-    launch_proj_bwd_dw(ctx, T, N, w.Npad, x, W, gain, w.e, w.G, dW, dgain, accumulate_params, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dw");
-    return MHCLITE_OK;
+    return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W, gain, dx, 0, dW, dgain, accumulate_params, s);
 }
 
 // ---- SK comparison path --------------------------------------------------------------------------
@@ -354,14 +379,12 @@ int mhc_sk20_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
     const int N = n_cols(ctx->n, 1);
     rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
     if (rc) return rc;
-    launch_sk_act_bwd(ctx, T, w.Npad, iters, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post, w.e,
-                      w.kappa, db, dalpha, s);
+    const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
+    launch_sk_act_bwd(ctx, T, w.Npad, iters, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post,
+                      tp.supported ? nullptr : w.e, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "sk_act_bwd");
-    launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W_sk, gain, w.e, w.kappa, dx, accumulate_dx, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dx");
-    launch_proj_bwd_dw(ctx, T, N, w.Npad, x, W_sk, gain, w.e, w.G, dW, dgain, accumulate_params, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dw");
-    return MHCLITE_OK;
+    return proj_backward(ctx, T, N, w, tp, x, nullptr, nullptr, nullptr, nullptr, W_sk, gain, dx, accumulate_dx, dW,
+                         dgain, accumulate_params, s);
 }
 
 int mhclite_ds_gap(mhclite_ctx* ctx, int64_t T, const float* H_res, float* l1_err, float* colsum_dev, void* stream) {

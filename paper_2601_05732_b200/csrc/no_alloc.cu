@@ -60,7 +60,11 @@ int mhclite_coeffs_bwd_static(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x
     for (const void* p : ptrs)
         if (!p || ((uintptr_t)p & 15)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "null or misaligned pointer");
     if (ctx->device >= kMaxDevices) return fail(ctx, MHCLITE_ERR_BAD_ARG, "device index %d not supported", ctx->device);
-    const size_t need = plan_workspace(ctx->n, ctx->C, T, 0, nullptr).bytes;
+    // scratch of this call: e [T][Npad], kappa [T], G [nC][Npad] (fp32), each 256-byte aligned
+    const int N = n_cols(ctx->n, 0), Npad = round_up(N, 8), nC = ctx->n * ctx->C;
+    auto up256 = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    const size_t o_kappa = up256((size_t)T * Npad * 4), o_G = o_kappa + up256((size_t)T * 4);
+    const size_t need = o_G + up256((size_t)nC * Npad * 4);
     if (need > kStaticScratchBytes)
         return fail(ctx, MHCLITE_ERR_WORKSPACE,
                     "mhclite_coeffs_bwd_static: n=%d C=%d T=%lld needs %zu bytes of scratch, the built-in array holds "
@@ -74,9 +78,10 @@ int mhclite_coeffs_bwd_static(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x
     void* base = nullptr;
     int rc = check_cuda(ctx, static_scratch_address(ctx->device, &base), "cudaGetSymbolAddress(static scratch)");
     if (rc == MHCLITE_OK) {
-        const Workspace w = plan_workspace(ctx->n, ctx->C, T, 0, base);
+        float* e = (float*)base;
+        float* kappa = (float*)((char*)base + o_kappa);
+        float* G = (float*)((char*)base + o_G);
         cudaStream_t s = (cudaStream_t)stream;
-        const int N = n_cols(ctx->n, 0);
         if (!accumulate_params) {
             rc = check_cuda(ctx, cudaMemsetAsync(db, 0, (size_t)N * sizeof(float), s), "memset db");
             if (rc == MHCLITE_OK) rc = check_cuda(ctx, cudaMemsetAsync(dalpha, 0, 3 * sizeof(float), s), "memset dalpha");
@@ -84,10 +89,10 @@ int mhclite_coeffs_bwd_static(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x
         if (rc == MHCLITE_OK) {
             // every region of the array that the kernels read is written first within this call: e and
             // kappa by the activation backward, G by a memset inside launch_proj_bwd_dw
-            launch_lite_act_bwd(ctx, T, w.Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post,
-                                w.e, w.kappa, db, dalpha, s);
-            launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W, gain, w.e, w.kappa, dx, accumulate_dx, s);
-            launch_proj_bwd_dw(ctx, T, N, w.Npad, x, W, gain, w.e, w.G, dW, dgain, accumulate_params, s);
+            launch_lite_act_bwd(ctx, T, Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post,
+                                e, nullptr, nullptr, 0, kappa, db, dalpha, s);
+            launch_proj_bwd_dx(ctx, T, N, Npad, x, W, gain, e, kappa, dx, accumulate_dx, s);
+            launch_proj_bwd_dw(ctx, T, N, Npad, x, W, gain, e, G, dW, dgain, accumulate_params, s);
             rc = check_cuda(ctx, cudaGetLastError(), "coeffs_bwd_static launch");
         }
     }

@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(kThreads) tail_mix_k(int64_t T, int C8, const 
         }
 #pragma unroll
         for (int j = 0; j < N_; ++j) r[j] = warp_sum(r[j]);
-        if (lane == 0) {
+        if (lane == 0 && dH_pre) {
 #pragma unroll
             for (int j = 0; j < N_; ++j) dH_pre[t * N_ + j] = r[j];
         }

@@ -106,9 +106,24 @@ def staged_dx_allowance(ref, fused):
     the other way on the GPU (fp32 sums) than in fp64, which moves dx by up to 2^-8 |v|."""
     d2 = ref["dx"] - ref["dx_coeffs"]                     # after H_res^T g + H_pre du
     if fused:
-        return 2.0 ** -8 * np.abs(d2)
+        return 0.0                                        # the fused tail writes dx once
     d1 = d2 - ref["dx_premix"]                            # after H_res^T g
     return 2.0 ** -8 * (np.abs(d1) + np.abs(d2))
+
+
+def dxhat_allowance(inp, dz, eps=1e-6):
+    """Allowance for the projection-backward term of dx, sum_c e[t,c] W'[m,c]: the tensor-core kernel
+    rounds both operands to bf16 (as bf16 mixed-precision training does for this matmul), so each
+    product carries up to 2^-8 relative error: |error| <= 2^-8 sum_c |e[t,c]| |W'[m,c]|."""
+    o = oracle_inputs(inp)
+    x = o["x"]; T, n, C = x.shape
+    xh = x.reshape(T, n * C)
+    rstd = 1.0 / np.sqrt((xh * xh).mean(axis=1) + eps)
+    n_res = dz.shape[1] - 2 * n
+    av = np.concatenate([np.full(n_res, o["alpha"][0]), np.full(n, o["alpha"][1]), np.full(n, o["alpha"][2])])
+    e = np.abs(rstd[:, None] * av * dz)
+    Wp = np.abs(o["gain"][:, None] * o["W"])
+    return 2.0 ** -8 * (e @ Wp.T).reshape(T, n, C)
 
 
 def compare_backward(G, ref, grad_rel=1e-3, fused=True):
@@ -116,7 +131,7 @@ def compare_backward(G, ref, grad_rel=1e-3, fused=True):
     check_bf16("dy", host(B.dy), ref["dy"])
     check_f32("dH_res", host(B.dH_res), ref["dH_res"], 2e-5)
     check_f32("dH_post", host(B.dH_post), ref["dH_post"], 2e-5)
-    check_bf16("dx", host(B.dx), ref["dx"], extra=staged_dx_allowance(ref, fused))
+    check_bf16("dx", host(B.dx), ref["dx"], extra=staged_dx_allowance(ref, fused) + dxhat_allowance(G.inp, ref["dz"], G.eps))
     check_f32("dW", host(B.dW), ref["dW"], grad_rel)
     check_f32("db", host(B.db), ref["db"], grad_rel)
     check_f32("dalpha", host(B.dalpha), ref["dalpha"], grad_rel)

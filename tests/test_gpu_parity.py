@@ -9,8 +9,8 @@ import torch
 from oracle import mhclite_oracle as O
 from paper_2601_05732_b200 import synth
 from paper_2601_05732_b200 import layer as L
-from parity_utils import (DEV, GpuLayer, check_bf16, check_f32, compare_backward, compare_forward, host,
-                          oracle_bwd, oracle_fwd, oracle_inputs)
+from parity_utils import (DEV, GpuLayer, check_bf16, check_f32, compare_backward, compare_forward, dxhat_allowance,
+                          host, oracle_bwd, oracle_fwd, oracle_inputs)
 
 pytestmark = pytest.mark.gpu
 
@@ -97,7 +97,8 @@ def test_coeffs_bwd_in_isolation():
     G.ctx.coeffs_bwd(G.x, P.W, P.alpha, P.gain, 1e-6, B.a_saved, B.p_saved, B.rstd, B.H_pre, B.H_post,
                      dHr, dHp, dHo, B.dx, False, B.dW, B.db, B.dalpha, B.dgain, False)
     torch.cuda.synchronize()
-    check_bf16("dx_coeffs", host(B.dx), ref["dx_coeffs"])
+    allow = dxhat_allowance(inp, ref["dz"])
+    check_bf16("dx_coeffs", host(B.dx), ref["dx_coeffs"], extra=allow)
     check_f32("dW", host(B.dW), ref["dW"], 1e-3)
     check_f32("dgain", host(B.dgain), ref["dgain"], 1e-3)
     check_f32("db", host(B.db), ref["db"], 1e-3)
@@ -110,7 +111,7 @@ def test_coeffs_bwd_in_isolation():
     check_f32("db x2", host(B.db), 2 * ref["db"], 1e-3)
     check_f32("dalpha x2", host(B.dalpha), 2 * ref["dalpha"], 1e-3)
     check_f32("dgain x2", host(B.dgain), 2 * ref["dgain"], 1e-3)
-    check_bf16("dx x2", host(B.dx), 2 * ref["dx_coeffs"], rel=3e-2)
+    check_bf16("dx x2", host(B.dx), 2 * ref["dx_coeffs"], rel=3e-2, extra=2 * allow)
 
 
 @pytest.mark.parametrize("T", [0, 1, 2, 31, 33])

@@ -15,10 +15,18 @@ import pytest
 import torch
 
 from paper_2601_05732_b200 import synth
-from paper_2601_05732_b200.binding import MhcLite, ERR_WORKSPACE, workspace_bytes, load
-from parity_utils import DEV, GpuLayer, check_bf16, check_f32, host
+from paper_2601_05732_b200.binding import MhcLite, ERR_WORKSPACE, load
+from oracle import mhclite_oracle as O
+from parity_utils import DEV, GpuLayer, check_bf16, check_f32, dxhat_allowance, host, oracle_inputs
 
 pytestmark = pytest.mark.gpu
+
+
+def _scratch_need(n, C, T):
+    """Scratch the static entry point takes from its array (the formula of its header comment)."""
+    import math
+    Np = (math.factorial(n) + 2 * n + 7) // 8 * 8
+    return 4 * (T * Np + T + n * C * Np) + 3 * 256
 
 
 def _upstream(G, seed):
@@ -31,7 +39,7 @@ def _upstream(G, seed):
 
 def test_static_scratch_matches_workspace_entry_point_twice():
     n, C, T = 4, 256, 700
-    assert workspace_bytes(n, C, T, 0) <= load().mhclite_static_scratch_bytes()
+    assert _scratch_need(n, C, T) <= load().mhclite_static_scratch_bytes()
     outs = []
     for call, seed in enumerate((61, 62)):           # two calls in a row, different data
         inp = synth.make_layer_inputs(n, C, T, seed=seed, bias_std=0.5, alpha=[1.0, 1.0, 1.0], w_std=0.05)
@@ -54,7 +62,11 @@ def test_static_scratch_matches_workspace_entry_point_twice():
                                dHr, dHp, dHo, dx, False, dW, db, dal, dg, False)
         torch.cuda.synchronize()
         assert bare._ws is None
-        check_bf16(f"dx (call {call})", host(dx), ref["dx"])
+        # the workspace entry point rounds the operands of sum_c e W' to bf16 (tensor cores), this one
+        # keeps them in fp32: allow for that rounding exactly as the parity tests do
+        o = oracle_inputs(inp)
+        dz = O.coeffs_bwd(o["x"], o["W"], o["b"], o["alpha"], o["gain"], 1e-6, host(dHr), host(dHp), host(dHo))["dz"]
+        check_bf16(f"dx (call {call})", host(dx), ref["dx"], extra=dxhat_allowance(inp, dz))
         check_f32(f"dW (call {call})", host(dW), ref["dW"], 1e-3)
         check_f32(f"db (call {call})", host(db), ref["db"], 1e-3)
         check_f32(f"dalpha (call {call})", host(dal), ref["dalpha"], 1e-3)
@@ -66,7 +78,7 @@ def test_static_scratch_matches_workspace_entry_point_twice():
 
 def test_static_scratch_rejects_oversized_problem():
     n, C, T = 4, 1024, 65536
-    assert workspace_bytes(n, C, T, 0) > load().mhclite_static_scratch_bytes()
+    assert _scratch_need(n, C, T) > load().mhclite_static_scratch_bytes()
     ctx = MhcLite(n, C)
     z = torch.zeros(64, device=DEV)
     zb = torch.zeros(64, device=DEV, dtype=torch.bfloat16)
