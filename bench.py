@@ -174,12 +174,14 @@ def run_ours(args, wl, rank, world):
     x, y, g, du = (L.to_device_bf16(inp[k], dev) for k in ("x", "y", "g", "du"))
     eps = 1e-6
 
+    fused = not args.unfused
+
     def step():
-        L.pre_fwd(ctx, P, B, x, eps, True)
+        L.pre_fwd(ctx, P, B, x, eps, fused)
         L.post_fwd(ctx, B, x, y)
         if wl.backward:
-            L.post_bwd(ctx, B, x, y, g, True)
-            L.tail_bwd(ctx, P, B, x, g, du, eps, True)
+            L.post_bwd(ctx, B, x, y, g, fused)
+            L.tail_bwd(ctx, P, B, x, g, du, eps, fused)
 
     def barrier():
         if world > 1:
@@ -214,10 +216,10 @@ def run_ours(args, wl, rank, world):
         ms = float(tt.item())
 
     # ---- per-stage device time (same launch configuration), for the roofline of the dominant stage
-    stages = [("pre_fwd", lambda: L.pre_fwd(ctx, P, B, x, eps, True)), ("post_fwd", lambda: L.post_fwd(ctx, B, x, y))]
+    stages = [("pre_fwd", lambda: L.pre_fwd(ctx, P, B, x, eps, fused)), ("post_fwd", lambda: L.post_fwd(ctx, B, x, y))]
     if wl.backward:
-        stages += [("post_bwd", lambda: L.post_bwd(ctx, B, x, y, g, True)),
-                   ("tail_bwd", lambda: L.tail_bwd(ctx, P, B, x, g, du, eps, True))]
+        stages += [("post_bwd", lambda: L.post_bwd(ctx, B, x, y, g, fused)),
+                   ("tail_bwd", lambda: L.tail_bwd(ctx, P, B, x, g, du, eps, fused))]
     ev = {k: [] for k, _ in stages}
     for _ in range(args.steps):
         for k, fn in stages:
@@ -272,7 +274,7 @@ def run_ours(args, wl, rank, world):
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, f32 accumulate",
             "data": "synthetic",
-            "config": {"workload": wl.name, "n": n, "C": C, "T_per_gpu": T, "passes": "fwd+bwd" if wl.backward else "fwd",
+            "config": {"workload": wl.name, "n": n, "C": C, "T_per_gpu": T, "passes": "fwd+bwd" if wl.backward else "fwd", "calls": "fused" if fused else "unfused",
                        "note": wl.note, "l2": "inputs larger than L2 (working set %.0f MB)" % (total_bytes / 1e6)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
             "cpu_baseline": cpu_baseline,
@@ -293,6 +295,7 @@ def main():
     ap.add_argument("--cpu-sample", type=int, default=16384, help="tokens of the oracle's timed sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--unfused", action="store_true", help="time the un-fused call sequence (six entry points)")
     args = ap.parse_args()
 
     from paper_2601_05732_b200 import synth

@@ -67,6 +67,90 @@ __device__ __forceinline__ void finish_projection(int64_t t, int64_t T, int N, i
     }
 }
 
+// Per-block shared state of the mHC-lite activation kernels.  The permutation tables are copied from
+// constant memory once per block: lanes index them with different addresses, which the constant cache
+// would serialise.
+struct LiteShared {
+    uint8_t sigma[kMaxFact * kMaxN];
+    uint8_t klist[kMaxN * kMaxN * 24];
+    float a_s[kActWarps][kMaxFact + 8];
+    float p_s[kActWarps][kMaxCols + 6];
+    float dh_s[kActWarps][32];
+    float red[kActWarps][kMaxCols + 3];
+};
+__device__ __forceinline__ void load_tables(LiteShared& sh, int n) {
+    const PermTables& tab = c_perm[n];
+    for (int i = threadIdx.x; i < kMaxFact * kMaxN; i += blockDim.x) { sh.sigma[i] = tab.sigma[i]; sh.klist[i] = tab.klist[i]; }
+    __syncthreads();
+}
+
+// Forward of one token by one warp, given its normalised projection row pt[0..N) (shared memory):
+// z = alpha p + b, sigmoid gates, softmax, H_res = sum_k a_k P_k.
+// Returns the gate of this lane: H_pre[lane] for lane < n, H_post[lane - n] for n <= lane < 2n.
+__device__ __forceinline__ float lite_token_fwd_core(LiteShared& sh, int w, int lane, int64_t t, int n, int nf,
+                                                     const float* pt, const float* __restrict__ b, float a_res,
+                                                     float a_pre, float a_post, float* __restrict__ H_res,
+                                                     float* __restrict__ H_pre, float* __restrict__ H_post,
+                                                     float* __restrict__ a_saved) {
+    const int per = nf / n, nn = n * n;
+    float z[4], m = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        const int k = lane + 32 * s;
+        z[s] = -INFINITY;
+        if (k < nf) { z[s] = fmaf(a_res, pt[k], __ldg(b + k)); m = fmaxf(m, z[s]); }
+    }
+    m = warp_max(m);
+    float sum = 0.f;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        z[s] = (lane + 32 * s < nf) ? expf(z[s] - m) : 0.f;
+        sum += z[s];
+    }
+    sum = warp_sum(sum);
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        const int k = lane + 32 * s;
+        if (k < nf) {
+            const float a = z[s] / sum;
+            sh.a_s[w][k] = a;
+            a_saved[t * nf + k] = a;
+        }
+    }
+    float gate = 0.f;
+    if (lane < 2 * n) {
+        const int c = nf + lane;
+        const float zz = fmaf(lane < n ? a_pre : a_post, pt[c], __ldg(b + c));
+        gate = sigmoidf_(zz);
+        if (lane < n) H_pre[t * n + lane] = gate; else { gate *= 2.f; H_post[t * n + lane - n] = gate; }
+    }
+    __syncwarp();
+    if (lane < nn) {
+        float h = 0.f;
+        for (int r = 0; r < per; ++r) h += sh.a_s[w][sh.klist[lane * per + r]];
+        H_res[t * nn + lane] = h;
+    }
+    __syncwarp();
+    return gate;
+}
+
+// The same, starting from the K-slice partials of the projection in global memory.
+__device__ __forceinline__ float lite_token_fwd(LiteShared& sh, int w, int lane, int64_t t, int64_t T, int n, int nf,
+                                                int Npad, int ksplit, float inv_nC, float eps,
+                                                const float* __restrict__ qpart, const float* __restrict__ ssq,
+                                                const float* __restrict__ b, float a_res, float a_pre, float a_post,
+                                                float* __restrict__ H_res, float* __restrict__ H_pre,
+                                                float* __restrict__ H_post, float* __restrict__ a_saved,
+                                                float* __restrict__ p_saved, float* __restrict__ rstd) {
+    const int N = nf + 2 * n;
+    float pv[5];
+    finish_projection(t, T, N, Npad, ksplit, inv_nC, eps, qpart, ssq, p_saved, rstd, lane, pv);
+#pragma unroll
+    for (int k = 0; k < 5; ++k) if (lane + 32 * k < N) sh.p_s[w][lane + 32 * k] = pv[k];
+    __syncwarp();
+    return lite_token_fwd_core(sh, w, lane, t, n, nf, sh.p_s[w], b, a_res, a_pre, a_post, H_res, H_pre, H_post, a_saved);
+}
+
 __global__ void __launch_bounds__(kActThreads) lite_act_fwd_k(int64_t T, int n, int nf, int Npad, int ksplit,
                                                              float inv_nC, float eps, const float* __restrict__ qpart,
                                                              const float* __restrict__ ssq,
@@ -74,138 +158,568 @@ __global__ void __launch_bounds__(kActThreads) lite_act_fwd_k(int64_t T, int n, 
                                                              float* __restrict__ H_res, float* __restrict__ H_pre,
                                                              float* __restrict__ H_post, float* __restrict__ a_saved,
                                                              float* __restrict__ p_saved, float* __restrict__ rstd) {
-    __shared__ float a_s[kActWarps][kMaxFact + 8];
-    __shared__ float p_s[kActWarps][kMaxCols + 6];
+    __shared__ LiteShared sh;
+    load_tables(sh, n);
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int N = nf + 2 * n, per = nf / n, nn = n * n;
-    const PermTables& tab = c_perm[n];
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
     const int64_t nwarps = (int64_t)gridDim.x * kActWarps;
-    for (int64_t t = (int64_t)blockIdx.x * kActWarps + w; t < T; t += nwarps) {
-        float pv[5];
-        finish_projection(t, T, N, Npad, ksplit, inv_nC, eps, qpart, ssq, p_saved, rstd, lane, pv);
-#pragma unroll
-        for (int k = 0; k < 5; ++k) if (lane + 32 * k < N) p_s[w][lane + 32 * k] = pv[k];
-        __syncwarp();
-        const float* pt = p_s[w];
-        float z[4], m = -INFINITY;
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            const int k = lane + 32 * s;
-            z[s] = -INFINITY;
-            if (k < nf) { z[s] = fmaf(a_res, pt[k], __ldg(b + k)); m = fmaxf(m, z[s]); }
+    for (int64_t t = (int64_t)blockIdx.x * kActWarps + w; t < T; t += nwarps)
+        lite_token_fwd(sh, w, lane, t, T, n, nf, Npad, ksplit, inv_nC, eps, qpart, ssq, b, a_res, a_pre, a_post,
+                       H_res, H_pre, H_post, a_saved, p_saved, rstd);
+}
+
+// Mappings + stream pre-mix in one kernel, in groups of kGroupTok tokens per block:
+//   L: the group's projection partials are added, normalised and staged in shared memory by all threads
+//      (one round of coalesced loads, so the per-token math below waits on no global load);
+//   A: one warp per token: gates, softmax, H_res;
+//   P: all threads stream the group's tokens: u[t,:] = sum_j H_pre[t,j] x[t,j,:]   (Eq. (1), inner term).
+constexpr int kGroupTok = 32;
+
+template <int N_>
+__global__ void __launch_bounds__(kActThreads) lite_act_premix_k(
+    int64_t T, int C8, int nf, int Npad, int ksplit, float inv_nC, float eps, const float* __restrict__ qpart,
+    const float* __restrict__ ssq, const float* __restrict__ b, const float* __restrict__ alpha,
+    float* __restrict__ H_res, float* __restrict__ H_pre, float* __restrict__ H_post, float* __restrict__ a_saved,
+    float* __restrict__ p_saved, float* __restrict__ rstd, const uint4* __restrict__ x, uint4* __restrict__ u) {
+    __shared__ LiteShared sh;
+    __shared__ float pg[kGroupTok][kMaxCols + 3];
+    __shared__ float rg[kGroupTok];
+    __shared__ float hg[kGroupTok][kMaxN];
+    load_tables(sh, N_);
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int N = nf + 2 * N_;
+    const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
+    const int64_t ngroups = (T + kGroupTok - 1) / kGroupTok;
+    for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
+        const int64_t t0 = grp * kGroupTok;
+        const int nt = (T - t0 < kGroupTok) ? (int)(T - t0) : kGroupTok;
+        // L
+        if (tid < nt) {
+            float ss = 0.f;
+            for (int s = 0; s < ksplit; ++s) ss += __ldg(ssq + (int64_t)s * T + t0 + tid);
+            const float r = 1.f / sqrtf(ss * inv_nC + eps);
+            rg[tid] = r;
+            rstd[t0 + tid] = r;
         }
-        m = warp_max(m);
-        float sum = 0.f;
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            z[s] = (lane + 32 * s < nf) ? expf(z[s] - m) : 0.f;
-            sum += z[s];
+        for (int i = tid; i < nt * N; i += kActThreads) {
+            const int tl = i / N, c = i - tl * N;
+            float q = 0.f;
+            for (int s = 0; s < ksplit; ++s) q += __ldg(qpart + ((int64_t)s * T + t0 + tl) * Npad + c);
+            pg[tl][c] = q;
         }
-        sum = warp_sum(sum);
+        __syncthreads();
+        for (int i = tid; i < nt * N; i += kActThreads) {
+            const int tl = i / N, c = i - tl * N;
+            const float pv = pg[tl][c] * rg[tl];
+            pg[tl][c] = pv;
+            p_saved[(t0 + tl) * N + c] = pv;
+        }
+        __syncthreads();
+        // A
+        for (int tl = w; tl < nt; tl += kActWarps) {
+            const float gate = lite_token_fwd_core(sh, w, lane, t0 + tl, N_, nf, pg[tl], b, a_res, a_pre, a_post, H_res,
+                                                   H_pre, H_post, a_saved);
+            if (lane < N_) hg[tl][lane] = gate;
+        }
+        __syncthreads();
+        // P
+        for (int i = tid; i < nt * C8; i += kActThreads) {
+            const int tl = i / C8, cv = i - tl * C8;
+            const int64_t t = t0 + tl;
+            uint4 v[N_];
 #pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            const int k = lane + 32 * s;
-            if (k < nf) {
-                const float a = z[s] / sum;
-                a_s[w][k] = a;
-                a_saved[t * nf + k] = a;
+            for (int j = 0; j < N_; ++j) v[j] = ld_stream(x + (t * N_ + j) * C8 + cv);
+            float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+            for (int j = 0; j < N_; ++j) {
+                const float h = hg[tl][j];
+                float f[8];
+                unpack8(v[j], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = fmaf(h, f[e], acc[e]);
             }
+            st_stream(u + t * C8 + cv, pack8(acc));
         }
-        if (lane < 2 * n) {
-            const int c = nf + lane;
-            const float zz = fmaf(lane < n ? a_pre : a_post, pt[c], __ldg(b + c));
-            const float sg = sigmoidf_(zz);
-            if (lane < n) H_pre[t * n + lane] = sg; else H_post[t * n + lane - n] = 2.f * sg;
-        }
-        __syncwarp();
-        if (lane < nn) {
-            float h = 0.f;
-            for (int r = 0; r < per; ++r) h += a_s[w][tab.klist[lane * per + r]];
-            H_res[t * nn + lane] = h;
-        }
-        __syncwarp();
+        __syncthreads();
     }
 }
 
-// Shared tail of both backward kernels: from dz of one column to e, kappa, db, dalpha partials.
-// ------------------------------------------------------------------------------------------------
+// Backward of one token by one warp (gradient of Eq. (4), (5)): from dH_res, dH_post (global) and this
+// lane's dH_pre (lane j < n holds dH_pre[j]) to e = rstd alpha dz, kappa, and the db / dalpha partials.
+struct LiteBwdAcc { float db_res[4], db_gate, dal_res, dal_gate; };
+
+__device__ __forceinline__ void lite_token_bwd(LiteShared& sh, int w, int lane, int64_t t, int n, int nf, float inv_nC,
+                                               const float* a_tok, const float* pt, float rs, float a_res, float a_pre,
+                                               float a_post, const float* hpre_tok, const float* hpost_tok,
+                                               const float* dhres_tok, float dhpre_lane, const float* dhpost_tok,
+                                               const EOut& eo, float* __restrict__ kappa, LiteBwdAcc& acc) {
+    // *_tok point at this token's rows (global or shared memory)
+    const int N = nf + 2 * n, nn = n * n;
+    if (lane < nn) sh.dh_s[w][lane] = dhres_tok[lane];
+    __syncwarp();
+    float a[4], da[4], dot = 0.f;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        const int k = lane + 32 * s;
+        a[s] = 0.f; da[s] = 0.f;
+        if (k < nf) {
+            a[s] = a_tok[k];
+            float d = 0.f;
+            for (int i = 0; i < n; ++i) d += sh.dh_s[w][i * n + sh.sigma[k * n + i]];   // Eq. (5): dL/da_k
+            da[s] = d;
+            dot = fmaf(a[s], d, dot);
+        }
+    }
+    dot = warp_sum(dot);
+    float kap = 0.f;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        const int k = lane + 32 * s;
+        if (k < nf) {
+            const float dz = a[s] * (da[s] - dot);
+            const float ed = a_res * dz, pv = pt[k];
+            store_e(eo, t, k, rs * ed);
+            kap = fmaf(ed, pv, kap);
+            acc.db_res[s] += dz;
+            acc.dal_res = fmaf(dz, pv, acc.dal_res);
+        }
+    }
+    if (lane < 2 * n) {
+        const int c = nf + lane;
+        float dz;
+        if (lane < n) { const float h = hpre_tok[lane]; dz = dhpre_lane * h * (1.f - h); }
+        else { const float h = hpost_tok[lane - n]; dz = dhpost_tok[lane - n] * h * (1.f - 0.5f * h); }
+        const float ed = (lane < n ? a_pre : a_post) * dz, pv = pt[c];
+        store_e(eo, t, c, rs * ed);
+        kap = fmaf(ed, pv, kap);
+        acc.db_gate += dz;
+        acc.dal_gate = fmaf(dz, pv, acc.dal_gate);
+    }
+    pad_e(eo, t, N, lane, 32);
+    kap = warp_sum(kap);
+    if (lane == 0) kappa[t] = rs * rs * kap * inv_nC;
+    __syncwarp();
+}
+
+// Block reduction of the parameter-gradient partials, then one atomic per column per block.
+__device__ __forceinline__ void lite_bwd_reduce(LiteShared& sh, int w, int lane, int n, int nf, const LiteBwdAcc& acc,
+                                                float* db, float* dalpha) {
+    const int N = nf + 2 * n;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) if (lane + 32 * s < nf) sh.red[w][lane + 32 * s] = acc.db_res[s];
+    if (lane < 2 * n) sh.red[w][nf + lane] = acc.db_gate;
+    const float d0 = warp_sum(acc.dal_res);
+    const float d1 = warp_sum(lane < n ? acc.dal_gate : 0.f);
+    const float d2 = warp_sum((lane >= n && lane < 2 * n) ? acc.dal_gate : 0.f);
+    if (lane == 0) { sh.red[w][N] = d0; sh.red[w][N + 1] = d1; sh.red[w][N + 2] = d2; }
+    __syncthreads();
+    for (int c = threadIdx.x; c < N + 3; c += kActThreads) {
+        float v = 0.f;
+#pragma unroll
+        for (int ww = 0; ww < kActWarps; ++ww) v += sh.red[ww][c];
+        if (c < N) atomicAdd(db + c, v); else atomicAdd(dalpha + (c - N), v);
+    }
+}
+
 __global__ void __launch_bounds__(kActThreads) lite_act_bwd_k(
     int64_t T, int n, int nf, float inv_nC, const float* __restrict__ a_saved, const float* __restrict__ p,
     const float* __restrict__ rstd, const float* __restrict__ alpha, const float* __restrict__ H_pre,
     const float* __restrict__ H_post, const float* __restrict__ dH_res, const float* __restrict__ dH_pre,
     const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa, float* db, float* dalpha) {
-    __shared__ float dh_s[kActWarps][32];
-    __shared__ float red[kActWarps][kMaxCols + 3];
+    __shared__ LiteShared sh;
+    load_tables(sh, n);
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int N = nf + 2 * n, nn = n * n;
-    const PermTables& tab = c_perm[n];
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
-    float db_res[4] = {0, 0, 0, 0}, db_gate = 0.f, dal_res = 0.f, dal_gate = 0.f;
+    LiteBwdAcc acc = {{0, 0, 0, 0}, 0.f, 0.f, 0.f};
     const int64_t nwarps = (int64_t)gridDim.x * kActWarps;
     for (int64_t t = (int64_t)blockIdx.x * kActWarps + w; t < T; t += nwarps) {
-        const float* pt = p + t * N;
-        const float rs = __ldg(rstd + t);
-        if (lane < nn) dh_s[w][lane] = dH_res[t * nn + lane];
-        __syncwarp();
-        float a[4], da[4], dot = 0.f;
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            const int k = lane + 32 * s;
-            a[s] = 0.f; da[s] = 0.f;
-            if (k < nf) {
-                a[s] = a_saved[t * nf + k];
-                float d = 0.f;
-                for (int i = 0; i < n; ++i) d += dh_s[w][i * n + tab.sigma[k * n + i]];   // Eq. (5): dL/da_k
-                da[s] = d;
-                dot = fmaf(a[s], d, dot);
-            }
-        }
-        dot = warp_sum(dot);
-        float kap = 0.f;
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            const int k = lane + 32 * s;
-            if (k < nf) {
-                const float dz = a[s] * (da[s] - dot);
-                const float ed = a_res * dz, pv = pt[k];
-                store_e(eo, t, k, rs * ed);
-                kap = fmaf(ed, pv, kap);
-                db_res[s] += dz;
-                dal_res = fmaf(dz, pv, dal_res);
-            }
-        }
-        if (lane < 2 * n) {
-            const int c = nf + lane;
-            float dz;
-            if (lane < n) { const float h = H_pre[t * n + lane]; dz = dH_pre[t * n + lane] * h * (1.f - h); }
-            else { const float h = H_post[t * n + lane - n]; dz = dH_post[t * n + lane - n] * h * (1.f - 0.5f * h); }
-            const float ed = (lane < n ? a_pre : a_post) * dz, pv = pt[c];
-            store_e(eo, t, c, rs * ed);
-            kap = fmaf(ed, pv, kap);
-            db_gate += dz;
-            dal_gate = fmaf(dz, pv, dal_gate);
-        }
-        pad_e(eo, t, N, lane, 32);
-        kap = warp_sum(kap);
-        if (lane == 0) kappa[t] = rs * rs * kap * inv_nC;
-        __syncwarp();
+        const float dhp = (lane < n) ? dH_pre[t * n + lane] : 0.f;
+        lite_token_bwd(sh, w, lane, t, n, nf, inv_nC, a_saved + t * nf, p + t * (nf + 2 * n), __ldg(rstd + t), a_res,
+                       a_pre, a_post, H_pre + t * n, H_post + t * n, dH_res + t * n * n, dhp, dH_post + t * n, eo,
+                       kappa, acc);
     }
-    // block reduction of the parameter-gradient partials, then one atomic per column per block
+    lite_bwd_reduce(sh, w, lane, n, nf, acc, db, dalpha);
+}
+
+// First kernel of the fused backward tail, in groups of kGroupTok tokens per block:
+//   L: the per-token inputs of the activation backward are copied to shared memory with cp.async
+//      (they arrive while D streams);
+//   D: one warp per token streams x and du: dH_pre[j] = <du, x_j>;
+//   A: one warp per token: activation backward from shared memory (no global load on the way).
+// (one token's staged inputs, as floats: a | p | dH_res | H_pre | H_post | dH_post | rstd)
+template <int N_>
+__global__ void __launch_bounds__(kActThreads) lite_tailpre_k(
+    int64_t T, int C8, int nf, float inv_nC, const uint4* __restrict__ x, const uint4* __restrict__ du,
+    const float* __restrict__ a_saved, const float* __restrict__ p, const float* __restrict__ rstd,
+    const float* __restrict__ alpha, const float* __restrict__ H_pre, const float* __restrict__ H_post,
+    const float* __restrict__ dH_res, const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa,
+    float* db, float* dalpha) {
+    __shared__ LiteShared sh;
+    constexpr int NN = N_ * N_;
+    constexpr int kFact = (N_ == 2) ? 2 : (N_ == 3) ? 6 : (N_ == 4) ? 24 : 120;
+    constexpr int kStride = kFact + (kFact + 2 * N_) + NN + 3 * N_ + 1 + 1;
+    constexpr int kGroupTok = (N_ == 5) ? 16 : 32;              // keeps the staging under the static shared-memory limit
+    __shared__ float in_s[kGroupTok][kStride];
+    __shared__ float dhp_s[kGroupTok][kMaxN];
+    load_tables(sh, N_);
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int N = nf + 2 * N_;
+    const int o_p = nf, o_dhres = o_p + N, o_hpre = o_dhres + NN, o_hpost = o_hpre + N_, o_dhpost = o_hpost + N_,
+              o_rstd = o_dhpost + N_, nin = o_rstd + 1;
+    const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
+    LiteBwdAcc acc = {{0, 0, 0, 0}, 0.f, 0.f, 0.f};
+    const int64_t ngroups = (T + kGroupTok - 1) / kGroupTok;
+    for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
+        const int64_t t0 = grp * kGroupTok;
+        const int nt = (T - t0 < kGroupTok) ? (int)(T - t0) : kGroupTok;
+        // L
+        for (int i = tid; i < nt * nin; i += kActThreads) {
+            const int tl = i / nin, c = i - tl * nin;
+            const int64_t t = t0 + tl;
+            const float* src;
+            if (c < o_p) src = a_saved + t * nf + c;
+            else if (c < o_dhres) src = p + t * N + (c - o_p);
+            else if (c < o_hpre) src = dH_res + t * NN + (c - o_dhres);
+            else if (c < o_hpost) src = H_pre + t * N_ + (c - o_hpre);
+            else if (c < o_dhpost) src = H_post + t * N_ + (c - o_hpost);
+            else if (c < o_rstd) src = dH_post + t * N_ + (c - o_dhpost);
+            else src = rstd + t;
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&in_s[tl][c])), "l"(src) : "memory");
+        }
+        cp_async_commit();
+        // D
+        for (int tl = w; tl < nt; tl += kActWarps) {
+            const int64_t t = t0 + tl;
+            float r[N_];
 #pragma unroll
-    for (int s = 0; s < 4; ++s) if (lane + 32 * s < nf) red[w][lane + 32 * s] = db_res[s];
-    if (lane < 2 * n) red[w][nf + lane] = db_gate;
-    const float d0 = warp_sum(dal_res);
-    const float d1 = warp_sum(lane < n ? dal_gate : 0.f);
-    const float d2 = warp_sum((lane >= n && lane < 2 * n) ? dal_gate : 0.f);
-    if (lane == 0) { red[w][N] = d0; red[w][N + 1] = d1; red[w][N + 2] = d2; }
+            for (int j = 0; j < N_; ++j) r[j] = 0.f;
+            for (int cv = lane; cv < C8; cv += 32) {
+                uint4 xv[N_];
+#pragma unroll
+                for (int j = 0; j < N_; ++j) xv[j] = ld_stream(x + (t * N_ + j) * C8 + cv);
+                float df[8];
+                unpack8(ld_stream(du + t * C8 + cv), df);
+#pragma unroll
+                for (int j = 0; j < N_; ++j) {
+                    float xf[8];
+                    unpack8(xv[j], xf);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) r[j] = fmaf(df[e], xf[e], r[j]);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < N_; ++j) { r[j] = warp_sum(r[j]); if (lane == j) dhp_s[tl][j] = r[j]; }
+        }
+        cp_async_wait<0>();
+        __syncthreads();
+        // A
+        for (int tl = w; tl < nt; tl += kActWarps) {
+            const float* in = in_s[tl];
+            const float dhp = (lane < N_) ? dhp_s[tl][lane] : 0.f;
+            lite_token_bwd(sh, w, lane, t0 + tl, N_, nf, inv_nC, in, in + o_p, in[o_rstd], a_res, a_pre, a_post,
+                           in + o_hpre, in + o_hpost, in + o_dhres, dhp, in + o_dhpost, eo, kappa, acc);
+        }
+        __syncthreads();
+    }
+    lite_bwd_reduce(sh, w, lane, N_, nf, acc, db, dalpha);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Thread-per-token versions for n <= 4 (n! <= 24 logits fit in registers).  A warp working on one token
+// spends ~500 dependent instructions on shuffles and reductions; a thread working on one token spends a
+// similar count for 32 tokens at once.  Inputs and outputs are staged in shared memory so that global
+// traffic stays coalesced.
+// ------------------------------------------------------------------------------------------------
+template <int N_>
+struct LiteDims {
+    static constexpr int kFact = (N_ == 2) ? 2 : (N_ == 3) ? 6 : 24;
+    static constexpr int kN = kFact + 2 * N_;
+    static constexpr int kNN = N_ * N_;
+    static constexpr int kPer = kFact / N_;
+    static constexpr int kOut = kFact + kNN + 2 * N_;        // a | H_res | H_pre | H_post
+    static constexpr int kIn = kFact + kN + kNN + 3 * N_ + 1; // a | p | dH_res | H_pre | H_post | dH_post | rstd
+};
+
+template <int N_>
+__device__ __forceinline__ void lite_thread_fwd(const float* prow, float* orow, const float* b_s, float a_res,
+                                                float a_pre, float a_post, const uint8_t* klist_s) {
+    using D = LiteDims<N_>;
+    float z[D::kFact], m = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < D::kFact; ++k) { z[k] = fmaf(a_res, prow[k], b_s[k]); m = fmaxf(m, z[k]); }
+    float sum = 0.f;
+#pragma unroll
+    for (int k = 0; k < D::kFact; ++k) { z[k] = expf(z[k] - m); sum += z[k]; }
+#pragma unroll
+    for (int k = 0; k < D::kFact; ++k) orow[k] = z[k] / sum;
+#pragma unroll
+    for (int e = 0; e < D::kNN; ++e) {
+        float h = 0.f;
+#pragma unroll
+        for (int r = 0; r < D::kPer; ++r) h += orow[klist_s[e * D::kPer + r]];
+        orow[D::kFact + e] = h;
+    }
+#pragma unroll
+    for (int j = 0; j < N_; ++j) {
+        orow[D::kFact + D::kNN + j] = sigmoidf_(fmaf(a_pre, prow[D::kFact + j], b_s[D::kFact + j]));
+        orow[D::kFact + D::kNN + N_ + j] = 2.f * sigmoidf_(fmaf(a_post, prow[D::kFact + N_ + j], b_s[D::kFact + N_ + j]));
+    }
+}
+
+constexpr int kTokGroup = 32;    // tokens per block iteration of the thread-per-token kernels
+
+template <int N_>
+__global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
+    int64_t T, int C8, int Npad, int ksplit, float inv_nC, float eps, const float* __restrict__ qpart,
+    const float* __restrict__ ssq, const float* __restrict__ b, const float* __restrict__ alpha,
+    float* __restrict__ H_res, float* __restrict__ H_pre, float* __restrict__ H_post, float* __restrict__ a_saved,
+    float* __restrict__ p_saved, float* __restrict__ rstd, const uint4* __restrict__ x, uint4* __restrict__ u) {
+    using D = LiteDims<N_>;
+    __shared__ uint8_t klist_s[D::kNN * D::kPer];
+    __shared__ float b_s[D::kN];
+    __shared__ float pg[kTokGroup][D::kN + 1];
+    __shared__ float og[kTokGroup][D::kOut + 1];
+    __shared__ float rg[kTokGroup];
+    const int tid = threadIdx.x;
+    for (int i = tid; i < D::kNN * D::kPer; i += kActThreads) klist_s[i] = c_perm[N_].klist[i];
+    for (int i = tid; i < D::kN; i += kActThreads) b_s[i] = __ldg(b + i);
+    const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
     __syncthreads();
-    for (int c = threadIdx.x; c < N + 3; c += kActThreads) {
-        float v = 0.f;
+    const int64_t ngroups = (T + kTokGroup - 1) / kTokGroup;
+    for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
+        const int64_t t0 = grp * kTokGroup;
+        const int nt = (T - t0 < kTokGroup) ? (int)(T - t0) : kTokGroup;
+        // L: partials -> normalised projection rows in shared memory (and p_saved, rstd)
+        if (tid < nt) {
+            float ss = 0.f;
+            for (int s = 0; s < ksplit; ++s) ss += __ldg(ssq + (int64_t)s * T + t0 + tid);
+            const float r = 1.f / sqrtf(ss * inv_nC + eps);
+            rg[tid] = r;
+            rstd[t0 + tid] = r;
+        }
+        float qv[(kTokGroup * D::kN + kActThreads - 1) / kActThreads];
 #pragma unroll
-        for (int ww = 0; ww < kActWarps; ++ww) v += red[ww][c];
-        if (c < N) atomicAdd(db + c, v); else atomicAdd(dalpha + (c - N), v);
+        for (int it = 0; it < (kTokGroup * D::kN + kActThreads - 1) / kActThreads; ++it) {
+            const int i = tid + it * kActThreads;
+            qv[it] = 0.f;
+            if (i < nt * D::kN) {
+                const int tl = i / D::kN, c = i - tl * D::kN;
+                for (int s = 0; s < ksplit; ++s) qv[it] += __ldg(qpart + ((int64_t)s * T + t0 + tl) * Npad + c);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int it = 0; it < (kTokGroup * D::kN + kActThreads - 1) / kActThreads; ++it) {
+            const int i = tid + it * kActThreads;
+            if (i < nt * D::kN) {
+                const int tl = i / D::kN, c = i - tl * D::kN;
+                const float pv = qv[it] * rg[tl];
+                pg[tl][c] = pv;
+                p_saved[(t0 + tl) * D::kN + c] = pv;
+            }
+        }
+        __syncthreads();
+        // A: one thread per token
+        if (tid < nt) lite_thread_fwd<N_>(pg[tid], og[tid], b_s, a_res, a_pre, a_post, klist_s);
+        __syncthreads();
+        // W: coalesced write-out of the mappings
+        for (int i = tid; i < nt * D::kOut; i += kActThreads) {
+            const int tl = i / D::kOut, c = i - tl * D::kOut;
+            const int64_t t = t0 + tl;
+            const float v = og[tl][c];
+            if (c < D::kFact) a_saved[t * D::kFact + c] = v;
+            else if (c < D::kFact + D::kNN) H_res[t * D::kNN + (c - D::kFact)] = v;
+            else if (c < D::kFact + D::kNN + N_) H_pre[t * N_ + (c - D::kFact - D::kNN)] = v;
+            else H_post[t * N_ + (c - D::kFact - D::kNN - N_)] = v;
+        }
+        // P: u[t,:] = sum_j H_pre[t,j] x[t,j,:]  (two vectors per thread in flight)
+        for (int i0 = tid; i0 < nt * C8; i0 += 2 * kActThreads) {
+            const int i1 = i0 + kActThreads;
+            const bool has1 = i1 < nt * C8;
+            const int tl0 = i0 / C8, cv0 = i0 - tl0 * C8;
+            const int tl1 = has1 ? i1 / C8 : tl0, cv1 = has1 ? i1 - tl1 * C8 : cv0;
+            uint4 v0[N_], v1[N_];
+#pragma unroll
+            for (int j = 0; j < N_; ++j) v0[j] = ld_stream(x + ((t0 + tl0) * N_ + j) * C8 + cv0);
+#pragma unroll
+            for (int j = 0; j < N_; ++j) v1[j] = ld_stream(x + ((t0 + tl1) * N_ + j) * C8 + cv1);
+            float acc0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, acc1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+            for (int j = 0; j < N_; ++j) {
+                const float h0 = og[tl0][D::kFact + D::kNN + j], h1 = og[tl1][D::kFact + D::kNN + j];
+                float f0[8], f1[8];
+                unpack8(v0[j], f0);
+                unpack8(v1[j], f1);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { acc0[e] = fmaf(h0, f0[e], acc0[e]); acc1[e] = fmaf(h1, f1[e], acc1[e]); }
+            }
+            st_stream(u + (t0 + tl0) * C8 + cv0, pack8(acc0));
+            if (has1) st_stream(u + (t0 + tl1) * C8 + cv1, pack8(acc1));
+        }
+        __syncthreads();
     }
+}
+
+// Backward of one token by one thread.  in: a | p | dH_res | H_pre | H_post | dH_post | rstd (shared memory);
+// orow: e[0..kN) | kappa | dz[0..kN).
+template <int N_>
+__device__ __forceinline__ void lite_thread_bwd(const float* in, const float* dhpre, float* orow, const uint8_t* sigma_s,
+                                                float a_res, float a_pre, float a_post, float inv_nC) {
+    using D = LiteDims<N_>;
+    const float* a = in;
+    const float* pt = in + D::kFact;
+    const float* dh = pt + D::kN;
+    const float* hpre = dh + D::kNN;
+    const float* hpost = hpre + N_;
+    const float* dhpost = hpost + N_;
+    const float rs = dhpost[N_];
+    float dot = 0.f;
+#pragma unroll
+    for (int k = 0; k < D::kFact; ++k) {
+        float d = 0.f;
+#pragma unroll
+        for (int i = 0; i < N_; ++i) d += dh[i * N_ + sigma_s[k * N_ + i]];       // Eq. (5): dL/da_k
+        dot = fmaf(a[k], d, dot);
+    }
+    float kap = 0.f;
+#pragma unroll
+    for (int k = 0; k < D::kFact; ++k) {
+        float d = 0.f;
+#pragma unroll
+        for (int i = 0; i < N_; ++i) d += dh[i * N_ + sigma_s[k * N_ + i]];
+        const float dz = a[k] * (d - dot), ed = a_res * dz, pv = pt[k];
+        orow[k] = rs * ed;
+        orow[D::kN + 1 + k] = dz;
+        kap = fmaf(ed, pv, kap);
+    }
+#pragma unroll
+    for (int j = 0; j < N_; ++j) {
+        {
+            const float h = hpre[j], dz = dhpre[j] * h * (1.f - h), ed = a_pre * dz, pv = pt[D::kFact + j];
+            orow[D::kFact + j] = rs * ed; orow[D::kN + 1 + D::kFact + j] = dz; kap = fmaf(ed, pv, kap);
+        }
+        {
+            const float h = hpost[j], dz = dhpost[j] * h * (1.f - 0.5f * h), ed = a_post * dz, pv = pt[D::kFact + N_ + j];
+            orow[D::kFact + N_ + j] = rs * ed; orow[D::kN + 1 + D::kFact + N_ + j] = dz; kap = fmaf(ed, pv, kap);
+        }
+    }
+    orow[D::kN] = rs * rs * kap * inv_nC;
+}
+
+template <int N_>
+__global__ void __launch_bounds__(kActThreads, 3) lite_tailpre_t_k(
+    int64_t T, int C8, float inv_nC, const uint4* __restrict__ x, const uint4* __restrict__ du,
+    const float* __restrict__ a_saved, const float* __restrict__ p, const float* __restrict__ rstd,
+    const float* __restrict__ alpha, const float* __restrict__ H_pre, const float* __restrict__ H_post,
+    const float* __restrict__ dH_res, const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa,
+    float* db, float* dalpha) {
+    using D = LiteDims<N_>;
+    __shared__ uint8_t sigma_s[D::kFact * N_];
+    __shared__ float in_s[kTokGroup][D::kIn + 1];
+    __shared__ float dhp_s[kTokGroup][N_];
+    __shared__ float og[kTokGroup][2 * D::kN + 3];
+    __shared__ float dal_s[3];
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    for (int i = tid; i < D::kFact * N_; i += kActThreads) sigma_s[i] = c_perm[N_].sigma[i];
+    if (tid < 3) dal_s[tid] = 0.f;
+    const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
+    float db_col = 0.f, dal_col = 0.f;             // thread c < kN: column c of db, and sum_t dz[t,c] p[t,c]
+    constexpr int o_p = D::kFact, o_dhres = o_p + D::kN, o_hpre = o_dhres + D::kNN, o_hpost = o_hpre + N_,
+                  o_dhpost = o_hpost + N_, o_rstd = o_dhpost + N_;
+    __syncthreads();
+    const int64_t ngroups = (T + kTokGroup - 1) / kTokGroup;
+    for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
+        const int64_t t0 = grp * kTokGroup;
+        const int nt = (T - t0 < kTokGroup) ? (int)(T - t0) : kTokGroup;
+        // L: stage the per-token inputs with cp.async (they arrive while D streams)
+        for (int i = tid; i < nt * D::kIn; i += kActThreads) {
+            const int tl = i / D::kIn, c = i - tl * D::kIn;
+            const int64_t t = t0 + tl;
+            const float* src;
+            if (c < o_p) src = a_saved + t * D::kFact + c;
+            else if (c < o_dhres) src = p + t * D::kN + (c - o_p);
+            else if (c < o_hpre) src = dH_res + t * D::kNN + (c - o_dhres);
+            else if (c < o_hpost) src = H_pre + t * N_ + (c - o_hpre);
+            else if (c < o_dhpost) src = H_post + t * N_ + (c - o_hpost);
+            else if (c < o_rstd) src = dH_post + t * N_ + (c - o_dhpost);
+            else src = rstd + t;
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&in_s[tl][c])), "l"(src) : "memory");
+        }
+        cp_async_commit();
+        // D: dH_pre[j] = <du, x_j>, one warp per token
+        for (int tl = w; tl < nt; tl += kActWarps) {
+            const int64_t t = t0 + tl;
+            float r[N_];
+#pragma unroll
+            for (int j = 0; j < N_; ++j) r[j] = 0.f;
+            for (int cv = lane; cv < C8; cv += 64) {               // two vectors per lane in flight
+                const int cw = cv + 32;
+                const bool has1 = cw < C8;
+                uint4 xv[N_], xw[N_], dv, dw = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int j = 0; j < N_; ++j) xv[j] = ld_stream(x + (t * N_ + j) * C8 + cv);
+                dv = ld_stream(du + t * C8 + cv);
+                if (has1) {
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) xw[j] = ld_stream(x + (t * N_ + j) * C8 + cw);
+                    dw = ld_stream(du + t * C8 + cw);
+                }
+                float df[8], dg[8];
+                unpack8(dv, df);
+                unpack8(dw, dg);
+#pragma unroll
+                for (int j = 0; j < N_; ++j) {
+                    float xf[8];
+                    unpack8(xv[j], xf);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) r[j] = fmaf(df[e], xf[e], r[j]);
+                    if (has1) {
+                        unpack8(xw[j], xf);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) r[j] = fmaf(dg[e], xf[e], r[j]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < N_; ++j) { r[j] = warp_sum(r[j]); if (lane == j) dhp_s[tl][j] = r[j]; }
+        }
+        cp_async_wait<0>();
+        __syncthreads();
+        // A: one thread per token
+        if (tid < nt) lite_thread_bwd<N_>(in_s[tid], dhp_s[tid], og[tid], sigma_s, a_res, a_pre, a_post, inv_nC);
+        __syncthreads();
+        if (tid < D::kN) {
+            for (int tl = 0; tl < nt; ++tl) {
+                const float dz = og[tl][D::kN + 1 + tid];
+                db_col += dz;
+                dal_col = fmaf(dz, in_s[tl][o_p + tid], dal_col);
+            }
+        }
+        // W: e as a bf16 pair (and / or fp32), kappa
+        const int cols = eo.ehi ? eo.Kp : eo.Npad;
+        for (int i = tid; i < nt * cols; i += kActThreads) {
+            const int tl = i / cols, c = i - tl * cols;
+            const float v = (c < D::kN) ? og[tl][c] : 0.f;
+            const int64_t t = t0 + tl;
+            if (eo.ehi) {
+                __nv_bfloat16 h, l;
+                split_bf16(v, h, l);
+                eo.ehi[t * eo.Kp + c] = h;
+                eo.elo[t * eo.Kp + c] = l;
+            }
+            if (eo.e && c < eo.Npad) eo.e[t * eo.Npad + c] = v;
+        }
+        if (tid < nt) kappa[t0 + tid] = og[tid][D::kN];
+        __syncthreads();
+    }
+    // parameter-gradient partials of this block
+    (void)lane; (void)w;
+    if (tid < D::kN) {
+        atomicAdd(db + tid, db_col);
+        atomicAdd(&dal_s[tid < D::kFact ? 0 : (tid < D::kFact + N_ ? 1 : 2)], dal_col);
+    }
+    __syncthreads();
+    if (tid < 3) atomicAdd(dalpha + tid, dal_s[tid]);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -383,6 +897,13 @@ static int warp_grid(int64_t T, int sm_count) {
     return (int)(blocks < 1 ? 1 : blocks);
 }
 
+static int group_grid(int64_t T, int group, int sm_count) {
+    int64_t blocks = (T + group - 1) / group;
+    const int64_t cap = (int64_t)sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    return (int)(blocks < 1 ? 1 : blocks);
+}
+
 void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, const float* qpart, const float* ssq,
                          float eps, const float* b, const float* alpha, float* H_res, float* H_pre, float* H_post,
                          float* a_saved, float* p_saved, float* rstd, cudaStream_t s) {
@@ -405,6 +926,49 @@ void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float*
     lite_act_bwd_k<<<(int)blocks, kActThreads, 0, s>>>(T, c->n, c->nfact, 1.f / (float)(c->n * c->C), a, p, rstd,
                                                         alpha, H_pre, H_post, dH_res, dH_pre, dH_post, eo, kappa, db,
                                                         dalpha);
+}
+
+void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, const float* qpart, const float* ssq,
+                            float eps, const float* b, const float* alpha, float* H_res, float* H_pre, float* H_post,
+                            float* a_saved, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s) {
+    c->launches += 1;
+    const int C8 = c->C / 8;
+    const float inv = 1.f / (float)(c->n * c->C);
+#define MHCL_AP_T(N_) lite_act_premix_t_k<N_><<<group_grid(T, kTokGroup, c->sm_count), kActThreads, 0, s>>>( \
+        T, C8, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, \
+        (const uint4*)x, (uint4*)u)
+    switch (c->n) {
+        case 2: MHCL_AP_T(2); break;
+        case 3: MHCL_AP_T(3); break;
+        case 4: MHCL_AP_T(4); break;
+        default:    // n = 5: 120 logits do not fit a thread's registers; one warp per token
+            lite_act_premix_k<5><<<group_grid(T, kGroupTok, c->sm_count), kActThreads, 0, s>>>(
+                T, C8, c->nfact, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b, alpha, H_res, H_pre, H_post, a_saved,
+                p_saved, rstd, (const uint4*)x, (uint4*)u);
+    }
+#undef MHCL_AP_T
+}
+
+void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const void* du, const float* a, const float* p,
+                         const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
+                         const float* dH_res, const float* dH_post, float* e, int Npad, void* ehi, void* elo, int Kp,
+                         float* kappa, float* db, float* dalpha, cudaStream_t s) {
+    c->launches += 1;
+    const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
+    const int C8 = c->C / 8;
+    const float inv = 1.f / (float)(c->n * c->C);
+#define MHCL_TP_T(N_) lite_tailpre_t_k<N_><<<group_grid(T, kTokGroup, c->sm_count), kActThreads, 0, s>>>( \
+        T, C8, inv, (const uint4*)x, (const uint4*)du, a, p, rstd, alpha, H_pre, H_post, dH_res, dH_post, eo, kappa, db, dalpha)
+    switch (c->n) {
+        case 2: MHCL_TP_T(2); break;
+        case 3: MHCL_TP_T(3); break;
+        case 4: MHCL_TP_T(4); break;
+        default:
+            lite_tailpre_k<5><<<group_grid(T, 16, c->sm_count), kActThreads, 0, s>>>(
+                T, C8, c->nfact, inv, (const uint4*)x, (const uint4*)du, a, p, rstd, alpha, H_pre, H_post, dH_res,
+                dH_post, eo, kappa, db, dalpha);
+    }
+#undef MHCL_TP_T
 }
 
 void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,

@@ -235,11 +235,26 @@ int mhclite_postres_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
 int mhclite_pre_fwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W, const float* b,
                           const float* alpha, const float* gain, float eps, float* H_res, float* H_pre, float* H_post,
                           float* a_saved, float* p_saved, float* rstd, mhclite_bf16* u, void* stream) {
-    MHCL_REQUIRE_CTX(ctx);
-    if (T > 0) MHCL_PTR(ctx, u);
-    int rc = mhclite_coeffs_fwd(ctx, T, x, W, b, alpha, gain, eps, H_res, H_pre, H_post, a_saved, p_saved, rstd, stream);
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, W); MHCL_PTR(ctx, b); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain);
+    MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, a_saved);
+    MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd); MHCL_PTR(ctx, u);
+    if (!(eps >= 0.f)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "eps must be >= 0");
+    Workspace w;
+    int rc = need_workspace(ctx, T, 0, &w);
     if (rc) return rc;
-    return mhclite_premix_fwd(ctx, T, x, H_pre, u, stream);
+    MHCL_DEVICE(ctx);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int N = n_cols(ctx->n, 0);
+    const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
+    launch_pack_w(ctx, pp, N, W, gain, w.Wp, s);
+    MHCL_LAUNCH_CHECK(ctx, "pack_w");
+    launch_proj_fwd_mma(ctx, T, pp, x, w.Wp, w.qpart, w.ssq, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_fwd_mma");
+    launch_lite_act_premix(ctx, T, pp, w.qpart, w.ssq, eps, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, x, u, s);
+    MHCL_LAUNCH_CHECK(ctx, "lite_act_premix");
+    return MHCLITE_OK;
 }
 
 // ---- backward ------------------------------------------------------------------------------------
@@ -324,11 +339,10 @@ int mhclite_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, c
     rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
     if (rc) return rc;
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
-    launch_premix_bwd(ctx, T, x, H_pre, du, w.dH_pre, nullptr, 0, s);
-    MHCL_LAUNCH_CHECK(ctx, "premix_bwd");
-    launch_lite_act_bwd(ctx, T, w.Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, w.dH_pre, dH_post,
-                        tp.supported ? nullptr : w.e, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
-    MHCL_LAUNCH_CHECK(ctx, "lite_act_bwd");
+    launch_lite_tailpre(ctx, T, x, du, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_post,
+                        tp.supported ? nullptr : w.e, w.Npad, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db,
+                        dalpha, s);
+    MHCL_LAUNCH_CHECK(ctx, "lite_tailpre");
     return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W, gain, dx, 0, dW, dgain, accumulate_params, s);
 }
 

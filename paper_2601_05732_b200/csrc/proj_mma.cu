@@ -201,7 +201,7 @@ ProjPlan plan_proj(int n, int C, int64_t T, int N, int sm_count) {
     p.nchunks = (n * C + kChunkK - 1) / kChunkK;
     p.ksteps = p.nchunks * 4;
     const int64_t tiles = (T + kTileTok - 1) / kTileTok;
-    int ks = tiles > 0 ? (int)((2 * (int64_t)sm_count + tiles - 1) / tiles) : 1;
+    int ks = tiles > 0 ? (int)((2 * (int64_t)sm_count) / tiles) : 1;      // fill 2 CTAs per SM, one wave
     if (ks > kMaxKSplit) ks = kMaxKSplit;
     if (ks > p.nchunks) ks = p.nchunks;
     if (ks < 1) ks = 1;

@@ -9,7 +9,7 @@
 //
 // One CTA owns a slice of 64 channels (of every stream) and walks over a range of tokens in tiles of 32,
 // so that the W' slice and the G accumulators stay on chip: x, g, du and e stream through shared memory
-// (cp.async, 3 stages).  Both contractions run on mma.sync.m16n8k16 (bf16, fp32 accumulate):
+// (cp.async, double buffered, two CTAs per SM).  Both contractions run on mma.sync.m16n8k16 (bf16, fp32 accumulate):
 //   (1) M = tokens, N = channels, K = projection columns; e and W' rounded to bf16 (this term is a small
 //       part of a bf16 output); the columns of each n-tile are permuted so that a thread ends up with 8
 //       consecutive channels of a token and stores 16 bytes.
@@ -25,7 +25,7 @@ namespace mhcl {
 
 constexpr int kTT = 32;            // tokens per tile
 constexpr int kCS = 64;            // channels per slice (128 bytes of bf16 per row)
-constexpr int kTailStages = 3;
+constexpr int kTailStages = 2;    // two CTAs per SM, each double-buffered
 
 // Row swizzle of the 128-byte tiles: 8 consecutive rows get 8 different 16-byte slots (ldmatrix), and
 // consecutive rows differ in bit 2 (a quarter warp reading 4 pieces of 2 consecutive rows is conflict free).
@@ -53,7 +53,8 @@ struct TailCfg {
     static constexpr int kDu = kTT * 128;
     static constexpr int kEStride = KS * 32 + 16;                  // bytes per row of an e tile (padded)
     static constexpr int kE = kTT * kEStride;
-    static constexpr int kCoefFloats = kTT * (1 + (FUSED ? N_ * N_ + N_ : 0));
+    static constexpr int kHresStride = N_ * N_ + 1;               // odd stride: rows of different tokens in different banks
+    static constexpr int kCoefFloats = kTT * (1 + (FUSED ? kHresStride + N_ : 0));
     static constexpr int oG = kX, oDu = oG + (FUSED ? kX : 0), oEh = oDu + (FUSED ? kDu : 0), oEl = oEh + kE,
                          oCoef = oEl + kE;
     static constexpr int kStage = (oCoef + kCoefFloats * 4 + 127) / 128 * 128;
@@ -65,7 +66,7 @@ struct TailCfg {
 };
 
 template <int N_, int KS, bool FUSED, bool ACC>
-__global__ void __launch_bounds__(256, 1) tail_mma_k(const TailArgs a) {
+__global__ void __launch_bounds__(256, 2) tail_mma_k(const TailArgs a) {
     using Cfg = TailCfg<N_, KS, FUSED>;
     constexpr int NT8 = 2 * KS;                                    // 8-column tiles of the projection
     extern __shared__ __align__(1024) unsigned char smem[];
@@ -138,7 +139,11 @@ __global__ void __launch_bounds__(256, 1) tail_mma_k(const TailArgs a) {
             int64_t idx;
             if (i < kTT) { src = a.kappa; idx = tt0 + i; if (idx >= t_end) idx = -1; }
             else if (i < kTT + kTT * N_) { src = a.H_pre; idx = tt0 * N_ + (i - kTT); if (idx >= t_end * N_) idx = -1; }
-            else { src = a.H_res; idx = tt0 * N_ * N_ + (i - kTT - kTT * N_); if (idx >= t_end * N_ * N_) idx = -1; }
+            else {
+                const int r = i - kTT - kTT * N_, tl = r / Cfg::kHresStride, e = r - tl * Cfg::kHresStride;
+                src = a.H_res; idx = (tt0 + tl) * N_ * N_ + e;
+                if (e >= N_ * N_ || tt0 + tl >= t_end) idx = -1;
+            }
             cp_async4(sb + Cfg::oCoef + i * 4, idx >= 0 ? (const void*)(src + idx) : (const void*)a.x, idx >= 0 ? 4 : 0);
         }
     };
@@ -223,7 +228,7 @@ __global__ void __launch_bounds__(256, 1) tail_mma_k(const TailArgs a) {
                             float gf[8];
                             const int grow = i * kTT + tl;
                             unpack8(*reinterpret_cast<const uint4*>(st + Cfg::oG + grow * 128 + ((pc ^ swz(grow)) << 4)), gf);
-                            const float hr = coef[kTT + kTT * N_ + tl * N_ * N_ + i * N_ + j];
+                            const float hr = coef[kTT + kTT * N_ + tl * Cfg::kHresStride + i * N_ + j];
 #pragma unroll
                             for (int e = 0; e < 8; ++e) o[e] = fmaf(hr, gf[e], o[e]);
                         }
@@ -320,8 +325,8 @@ TailPlan plan_tail(int n, int C, int64_t T, int N, int sm_count) {
     p.KS = p.Kp / 16;
     p.supported = p.KS <= 3;
     p.slices = (C + kCS - 1) / kCS;
-    if (sm_count > 148) sm_count = 148;                       // the workspace is sized for at most 148 CTAs
-    int64_t splits = sm_count / p.slices;
+    if (sm_count > 148) sm_count = 148;                       // the workspace is sized for at most 2 x 148 CTAs
+    int64_t splits = (2 * sm_count) / p.slices;
     const int64_t max_splits = (T + kTT - 1) / kTT;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
