@@ -136,15 +136,19 @@ proj_fwd_mma_k(int64_t T, int nC, int nchunks, int chunks_per_split, const __nv_
                     }
                 }
             }
+            // the hi and lo products of one accumulator are issued far apart: back-to-back MMAs on the same
+            // accumulator would wait for each other
+            uint4 bw[NTW];
 #pragma unroll
-            for (int j = 0; j < NTW; ++j) {
-                const uint4 bw = ws[(ks * NT + wn * NTW + j) * 32 + lane];
+            for (int j = 0; j < NTW; ++j) bw[j] = ws[(ks * NT + wn * NTW + j) * 32 + lane];
 #pragma unroll
-                for (int mt = 0; mt < 4; ++mt) {
-                    mma_bf16(acc[mt][j], a[mt], bw.x, bw.y);
-                    mma_bf16(acc[mt][j], a[mt], bw.z, bw.w);
-                }
-            }
+            for (int j = 0; j < NTW; ++j)
+#pragma unroll
+                for (int mt = 0; mt < 4; ++mt) mma_bf16(acc[mt][j], a[mt], bw[j].x, bw[j].y);
+#pragma unroll
+            for (int j = 0; j < NTW; ++j)
+#pragma unroll
+                for (int mt = 0; mt < 4; ++mt) mma_bf16(acc[mt][j], a[mt], bw[j].z, bw[j].w);
         }
     }
     cp_async_wait<0>();

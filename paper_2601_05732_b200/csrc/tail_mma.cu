@@ -246,32 +246,43 @@ __global__ void __launch_bounds__(256, 2) tail_mma_k(const TailArgs a) {
         }
 
         // ---- (2) G += x^T e -----------------------------------------------------------------------------
+        // The e fragments are the same for every m-tile: they are fetched once per (k-step, column pair);
+        // hi and lo products of one accumulator are kept apart in the issue order.
 #pragma unroll
-        for (int mi = 0; mi < Cfg::kMT2; ++mi) {
-            const int mtile = warp + 8 * mi;                       // (stream j, 16-channel block cb)
-            if (mtile >= N_ * 4) break;
-            const int j = mtile >> 2, cb = mtile & 3;
+        for (int kt = 0; kt < kTT / 16; ++kt) {
+            uint32_t af[Cfg::kMT2][4];
 #pragma unroll
-            for (int kt = 0; kt < kTT / 16; ++kt) {
-                uint32_t af[4];
-                {
+            for (int mi = 0; mi < Cfg::kMT2; ++mi) {
+                const int mtile = warp + 8 * mi;                   // (stream j, 16-channel block cb)
+                if (mtile < N_ * 4) {
                     // matrices: (t 0-7, piece 2cb), (t 0-7, piece 2cb+1), (t 8-15, piece 2cb), (t 8-15, piece 2cb+1)
+                    const int j = mtile >> 2, cb = mtile & 3;
                     const int row = j * kTT + kt * 16 + (lane & 7) + ((lane >> 4) & 1) * 8;
                     const int pc = 2 * cb + ((lane >> 3) & 1);
-                    ldmatrix_x4_trans(af, sb + row * 128 + ((pc ^ swz(row)) << 4));
+                    ldmatrix_x4_trans(af[mi], sb + row * 128 + ((pc ^ swz(row)) << 4));
+                }
+            }
+#pragma unroll
+            for (int jp = 0; jp < KS; ++jp) {                      // pairs of 8-column tiles
+                uint32_t bh[4], bl[4];
+                // matrices: (t 0-7, cols 16jp..+7), (t 8-15, same), (t 0-7, cols 16jp+8..), (t 8-15, same)
+                const int row = kt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+                const uint32_t off = row * Cfg::kEStride + (2 * jp + (lane >> 4)) * 16;
+                ldmatrix_x4_trans(bh, sb + Cfg::oEh + off);
+                ldmatrix_x4_trans(bl, sb + Cfg::oEl + off);
+#pragma unroll
+                for (int mi = 0; mi < Cfg::kMT2; ++mi) {
+                    if (warp + 8 * mi < N_ * 4) {
+                        mma_bf16(G[mi][2 * jp], af[mi], bh[0], bh[1]);
+                        mma_bf16(G[mi][2 * jp + 1], af[mi], bh[2], bh[3]);
+                    }
                 }
 #pragma unroll
-                for (int jp = 0; jp < KS; ++jp) {                  // pairs of 8-column tiles
-                    uint32_t bh[4], bl[4];
-                    // matrices: (t 0-7, cols 16jp..+7), (t 8-15, same), (t 0-7, cols 16jp+8..), (t 8-15, same)
-                    const int row = kt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-                    const uint32_t off = row * Cfg::kEStride + (2 * jp + (lane >> 4)) * 16;
-                    ldmatrix_x4_trans(bh, sb + Cfg::oEh + off);
-                    ldmatrix_x4_trans(bl, sb + Cfg::oEl + off);
-                    mma_bf16(G[mi][2 * jp], af, bh[0], bh[1]);
-                    mma_bf16(G[mi][2 * jp], af, bl[0], bl[1]);
-                    mma_bf16(G[mi][2 * jp + 1], af, bh[2], bh[3]);
-                    mma_bf16(G[mi][2 * jp + 1], af, bl[2], bl[3]);
+                for (int mi = 0; mi < Cfg::kMT2; ++mi) {
+                    if (warp + 8 * mi < N_ * 4) {
+                        mma_bf16(G[mi][2 * jp], af[mi], bl[0], bl[1]);
+                        mma_bf16(G[mi][2 * jp + 1], af[mi], bl[2], bl[3]);
+                    }
                 }
             }
         }
