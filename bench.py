@@ -147,7 +147,7 @@ def run_reference(args, wl, rank):
 # ----------------------------------------------------------------------------------------------
 def run_ours(args, wl, rank, world):
     import torch
-    import torch.distributed as dist
+    from paper_2601_05732_b200 import dist as D
     from paper_2601_05732_b200 import synth
     from paper_2601_05732_b200 import layer as L
     from paper_2601_05732_b200.binding import MhcLite
@@ -163,11 +163,11 @@ def run_ours(args, wl, rank, world):
 
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    D.init(world, "nccl", dev)
 
     n, C, T = wl.n, wl.C, wl.T
-    inp = synth.make_layer_inputs(n, C, T, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std, shard=rank)
+    inp = synth.make_layer_inputs(n, C, T, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std,
+                                  shard=D.shard_of(rank))
     ctx = MhcLite(n, C, local)
     P = L.LayerParams(inp["W"], inp["b"], inp["alpha"], inp["gain"], dev)
     B = L.LayerBuffers(ctx, T, "lite")
@@ -184,9 +184,7 @@ def run_ours(args, wl, rank, world):
             L.tail_bwd(ctx, P, B, x, g, du, eps, fused)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        D.barrier(world)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -210,10 +208,7 @@ def run_ours(args, wl, rank, world):
         step()
     torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
-    if world > 1:
-        tt = torch.tensor([ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt.item())
+    ms = D.max_over_ranks(ms, world, dev)
 
     # ---- per-stage device time (same launch configuration), for the roofline of the dominant stage
     stages = [("pre_fwd", lambda: L.pre_fwd(ctx, P, B, x, eps, fused)), ("post_fwd", lambda: L.post_fwd(ctx, B, x, y))]
@@ -248,14 +243,42 @@ def run_ours(args, wl, rank, world):
         b_.record()
         barrier()
         ms_e2e = a.elapsed_time(b_)
-        if world > 1:
-            tt = torch.tensor([ms_e2e], device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms_e2e = float(tt.item())
+        ms_e2e = D.max_over_ranks(ms_e2e, world, dev)
         h2d = sum(t.numel() * 2 for t in (hx, hy, hg, hdu))
         d2h = sum(t.numel() * 2 for t in (hu, hxn, hdy, hdx))
-        e2e = {"value": world * T * k_e2e / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": D.job_tokens_per_s(T, world, k_e2e, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / k_e2e}
+
+    # ---- the mHC (20 Sinkhorn-Knopp iterations) path on the same shapes, for comparison --------
+    sk20 = None
+    if not args.no_sk and wl.backward and rank == 0:
+        ski = synth.make_layer_inputs(n, C, T, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std,
+                                      kind="sk", shard=D.shard_of(rank))
+        Ps = L.LayerParams(ski["W"], ski["b"], ski["alpha"], ski["gain"], dev)
+        Bs = L.LayerBuffers(ctx, T, "sk")
+
+        def sk_step():
+            L.pre_fwd(ctx, Ps, Bs, x, eps, True)
+            L.post_fwd(ctx, Bs, x, y)
+            L.post_bwd(ctx, Bs, x, y, g, True)
+            L.tail_bwd(ctx, Ps, Bs, x, g, du, eps, True)
+
+        for _ in range(3):
+            sk_step()
+        torch.cuda.synchronize()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.steps):
+            sk_step()
+        b_.record()
+        torch.cuda.synchronize()
+        ms_sk = a.elapsed_time(b_) / args.steps
+        gap = torch.empty(T, device=dev); gap_l = torch.empty(T, device=dev)
+        ctx.ds_gap(Bs.H_res, gap, None); ctx.ds_gap(B.H_res, gap_l, None)
+        torch.cuda.synchronize()
+        sk20 = {"tokens_per_s": T / (ms_sk * 1e-3), "ms_per_step": ms_sk, "iters": 20,
+                "lite_over_sk20": ms_sk / (ms / args.steps) if world == 1 else None,
+                "l1_gap_max_sk20": float(gap.max()), "l1_gap_max_lite": float(gap_l.max())}
 
     if rank == 0:
         peak, peak_kind = load_peaks()
@@ -270,18 +293,17 @@ def run_ours(args, wl, rank, world):
                     "stage_ms": stage_ms,
                     "stage_gbs": {k: bpt[k] * T / (v * 1e-3) / 1e9 for k, v in stage_ms.items()}}
         line = {
-            "metric": METRIC, "value": world * T * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": D.job_tokens_per_s(T, world, args.steps, ms), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, f32 accumulate",
             "data": "synthetic",
             "config": {"workload": wl.name, "n": n, "C": C, "T_per_gpu": T, "passes": "fwd+bwd" if wl.backward else "fwd", "calls": "fused" if fused else "unfused",
                        "note": wl.note, "l2": "inputs larger than L2 (working set %.0f MB)" % (total_bytes / 1e6)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-            "cpu_baseline": cpu_baseline,
+            "cpu_baseline": cpu_baseline, "sk20_comparison": sk20,
         }
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    D.shutdown()
 
 
 def main():
@@ -295,6 +317,7 @@ def main():
     ap.add_argument("--cpu-sample", type=int, default=16384, help="tokens of the oracle's timed sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sk", action="store_true", help="skip the SK-20 comparison path")
     ap.add_argument("--unfused", action="store_true", help="time the un-fused call sequence (six entry points)")
     args = ap.parse_args()
 

@@ -202,6 +202,21 @@ MHCLITE_API int mhc_sk20_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_b
                         float* dW, float* db, float* dalpha, float* dgain, int accumulate_params,
                         void* stream);
 
+/* The SK path's counterpart of mhclite_tail_bwd_fused: dH_pre, the SK activation backward and the
+ * projection backward, with dx = H_res^T g + H_pre du + (gradient through the mappings) written once.
+ * dH_res and dH_post come from mhclite_postres_bwd called with dx = NULL (the streaming calls
+ * premix_* / postres_* take coefficients, so they serve both paths). */
+MHCLITE_API int mhc_sk20_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x,
+                        const float* W_sk, const float* b_sk, const float* alpha, const float* gain,
+                        float eps, int iters,
+                        const float* p_saved, const float* rstd,
+                        const float* H_res, const float* H_pre, const float* H_post,
+                        const mhclite_bf16* g, const mhclite_bf16* du,
+                        const float* dH_res, const float* dH_post,
+                        mhclite_bf16* dx,
+                        float* dW, float* db, float* dalpha, float* dgain, int accumulate_params,
+                        void* stream);
+
 /* ---- doubly-stochastic diagnostics (paper Section 3.1 footnote) -------------------------------- */
 
 /* Per token: l1_err[t] = ||H 1 - 1||_1 + ||H^T 1 - 1||_1 and colsum_dev[t] = max_j |sum_i H[i][j] - 1|

@@ -53,6 +53,8 @@ SIGNATURES = {
     "mhc_sk20_coeffs_fwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _i, _p, _p, _p, _p, _p, _p]),
     "mhc_sk20_coeffs_bwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _i, _p, _p, _p, _p, _p, _p, _p, _p, _i,
                                  _p, _p, _p, _p, _i, _p]),
+    "mhc_sk20_tail_bwd_fused": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _i, _p, _p, _p, _p, _p, _p, _p, _p, _p,
+                                     _p, _p, _p, _p, _p, _i, _p]),
     "mhclite_ds_gap": (_i, [_p, _i64, _p, _p, _p, _p]),
     "mhclite_step_host_bytes": (_sz, [_i, _i, _i64]),
     "mhclite_step_host": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p, _i,
@@ -161,6 +163,7 @@ class MhcLite:
     # -- forward ---------------------------------------------------------------------------------
     def coeffs_fwd(self, x, W, b, alpha, gain, eps, H_res, H_pre, H_post, a_saved, p_saved, rstd):
         t, f, h = self._torch, self._torch.float32, self._torch.bfloat16
+        self.ensure_workspace(x.shape[0], 0)
         self._check(self.lib.mhclite_coeffs_fwd(
             self._h, x.shape[0], self._ptr(x, h), self._ptr(W, f), self._ptr(b, f), self._ptr(alpha, f),
             self._ptr(gain, f), float(eps), self._ptr(H_res, f), self._ptr(H_pre, f), self._ptr(H_post, f),
@@ -251,6 +254,17 @@ class MhcLite:
             self._ptr(H_post, f), self._ptr(dH_res, f), self._ptr(dH_pre, f), self._ptr(dH_post, f), self._ptr(dx, h),
             int(accumulate_dx), self._ptr(dW, f), self._ptr(db, f), self._ptr(dalpha, f), self._ptr(dgain, f),
             int(accumulate_params), self._stream()), "mhc_sk20_coeffs_bwd")
+
+    def sk20_tail_bwd_fused(self, x, W_sk, b_sk, alpha, gain, eps, iters, p_saved, rstd, H_res, H_pre, H_post, g, du,
+                            dH_res, dH_post, dx, dW, db, dalpha, dgain, accumulate_params=False):
+        f, h = self._torch.float32, self._torch.bfloat16
+        self.ensure_workspace(x.shape[0], 1)
+        self._check(self.lib.mhc_sk20_tail_bwd_fused(
+            self._h, x.shape[0], self._ptr(x, h), self._ptr(W_sk, f), self._ptr(b_sk, f), self._ptr(alpha, f),
+            self._ptr(gain, f), float(eps), int(iters), self._ptr(p_saved, f), self._ptr(rstd, f), self._ptr(H_res, f),
+            self._ptr(H_pre, f), self._ptr(H_post, f), self._ptr(g, h), self._ptr(du, h), self._ptr(dH_res, f),
+            self._ptr(dH_post, f), self._ptr(dx, h), self._ptr(dW, f), self._ptr(db, f), self._ptr(dalpha, f),
+            self._ptr(dgain, f), int(accumulate_params), self._stream()), "mhc_sk20_tail_bwd_fused")
 
     def kernel_launches(self) -> int:
         return int(self.lib.mhclite_kernel_launches(self._h))

@@ -401,6 +401,37 @@ int mhc_sk20_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
                          dgain, accumulate_params, s);
 }
 
+int mhc_sk20_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W_sk, const float* b_sk,
+                            const float* alpha, const float* gain, float eps, int iters, const float* p_saved,
+                            const float* rstd, const float* H_res, const float* H_pre, const float* H_post,
+                            const mhclite_bf16* g, const mhclite_bf16* du, const float* dH_res, const float* dH_post,
+                            mhclite_bf16* dx, float* dW, float* db, float* dalpha, float* dgain,
+                            int accumulate_params, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    (void)eps;
+    if (iters < 1 || iters > 64) return fail(ctx, MHCLITE_ERR_BAD_ARG, "iters must be in [1,64]");
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, W_sk); MHCL_PTR(ctx, b_sk); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain);
+    MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd); MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post);
+    MHCL_PTR(ctx, g); MHCL_PTR(ctx, du); MHCL_PTR(ctx, dH_res); MHCL_PTR(ctx, dH_post); MHCL_PTR(ctx, dx);
+    MHCL_PTR(ctx, dW); MHCL_PTR(ctx, db); MHCL_PTR(ctx, dalpha); MHCL_PTR(ctx, dgain);
+    Workspace w;
+    int rc = need_workspace(ctx, T, 1, &w);
+    if (rc) return rc;
+    MHCL_DEVICE(ctx);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int N = n_cols(ctx->n, 1);
+    rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
+    if (rc) return rc;
+    const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
+    launch_premix_bwd(ctx, T, x, H_pre, du, w.dH_pre, nullptr, 0, s);
+    MHCL_LAUNCH_CHECK(ctx, "premix_bwd");
+    launch_sk_act_bwd(ctx, T, w.Npad, iters, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, w.dH_pre, dH_post,
+                      tp.supported ? nullptr : w.e, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
+    MHCL_LAUNCH_CHECK(ctx, "sk_act_bwd");
+    return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W_sk, gain, dx, 0, dW, dgain, accumulate_params, s);
+}
+
 int mhclite_ds_gap(mhclite_ctx* ctx, int64_t T, const float* H_res, float* l1_err, float* colsum_dev, void* stream) {
     MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
     if (T == 0) return MHCLITE_OK;

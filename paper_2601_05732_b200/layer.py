@@ -69,14 +69,17 @@ def post_fwd(ctx: MhcLite, B: LayerBuffers, x, y):
 
 def post_bwd(ctx: MhcLite, B: LayerBuffers, x, y, g, fused=True):
     """Backward of the merge: B.dy, B.dH_res, B.dH_post (and, unfused, the H_res^T g part of B.dx)."""
-    skip_dx = fused and B.kind == "lite"          # the fused tail recomputes H_res^T g from g
+    skip_dx = fused                                # the fused tail recomputes H_res^T g from g
     ctx.postres_bwd(x, y, B.H_res, B.H_post, g, B.dy, B.dH_res, B.dH_post, None if skip_dx else B.dx, False)
 
 
 def tail_bwd(ctx: MhcLite, P: LayerParams, B: LayerBuffers, x, g, du, eps=1e-6, fused=True, iters=20,
              accumulate_params=False):
     """Everything after the sublayer's backward: B.dx and the parameter gradients."""
-    if B.kind == "sk":
+    if B.kind == "sk" and fused:
+        ctx.sk20_tail_bwd_fused(x, P.W, P.b, P.alpha, P.gain, eps, iters, B.p_saved, B.rstd, B.H_res, B.H_pre, B.H_post,
+                                g, du, B.dH_res, B.dH_post, B.dx, B.dW, B.db, B.dalpha, B.dgain, accumulate_params)
+    elif B.kind == "sk":
         ctx.premix_bwd(x, B.H_pre, du, B.dH_pre, B.dx, True)
         ctx.sk20_coeffs_bwd(x, P.W, P.b, P.alpha, P.gain, eps, iters, B.p_saved, B.rstd, B.H_pre, B.H_post,
                             B.dH_res, B.dH_pre, B.dH_post, B.dx, True, B.dW, B.db, B.dalpha, B.dgain,

@@ -27,7 +27,7 @@ import numpy as np
 
 __all__ = [
     "Workload", "WORKLOADS", "normal", "to_bf16_bits", "bf16_bits_to_f64",
-    "bf16_bits_to_f32", "n_logits", "make_layer_inputs", "paper_init_bias",
+    "bf16_bits_to_f32", "n_logits", "make_layer_inputs", "make_layer_params", "paper_init_bias", "normal_bf16",
 ]
 
 
@@ -38,6 +38,18 @@ def normal(seed: int, stream: int, shape, std: float = 1.0) -> np.ndarray:
     """fp64 N(0, std^2) samples from the counter-based stream (seed, stream)."""
     bitgen = np.random.Philox(key=[int(seed) & (2**64 - 1), int(stream) & (2**64 - 1)])
     return np.random.Generator(bitgen).standard_normal(size=shape, dtype=np.float64) * std
+
+
+def normal_bf16(seed: int, stream: int, shape, std: float = 1.0, chunk: int = 1 << 24) -> np.ndarray:
+    """bf16 bit patterns of N(0, std^2) samples of stream (seed, stream), drawn and rounded in chunks
+    (same values as to_bf16_bits(normal(...)), without the fp64 copy of the whole tensor)."""
+    total = int(np.prod(shape))
+    out = np.empty(total, dtype=np.uint16)
+    gen = np.random.Generator(np.random.Philox(key=[int(seed) & (2**64 - 1), int(stream) & (2**64 - 1)]))
+    for a in range(0, total, chunk):
+        b = min(total, a + chunk)
+        out[a:b] = to_bf16_bits(gen.standard_normal(size=b - a, dtype=np.float64) * std)
+    return out.reshape(shape)
 
 
 def to_bf16_bits(a: np.ndarray) -> np.ndarray:
@@ -156,10 +168,21 @@ def make_layer_inputs(n: int, C: int, T: int, seed: int, *, layer: int = 0,
     N = n_logits(n, kind)
     base = 16 * layer
     tok = 4096 * int(shard)                    # token tensors: one stream per shard
-    x = to_bf16_bits(normal(seed, base + _S_X + tok, (T, n, C)))
-    y = to_bf16_bits(normal(seed, base + _S_Y + tok, (T, C)))
-    g = to_bf16_bits(normal(seed, base + _S_G + tok, (T, n, C)))
-    du = to_bf16_bits(normal(seed, base + _S_DU + tok, (T, C)))
+    x = normal_bf16(seed, base + _S_X + tok, (T, n, C))
+    y = normal_bf16(seed, base + _S_Y + tok, (T, C))
+    g = normal_bf16(seed, base + _S_G + tok, (T, n, C))
+    du = normal_bf16(seed, base + _S_DU + tok, (T, C))
+    p = make_layer_params(n, C, seed, layer=layer, bias_std=bias_std, alpha=alpha, w_std=w_std, kind=kind,
+                          gain_std=gain_std)
+    return dict(x=x, y=y, g=g, du=du, W=p["W"], b=p["b"], alpha=p["alpha"], gain=p["gain"],
+                n=n, C=C, T=T, N=N, kind=kind)
+
+
+def make_layer_params(n: int, C: int, seed: int, *, layer: int = 0, bias_std: float = 0.0, alpha=0.01,
+                      w_std: float = 0.02, kind: str = "lite", gain_std: float = 0.0) -> dict:
+    """The parameters of layer `layer` alone (W, b, alpha, gain), as make_layer_inputs draws them."""
+    N = n_logits(n, kind)
+    base = 16 * layer
     sw, sb = (_S_W, _S_B) if kind == "lite" else (_S_WSK, _S_BSK)
     W = normal(seed, base + sw, (n * C, N), w_std).astype(np.float32)
     if bias_std > 0:
@@ -172,5 +195,4 @@ def make_layer_inputs(n: int, C: int, T: int, seed: int, *, layer: int = 0,
         gain = (1.0 + normal(seed, base + _S_GAIN, (n * C,), gain_std)).astype(np.float32)
     else:
         gain = np.ones(n * C, dtype=np.float32)
-    return dict(x=x, y=y, g=g, du=du, W=W, b=b, alpha=alpha3, gain=gain,
-                n=n, C=C, T=T, N=N, kind=kind)
+    return dict(W=W, b=b, alpha=alpha3, gain=gain, n=n, C=C, N=N, kind=kind)

@@ -5,9 +5,10 @@ Tolerances (they follow the arithmetic: bf16 storage rounds to 2^-9 relative, fp
 n*C <= 2^15 terms leaves ~1e-6 relative):
   bf16 tensors : |gpu - ref| <= 2e-2 |ref| + 1e-3 rms(ref)          for every element
   fp32 mappings: |gpu - ref| <= 1e-5 max(|ref|, rms(ref))           (H_res, H_pre, H_post, a, rstd)
-  saved projection p = x' W: 4e-5 max(|ref|, rms(ref)) -- W' enters the tensor cores as a bf16 pair
-                hi + lo, which leaves up to 2^-18 relative error per weight (about 1e-5 of rms(p) in the
-                tails); alpha scales it down by 100x before it reaches the mappings
+  saved projection p = x' W: 1e-4 max(|ref|, rms(ref)) -- W' enters the tensor cores as a bf16 pair
+                hi + lo (up to 2^-18 relative error per weight) and the tensor cores' fp32 accumulation
+                over n*C/8 steps adds a few 1e-5 of rms(p) at n*C = 7680; alpha scales this down by 100x
+                before it reaches the mappings, which are checked at 1e-5
   fp32 parameter gradients: |gpu - ref| <= 1e-3 max(|ref|, rms(ref)) (the binding tolerance is 2e-2)
 """
 import numpy as np
@@ -91,7 +92,7 @@ def oracle_bwd(inp, eps=1e-6, kind="lite", iters=20):
 def compare_forward(G, ref, coeff_rel=1e-5):
     B = G.B
     check_f32("rstd", host(B.rstd), ref["rstd"], coeff_rel)
-    check_f32("p_saved", host(B.p_saved), ref["p"], max(coeff_rel, 4e-5))
+    check_f32("p_saved", host(B.p_saved), ref["p"], max(coeff_rel, 1e-4))
     if G.kind == "lite":
         check_f32("a_saved", host(B.a_saved), ref["a"], coeff_rel)
     check_f32("H_res", host(B.H_res), ref["H_res"], coeff_rel)
@@ -111,19 +112,23 @@ def staged_dx_allowance(ref, fused):
     return 2.0 ** -8 * (np.abs(d1) + np.abs(d2))
 
 
-def dxhat_allowance(inp, dz, eps=1e-6):
+def dxhat_allowance_f(x, W, alpha, gain, dz, eps=1e-6):
     """Allowance for the projection-backward term of dx, sum_c e[t,c] W'[m,c]: the tensor-core kernel
     rounds both operands to bf16 (as bf16 mixed-precision training does for this matmul), so each
     product carries up to 2^-8 relative error: |error| <= 2^-8 sum_c |e[t,c]| |W'[m,c]|."""
-    o = oracle_inputs(inp)
-    x = o["x"]; T, n, C = x.shape
+    T, n, C = x.shape
     xh = x.reshape(T, n * C)
     rstd = 1.0 / np.sqrt((xh * xh).mean(axis=1) + eps)
     n_res = dz.shape[1] - 2 * n
-    av = np.concatenate([np.full(n_res, o["alpha"][0]), np.full(n, o["alpha"][1]), np.full(n, o["alpha"][2])])
+    av = np.concatenate([np.full(n_res, alpha[0]), np.full(n, alpha[1]), np.full(n, alpha[2])])
     e = np.abs(rstd[:, None] * av * dz)
-    Wp = np.abs(o["gain"][:, None] * o["W"])
+    Wp = np.abs(gain[:, None] * W)
     return 2.0 ** -8 * (e @ Wp.T).reshape(T, n, C)
+
+
+def dxhat_allowance(inp, dz, eps=1e-6):
+    o = oracle_inputs(inp)
+    return dxhat_allowance_f(o["x"], o["W"], o["alpha"], o["gain"], dz, eps)
 
 
 def compare_backward(G, ref, grad_rel=1e-3, fused=True):

@@ -1,0 +1,193 @@
+"""The five benchmark workloads at full size, in the launch configuration bench.py times (fused calls).
+
+Tokens are independent, so every per-token output (mappings, u, x_next, dy, dx, dH_*) of a sample of
+tokens is compared element by element with the oracle run on just those tokens; properties that hold at
+any size (H_res non-negative with unit row / column sums, everything finite) are checked on all tokens;
+the parameter gradients, which sum over all tokens, are compared with the oracle run over the whole
+batch in chunks."""
+import dataclasses
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mhclite_oracle as O
+from paper_2601_05732_b200 import synth
+from paper_2601_05732_b200 import layer as L
+from paper_2601_05732_b200.binding import MhcLite
+from parity_utils import (DEV, GpuLayer, check_bf16, check_f32, dxhat_allowance, dxhat_allowance_f, host,
+                          oracle_inputs, rms)
+
+pytestmark = pytest.mark.gpu
+NS = 48   # sampled tokens
+
+
+def _subset(inp, idx):
+    sub = dict(inp)
+    for k in ("x", "y", "g", "du"):
+        sub[k] = inp[k][idx]
+    sub["T"] = len(idx)
+    return sub
+
+
+def _oracle_param_grads(inp, kind, chunk=4096):
+    acc = None
+    for a in range(0, inp["T"], chunk):
+        idx = np.arange(a, min(inp["T"], a + chunk))
+        o = oracle_inputs(_subset(inp, idx))
+        r = O.layer_bwd(o["x"], o["y"], o["W"], o["b"], o["alpha"], o["gain"], 1e-6, o["g"], o["du"], kind=kind)
+        part = {k: r[k] for k in ("dW", "db", "dalpha", "dgain")}
+        acc = part if acc is None else {k: acc[k] + part[k] for k in acc}
+    return acc
+
+
+def _run_and_check(wl, kind="lite", param_grads=True, T=None):
+    T = T or wl.T
+    inp = synth.make_layer_inputs(wl.n, wl.C, T, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std, kind=kind)
+    G = GpuLayer(inp, kind=kind)
+    G.forward(True)
+    if wl.backward:
+        G.backward(True)
+    B = G.B
+    # properties on all tokens
+    Hr = B.H_res
+    assert float(Hr.min()) >= 0.0
+    if kind == "lite":
+        assert float((Hr.sum(1) - 1).abs().max()) < 1e-6 and float((Hr.sum(2) - 1).abs().max()) < 1e-6
+    for t in (B.u, B.x_next, B.H_pre, B.H_post, B.p_saved, B.rstd) + ((B.dx, B.dy, B.dW, B.dgain) if wl.backward else ()):
+        assert bool(torch.isfinite(t.float()).all())
+    # sampled tokens, element by element
+    idx = np.sort(np.random.default_rng(wl.seed).choice(T, NS, replace=False))
+    sub = _subset(inp, idx)
+    o = oracle_inputs(sub)
+    fw = O.layer_fwd(o["x"], o["y"], o["W"], o["b"], o["alpha"], o["gain"], 1e-6, kind=kind)
+    ti = torch.from_numpy(idx).to(DEV)
+    pick = lambda t: host(t.index_select(0, ti))
+    check_f32("rstd", pick(B.rstd), fw["rstd"])
+    check_f32("p_saved", pick(B.p_saved), fw["p"], 1e-4)
+    check_f32("H_res", pick(B.H_res), fw["H_res"])
+    check_f32("H_pre", pick(B.H_pre), fw["H_pre"])
+    check_f32("H_post", pick(B.H_post), fw["H_post"])
+    if kind == "lite":
+        check_f32("a_saved", pick(B.a_saved), fw["a"])
+    check_bf16("u", pick(B.u), fw["u"])
+    check_bf16("x_next", pick(B.x_next), fw["x_next"])
+    if not wl.backward:
+        return G
+    bw = O.layer_bwd(o["x"], o["y"], o["W"], o["b"], o["alpha"], o["gain"], 1e-6, o["g"], o["du"], kind=kind)
+    check_bf16("dy", pick(B.dy), bw["dy"])
+    check_f32("dH_res", pick(B.dH_res), bw["dH_res"], 2e-5)
+    check_f32("dH_post", pick(B.dH_post), bw["dH_post"], 2e-5)
+    check_bf16("dx", pick(B.dx), bw["dx"], extra=dxhat_allowance(sub, bw["dz"]))
+    if param_grads:
+        ref = _oracle_param_grads(inp, kind)
+        check_f32("dW", host(B.dW), ref["dW"], 1e-3)
+        check_f32("db", host(B.db), ref["db"], 1e-3)
+        check_f32("dalpha", host(B.dalpha), ref["dalpha"], 1e-3)
+        check_f32("dgain", host(B.dgain), ref["dgain"], 1e-3)
+    return G
+
+
+def test_cfg1_forward():
+    _run_and_check(synth.WORKLOADS["cfg1"])
+
+
+def test_cfg2_forward_backward():
+    _run_and_check(synth.WORKLOADS["cfg2"])
+
+
+def test_cfg4a_n3():
+    _run_and_check(synth.WORKLOADS["cfg4a"])
+
+
+def test_cfg4b_n5():
+    _run_and_check(synth.WORKLOADS["cfg4b"], param_grads=False)
+    # the parameter gradients of n = 5 on a quarter of the tokens (the oracle's n*C x 130 products are slow)
+    _run_and_check(synth.WORKLOADS["cfg4b"], T=8192)
+
+
+@pytest.mark.parametrize("T", [4096, 32768])
+def test_cfg5_lite_and_sk(T):
+    wl = synth.WORKLOADS["cfg5"]
+    GL = _run_and_check(wl, "lite", param_grads=(T == 4096), T=T)
+    GS = _run_and_check(wl, "sk", param_grads=(T == 4096), T=T)
+    # doubly-stochastic gap: none for mHC-lite; the SK path's gap matches the oracle's on the sampled tokens
+    l1 = torch.empty(T, device=DEV); l2 = torch.empty(T, device=DEV)
+    GL.ctx.ds_gap(GL.B.H_res, l1, None); GS.ctx.ds_gap(GS.B.H_res, l2, None)
+    torch.cuda.synchronize()
+    assert float(l1.max()) < 4e-6
+    assert float(l2.max()) < 1e-4          # near-uniform logits: SK converges; the stress case is in test_gpu_parity
+
+
+def test_cfg3_stack_of_24_layers():
+    wl = synth.WORKLOADS["cfg3"]
+    n, C, T, Ld, eps = wl.n, wl.C, wl.T, wl.layers, 1e-6
+    ctx = MhcLite(n, C, 0)
+    x0 = synth.normal_bf16(wl.seed, 0, (T, n, C))
+    gtop = synth.normal_bf16(wl.seed, 2, (T, n, C))
+    params = [synth.make_layer_params(n, C, wl.seed, layer=l, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std)
+              for l in range(Ld)]
+    P = [L.LayerParams(p["W"], p["b"], p["alpha"], p["gain"], DEV) for p in params]
+    Bs = [L.LayerBuffers(ctx, T) for _ in range(Ld)]
+
+    def standin(u):                                  # the harness's stand-in sublayer y = u / rms(u)
+        uf = u.float()
+        return (uf * torch.rsqrt(uf.pow(2).mean(-1, keepdim=True) + eps)).to(torch.bfloat16)
+
+    def standin_bwd(u, dy):
+        uf, d = u.float(), dy.float()
+        r = torch.rsqrt(uf.pow(2).mean(-1, keepdim=True) + eps)
+        return (r * d - uf * r.pow(3) * (uf * d).sum(-1, keepdim=True) / C).to(torch.bfloat16)
+
+    xs, ys = [L.to_device_bf16(x0, DEV)], []
+    for l in range(Ld):
+        L.pre_fwd(ctx, P[l], Bs[l], xs[l], eps, True)
+        ys.append(standin(Bs[l].u))
+        L.post_fwd(ctx, Bs[l], xs[l], ys[l])
+        xs.append(Bs[l].x_next)
+    gs, dus = {Ld: L.to_device_bf16(gtop, DEV)}, {}
+    for l in reversed(range(Ld)):
+        L.post_bwd(ctx, Bs[l], xs[l], ys[l], gs[l + 1], True)
+        dus[l] = standin_bwd(Bs[l].u, Bs[l].dy)
+        L.tail_bwd(ctx, P[l], Bs[l], xs[l], gs[l + 1], dus[l], eps, True)
+        gs[l] = Bs[l].dx
+    torch.cuda.synchronize()
+
+    # cumulative product of H_res over depth stays doubly stochastic, for every token
+    prod = Bs[0].H_res.clone()
+    for l in range(1, Ld):
+        prod = torch.bmm(Bs[l].H_res, prod)
+    assert float(prod.min()) >= 0.0
+    assert float((prod.sum(1) - 1).abs().max()) < Ld * 2e-6 and float((prod.sum(2) - 1).abs().max()) < Ld * 2e-6
+    for l in range(Ld):
+        assert float((Bs[l].H_res.sum(1) - 1).abs().max()) < 1e-6 and float((Bs[l].H_res.sum(2) - 1).abs().max()) < 1e-6
+
+    # every layer against the oracle, fed the tensors the GPU layer was fed (sampled tokens)
+    idx = np.sort(np.random.default_rng(wl.seed).choice(T, 32, replace=False))
+    ti = torch.from_numpy(idx).to(DEV)
+    pick = lambda t: host(t.index_select(0, ti))
+    oracle_H = []
+    for l in range(Ld):
+        p = {k: params[l][k].astype(np.float64) for k in ("W", "b", "alpha", "gain")}
+        xl, yl, gl, dul = pick(xs[l]), pick(ys[l]), pick(gs[l + 1]), pick(dus[l])
+        fw = O.layer_fwd(xl, yl, p["W"], p["b"], p["alpha"], p["gain"], eps)
+        oracle_H.append(fw["H_res"])
+        check_f32(f"H_res[{l}]", pick(Bs[l].H_res), fw["H_res"])
+        check_bf16(f"u[{l}]", pick(Bs[l].u), fw["u"])
+        check_bf16(f"x_next[{l}]", pick(Bs[l].x_next), fw["x_next"])
+        bw = O.layer_bwd(xl, yl, p["W"], p["b"], p["alpha"], p["gain"], eps, gl, dul)
+        check_bf16(f"dy[{l}]", pick(Bs[l].dy), bw["dy"])
+        check_bf16(f"dx[{l}]", pick(Bs[l].dx), bw["dx"],
+                   extra=dxhat_allowance_f(xl, p["W"], p["alpha"], p["gain"], bw["dz"], eps))
+    ref_prod = O.depth_product(oracle_H)
+    assert np.abs(pick(prod) - ref_prod).max() < 1e-5
+    # end to end: the oracle's own stack (bf16 storage between layers) on the sampled tokens
+    st = O.stack_fwd_bwd(pick(xs[0]), [(params[l]["W"].astype(np.float64), params[l]["b"].astype(np.float64),
+                                        params[l]["alpha"].astype(np.float64), params[l]["gain"].astype(np.float64))
+                                       for l in range(Ld)], pick(gs[Ld]), eps, bf16_storage=True)
+    # (single bf16 rounding flips compound over 24 layers, hence rms-level bounds here)
+    xe, xr = pick(xs[Ld]), st["xs"][Ld]
+    assert rms(xe - xr) <= 0.01 * rms(xr) and np.abs(xe - xr).max() <= 0.1 * np.abs(xr).max()
+    de, dr = pick(gs[0]), st["dx0"]
+    assert rms(de - dr) <= 0.02 * rms(dr)

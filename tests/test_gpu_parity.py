@@ -157,11 +157,12 @@ def test_bad_arguments_are_rejected_without_launch():
 
 # ------------------------------------------------------------------ SK comparison path (Eq. (2))
 @pytest.mark.parametrize("n,C,T", [(4, 256, 300), (3, 72, 100), (2, 64, 50), (5, 40, 70)])
-def test_sk_path_parity(n, C, T):
+@pytest.mark.parametrize("fused", [True, False])
+def test_sk_path_parity(n, C, T, fused):
     inp = synth.make_layer_inputs(n, C, T, seed=40 + n, bias_std=0.5, alpha=[1.0, 1.0, 1.0], w_std=0.05, kind="sk")
     G = GpuLayer(inp, kind="sk")
-    G.forward(); compare_forward(G, oracle_fwd(inp, kind="sk"), coeff_rel=1e-4)
-    G.backward(); compare_backward(G, oracle_bwd(inp, kind="sk"), grad_rel=2e-3, fused=False)
+    G.forward(fused); compare_forward(G, oracle_fwd(inp, kind="sk"), coeff_rel=1e-4)
+    G.backward(fused); compare_backward(G, oracle_bwd(inp, kind="sk"), grad_rel=2e-3, fused=fused)
 
 
 def test_sk_gap_vs_lite_on_ill_conditioned_logits():
