@@ -40,6 +40,35 @@ def algorithmic_bytes_per_token(n: int, C: int) -> dict:
     }
 
 
+def kernel_bytes_per_token(n: int, C: int) -> dict:
+    """Algorithmic bf16 bytes per token of each main kernel of the fused call sequence."""
+    return {
+        "proj_fwd": 2 * n * C,               # read x_l
+        "act_premix": (2 * n + 2) * C,       # read x_l, write u
+        "postres_fwd": (4 * n + 2) * C,      # read x_l, y; write x_next
+        "postres_bwd": (4 * n + 4) * C,      # read g, x_l, y; write dy
+        "tail_pre": (2 * n + 2) * C,         # read x_l, du
+        "tail_mma": (6 * n + 2) * C,         # read du, x_l, g; write dx
+    }
+
+
+def ncu_traffic(kernel: str, workload: str, T: int):
+    """DRAM bytes per launch of `kernel` from the committed ncu capture of this workload, or None when
+    there is none or the kernel's source has changed since (profiles/dram_traffic_<workload>.txt:
+    lines `kernel  tokens  dram_bytes  source_file  sha256_of_source`)."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", f"dram_traffic_{workload}.txt")
+    if not os.path.exists(path):
+        return None
+    for line in open(path):
+        f = line.split()
+        if len(f) == 5 and f[0] == kernel:
+            src = os.path.join(ROOT, "paper_2601_05732_b200", "csrc", f[3])
+            if os.path.exists(src) and hashlib.sha256(open(src, "rb").read()).hexdigest() == f[4]:
+                return float(f[2]) * T / float(f[1])
+    return None
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -210,19 +239,29 @@ def run_ours(args, wl, rank, world):
     clocks = sampler.stop() if sampler else None
     ms = D.max_over_ranks(ms, world, dev)
 
-    # ---- per-stage device time (same launch configuration), for the roofline of the dominant stage
-    stages = [("pre_fwd", lambda: L.pre_fwd(ctx, P, B, x, eps, fused)), ("post_fwd", lambda: L.post_fwd(ctx, B, x, y))]
-    if wl.backward:
-        stages += [("post_bwd", lambda: L.post_bwd(ctx, B, x, y, g, fused)),
-                   ("tail_bwd", lambda: L.tail_bwd(ctx, P, B, x, g, du, eps, fused))]
-    ev = {k: [] for k, _ in stages}
+    # ---- per-kernel device time (same launch configuration): CUDA events recorded by the library
+    #      around each of its main kernels, on the launching stream
+    ctx.set_kernel_timing(True)
+    ksum = {k: 0.0 for k in ctx.KERNELS}
+    stage_ev = []
     for _ in range(args.steps):
-        for k, fn in stages:
-            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(); fn(); b_.record()
-            ev[k].append((a, b_))
-    torch.cuda.synchronize()
-    stage_ms = {k: sum(a.elapsed_time(b_) for a, b_ in v) / len(v) for k, v in ev.items()}
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        evs[0].record(); L.pre_fwd(ctx, P, B, x, eps, fused)
+        evs[1].record(); L.post_fwd(ctx, B, x, y)
+        evs[2].record()
+        if wl.backward:
+            L.post_bwd(ctx, B, x, y, g, fused)
+            evs[3].record(); L.tail_bwd(ctx, P, B, x, g, du, eps, fused)
+            evs[4].record()
+        torch.cuda.synchronize()
+        stage_ev.append(evs)
+        for i, k in enumerate(ctx.KERNELS):
+            if fused and (wl.backward or i < 3):
+                ksum[k] += ctx.kernel_time_ms(i)
+    ctx.set_kernel_timing(False)
+    kernel_ms = {k: v / args.steps for k, v in ksum.items() if v > 0}
+    names = ["pre_fwd", "post_fwd", "post_bwd", "tail_bwd"][: 4 if wl.backward else 2]
+    stage_ms = {nm: sum(e[i].elapsed_time(e[i + 1]) for e in stage_ev) / len(stage_ev) for i, nm in enumerate(names)}
 
     # ---- end to end through the C ABI with host buffers ----------------------------------------
     e2e = None
@@ -283,13 +322,21 @@ def run_ours(args, wl, rank, world):
     if rank == 0:
         peak, peak_kind = load_peaks()
         bpt = algorithmic_bytes_per_token(n, C)
-        dom = max(stage_ms, key=stage_ms.get)
-        achieved = bpt[dom] * T / (stage_ms[dom] * 1e-3) / 1e9
         total_bytes = sum(bpt[k] for k in stage_ms) * T
+        kb = kernel_bytes_per_token(n, C)
+        if kernel_ms:
+            dom = max(kernel_ms, key=kernel_ms.get)
+            achieved = kb[dom] * T / (kernel_ms[dom] * 1e-3) / 1e9
+        else:                                   # un-fused sequence: report the slowest call
+            dom = max(stage_ms, key=stage_ms.get)
+            achieved = bpt[dom] * T / (stage_ms[dom] * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
-                    "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                    "unit": "GB/s", "frac": achieved / peak, "traffic": ncu_traffic(dom, wl.name, T),
                     "whole_step_gbs": total_bytes / (ms / args.steps * 1e-3) / 1e9,
                     "whole_step_frac_of_8TBs": total_bytes / (ms / args.steps * 1e-3) / 8e12,
+                    "whole_step_frac_of_measured": total_bytes / (ms / args.steps * 1e-3) / 1e9 / peak,
+                    "kernel_ms": kernel_ms,
+                    "kernel_gbs": {k: kb[k] * T / (v * 1e-3) / 1e9 for k, v in kernel_ms.items()},
                     "stage_ms": stage_ms,
                     "stage_gbs": {k: bpt[k] * T / (v * 1e-3) / 1e9 for k, v in stage_ms.items()}}
         line = {

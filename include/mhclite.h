@@ -245,6 +245,22 @@ MHCLITE_API int mhclite_step_host(mhclite_ctx* ctx, int64_t T,
                       float* dW, float* db, float* dalpha, float* dgain, int accumulate_params,
                       void* staging, size_t staging_bytes, void* stream);
 
+/* Per-kernel device time, for roofline accounting.  With timing on, the library records a pair of CUDA
+ * events on the call's stream around each launch of the kernels below (a few microseconds of overhead
+ * per launch: switch it off for throughput runs).  mhclite_kernel_time_ms returns the duration of the
+ * most recent launch of that kernel; the caller must have synchronised the stream since. */
+typedef enum mhclite_kernel {
+    MHCLITE_KERNEL_PROJ_FWD = 0,     /* tensor-core projection + sum of squares        reads x            */
+    MHCLITE_KERNEL_ACT_PREMIX = 1,   /* mappings + pre-mix                              reads x, writes u  */
+    MHCLITE_KERNEL_POSTRES_FWD = 2,  /* merge                                           reads x, y; writes x_next */
+    MHCLITE_KERNEL_POSTRES_BWD = 3,  /* merge backward                                  reads g, x, y; writes dy  */
+    MHCLITE_KERNEL_TAIL_PRE = 4,     /* dH_pre + activation backward                    reads x, du        */
+    MHCLITE_KERNEL_TAIL_MMA = 5,     /* projection backward + dx + dW                   reads x, g, du; writes dx */
+    MHCLITE_KERNEL_COUNT = 6
+} mhclite_kernel;
+MHCLITE_API int mhclite_set_kernel_timing(mhclite_ctx* ctx, int on);
+MHCLITE_API int mhclite_kernel_time_ms(mhclite_ctx* ctx, int kernel, float* ms);
+
 /* Number of kernels this context has launched since it was created (for accounting; host counter). */
 MHCLITE_API int64_t mhclite_kernel_launches(const mhclite_ctx* ctx);
 

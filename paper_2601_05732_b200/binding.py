@@ -60,6 +60,8 @@ SIGNATURES = {
     "mhclite_step_host": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p, _i,
                                _p, _sz, _p]),
     "mhclite_kernel_launches": (_i64, [_p]),
+    "mhclite_set_kernel_timing": (_i, [_p, _i]),
+    "mhclite_kernel_time_ms": (_i, [_p, _i, C.POINTER(_f)]),
 }
 
 
@@ -265,6 +267,16 @@ class MhcLite:
             self._ptr(H_pre, f), self._ptr(H_post, f), self._ptr(g, h), self._ptr(du, h), self._ptr(dH_res, f),
             self._ptr(dH_post, f), self._ptr(dx, h), self._ptr(dW, f), self._ptr(db, f), self._ptr(dalpha, f),
             self._ptr(dgain, f), int(accumulate_params), self._stream()), "mhc_sk20_tail_bwd_fused")
+
+    KERNELS = ("proj_fwd", "act_premix", "postres_fwd", "postres_bwd", "tail_pre", "tail_mma")
+
+    def set_kernel_timing(self, on: bool):
+        self._check(self.lib.mhclite_set_kernel_timing(self._h, int(on)), "mhclite_set_kernel_timing")
+
+    def kernel_time_ms(self, kernel: int) -> float:
+        ms = _f()
+        self._check(self.lib.mhclite_kernel_time_ms(self._h, kernel, C.byref(ms)), "mhclite_kernel_time_ms")
+        return float(ms.value)
 
     def kernel_launches(self) -> int:
         return int(self.lib.mhclite_kernel_launches(self._h))

@@ -932,6 +932,7 @@ void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp,
                             float eps, const float* b, const float* alpha, float* H_res, float* H_pre, float* H_post,
                             float* a_saved, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s) {
     c->launches += 1;
+    KernelTimer timer_(c, MHCLITE_KERNEL_ACT_PREMIX, s);
     const int C8 = c->C / 8;
     const float inv = 1.f / (float)(c->n * c->C);
 #define MHCL_AP_T(N_) lite_act_premix_t_k<N_><<<group_grid(T, kTokGroup, c->sm_count), kActThreads, 0, s>>>( \
@@ -954,6 +955,7 @@ void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const v
                          const float* dH_res, const float* dH_post, float* e, int Npad, void* ehi, void* elo, int Kp,
                          float* kappa, float* db, float* dalpha, cudaStream_t s) {
     c->launches += 1;
+    KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_PRE, s);
     const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
     const int C8 = c->C / 8;
     const float inv = 1.f / (float)(c->n * c->C);

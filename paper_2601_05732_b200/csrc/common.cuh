@@ -24,6 +24,8 @@ struct mhclite_ctx {
     void* ws;
     size_t ws_bytes;
     mutable int64_t launches;     // kernels launched through this context
+    bool timing;                  // record CUDA events around the main kernels (mhclite_set_kernel_timing)
+    cudaEvent_t ev[MHCLITE_KERNEL_COUNT][2];
     char err[256];
 };
 
@@ -36,6 +38,15 @@ inline int64_t round_up64(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 // Number of projection columns. kind 0: n!+2n (mHC-lite); kind 1: n*n+2n (SK path).
 inline int n_res_cols(int n, int kind) { return kind == 0 ? ipow_fact(n) : n * n; }
 inline int n_cols(int n, int kind) { return n_res_cols(n, kind) + 2 * n; }
+
+// Brackets one kernel launch with the context's events when kernel timing is switched on.
+struct KernelTimer {
+    const mhclite_ctx* c; int id; cudaStream_t s;
+    KernelTimer(const mhclite_ctx* c_, int id_, cudaStream_t s_) : c(c_), id(id_), s(s_) {
+        if (c->timing) cudaEventRecord(c->ev[id][0], s);
+    }
+    ~KernelTimer() { if (c->timing) cudaEventRecord(c->ev[id][1], s); }
+};
 
 int fail(mhclite_ctx* ctx, int status, const char* fmt, ...);
 int check_cuda(mhclite_ctx* ctx, cudaError_t e, const char* what);

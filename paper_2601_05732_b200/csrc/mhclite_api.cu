@@ -138,7 +138,8 @@ int mhclite_create(mhclite_ctx** out, int n, int C, int device) {
     mhclite_ctx* ctx = new (std::nothrow) mhclite_ctx();
     if (!ctx) return MHCLITE_ERR_CUDA;
     ctx->n = n; ctx->C = C; ctx->device = device; ctx->nfact = ipow_fact(n);
-    ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->err[0] = 0; ctx->launches = 0;
+    ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->err[0] = 0; ctx->launches = 0; ctx->timing = false;
+    for (int k = 0; k < MHCLITE_KERNEL_COUNT; ++k) ctx->ev[k][0] = ctx->ev[k][1] = nullptr;
     {
         DeviceGuard g(device);
         cudaError_t e = g.err;
@@ -152,6 +153,9 @@ int mhclite_create(mhclite_ctx** out, int n, int C, int device) {
 
 int mhclite_destroy(mhclite_ctx* ctx) {
     if (!ctx) return MHCLITE_ERR_BAD_ARG;
+    for (int k = 0; k < MHCLITE_KERNEL_COUNT; ++k)
+        for (int e = 0; e < 2; ++e)
+            if (ctx->ev[k][e]) cudaEventDestroy(ctx->ev[k][e]);
     delete ctx;
     return MHCLITE_OK;
 }
@@ -514,5 +518,27 @@ int mhclite_step_host(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x_host, c
 }
 
 int64_t mhclite_kernel_launches(const mhclite_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int mhclite_set_kernel_timing(mhclite_ctx* ctx, int on) {
+    MHCL_REQUIRE_CTX(ctx);
+    MHCL_DEVICE(ctx);
+    if (on) {
+        for (int k = 0; k < MHCLITE_KERNEL_COUNT; ++k)
+            for (int e = 0; e < 2; ++e)
+                if (!ctx->ev[k][e]) {
+                    int rc = check_cuda(ctx, cudaEventCreate(&ctx->ev[k][e]), "cudaEventCreate");
+                    if (rc) return rc;
+                }
+    }
+    ctx->timing = on != 0;
+    return MHCLITE_OK;
+}
+
+int mhclite_kernel_time_ms(mhclite_ctx* ctx, int kernel, float* ms) {
+    MHCL_REQUIRE_CTX(ctx);
+    if (kernel < 0 || kernel >= MHCLITE_KERNEL_COUNT || !ms) return fail(ctx, MHCLITE_ERR_BAD_ARG, "bad kernel id");
+    if (!ctx->ev[kernel][0]) return fail(ctx, MHCLITE_ERR_BAD_ARG, "kernel timing was never switched on");
+    return check_cuda(ctx, cudaEventElapsedTime(ms, ctx->ev[kernel][0], ctx->ev[kernel][1]), "cudaEventElapsedTime");
+}
 
 }  // extern "C"

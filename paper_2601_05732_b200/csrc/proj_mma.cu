@@ -234,6 +234,7 @@ static void launch_fwd_t(int64_t T, int nC, const ProjPlan& p, const void* x, co
 void launch_proj_fwd_mma(const mhclite_ctx* c, int64_t T, const ProjPlan& p, const void* x, const void* Wp,
                          float* qpart, float* ssq, cudaStream_t s) {
     c->launches += 1;
+    KernelTimer timer_(c, MHCLITE_KERNEL_PROJ_FWD, s);
     const int nC = c->n * c->C;
     switch (p.NT) {
         case 1: launch_fwd_t<1, 1>(T, nC, p, x, Wp, qpart, ssq, s); break;

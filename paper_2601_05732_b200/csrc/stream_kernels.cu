@@ -304,6 +304,7 @@ void launch_premix_fwd(const mhclite_ctx* c, int64_t T, const void* x, const flo
 void launch_postres_fwd(const mhclite_ctx* c, int64_t T, const void* x, const void* y, const float* H_res,
                         const float* H_post, void* x_next, cudaStream_t s) {
     c->launches += 1;
+    KernelTimer timer_(c, MHCLITE_KERNEL_POSTRES_FWD, s);
     const int C8 = c->C / 8;
     const int grid = grid_for(T * C8, c->sm_count, 8);
     MHCL_DISPATCH_N(c->n, postres_fwd_k<N_><<<grid, kThreads, 0, s>>>(T, C8, (const uint4*)x, (const uint4*)y, H_res,
@@ -314,6 +315,7 @@ void launch_postres_bwd(const mhclite_ctx* c, int64_t T, const void* x, const vo
                         const float* H_post, const void* g, void* dy, float* dH_res, float* dH_post, void* dx,
                         int acc, cudaStream_t s) {
     c->launches += 1;
+    KernelTimer timer_(c, MHCLITE_KERNEL_POSTRES_BWD, s);
     const int C8 = c->C / 8;
     const int grid = grid_for(T * 32, c->sm_count, 8);
 #define MHCL_PB(W, A) postres_bwd_k<N_, W, A><<<grid, kThreads, 0, s>>>(T, C8, (const uint4*)x, (const uint4*)y, \

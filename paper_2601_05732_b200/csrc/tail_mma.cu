@@ -381,7 +381,10 @@ void launch_tail_mma(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, 
         case 2: launch_tail_t<N_, 2>(p, a, fused, acc_dx != 0, s); break;         \
         default: launch_tail_t<N_, 3>(p, a, fused, acc_dx != 0, s); break;        \
     }
-    MHCL_DISPATCH_N(c->n, MHCL_TAIL_KS(N_));
+    {
+        KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_MMA, s);
+        MHCL_DISPATCH_N(c->n, MHCL_TAIL_KS(N_));
+    }
 #undef MHCL_TAIL_KS
     const int nC = c->n * c->C;
     const int fg = (nC + 7) / 8;
