@@ -440,6 +440,29 @@ struct LiteDims {
     static constexpr int kIn = kFact + kN + kNN + 3 * N_ + 1; // a | p | dH_res | H_pre | H_post | dH_post | rstd
 };
 
+// The lexicographic permutation table as a compile-time constant: with the loops below fully unrolled
+// every index into it is a constant, so the Birkhoff sum and its gradient become plain register adds.
+template <int N_>
+struct PermConst { unsigned char s[LiteDims<N_>::kFact][N_]; };
+
+template <int N_>
+__host__ __device__ constexpr PermConst<N_> make_perm_const() {
+    PermConst<N_> t{};
+    int cur[N_] = {};
+    for (int i = 0; i < N_; ++i) cur[i] = i;
+    for (int k = 0; k < LiteDims<N_>::kFact; ++k) {
+        for (int i = 0; i < N_; ++i) t.s[k][i] = (unsigned char)cur[i];
+        int a = N_ - 2;                              // successor in lexicographic order
+        while (a >= 0 && cur[a] > cur[a + 1]) --a;
+        if (a < 0) break;
+        int b = N_ - 1;
+        while (cur[b] < cur[a]) --b;
+        int tmp = cur[a]; cur[a] = cur[b]; cur[b] = tmp;
+        for (int lo = a + 1, hi = N_ - 1; lo < hi; ++lo, --hi) { tmp = cur[lo]; cur[lo] = cur[hi]; cur[hi] = tmp; }
+    }
+    return t;
+}
+
 template <int N_>
 __device__ __forceinline__ void lite_thread_fwd(const float* prow, float* orow, const float* b_s, float a_res,
                                                 float a_pre, float a_post, const uint8_t* klist_s) {
@@ -450,15 +473,20 @@ __device__ __forceinline__ void lite_thread_fwd(const float* prow, float* orow, 
     float sum = 0.f;
 #pragma unroll
     for (int k = 0; k < D::kFact; ++k) { z[k] = expf(z[k] - m); sum += z[k]; }
+    constexpr PermConst<N_> tab = make_perm_const<N_>();
+    (void)klist_s;
+    float h[D::kNN];
 #pragma unroll
-    for (int k = 0; k < D::kFact; ++k) orow[k] = z[k] / sum;
+    for (int e = 0; e < D::kNN; ++e) h[e] = 0.f;
 #pragma unroll
-    for (int e = 0; e < D::kNN; ++e) {
-        float h = 0.f;
+    for (int k = 0; k < D::kFact; ++k) {
+        const float a = z[k] / sum;
+        orow[k] = a;
 #pragma unroll
-        for (int r = 0; r < D::kPer; ++r) h += orow[klist_s[e * D::kPer + r]];
-        orow[D::kFact + e] = h;
+        for (int i = 0; i < N_; ++i) h[i * N_ + tab.s[k][i]] += a;          // Eq. (5): P_k[i][sigma_k(i)] = 1
     }
+#pragma unroll
+    for (int e = 0; e < D::kNN; ++e) orow[D::kFact + e] = h[e];
 #pragma unroll
     for (int j = 0; j < N_; ++j) {
         orow[D::kFact + D::kNN + j] = sigmoidf_(fmaf(a_pre, prow[D::kFact + j], b_s[D::kFact + j]));
@@ -573,20 +601,23 @@ __device__ __forceinline__ void lite_thread_bwd(const float* in, const float* dh
     const float* hpost = hpre + N_;
     const float* dhpost = hpost + N_;
     const float rs = dhpost[N_];
-    float dot = 0.f;
+    constexpr PermConst<N_> tab = make_perm_const<N_>();
+    (void)sigma_s;
+    float dhr[D::kNN], da[D::kFact], dot = 0.f;
+#pragma unroll
+    for (int e = 0; e < D::kNN; ++e) dhr[e] = dh[e];
 #pragma unroll
     for (int k = 0; k < D::kFact; ++k) {
         float d = 0.f;
 #pragma unroll
-        for (int i = 0; i < N_; ++i) d += dh[i * N_ + sigma_s[k * N_ + i]];       // Eq. (5): dL/da_k
+        for (int i = 0; i < N_; ++i) d += dhr[i * N_ + tab.s[k][i]];                // Eq. (5): dL/da_k
+        da[k] = d;
         dot = fmaf(a[k], d, dot);
     }
     float kap = 0.f;
 #pragma unroll
     for (int k = 0; k < D::kFact; ++k) {
-        float d = 0.f;
-#pragma unroll
-        for (int i = 0; i < N_; ++i) d += dh[i * N_ + sigma_s[k * N_ + i]];
+        const float d = da[k];
         const float dz = a[k] * (d - dot), ed = a_res * dz, pv = pt[k];
         orow[k] = rs * ed;
         orow[D::kN + 1 + k] = dz;
@@ -606,33 +637,34 @@ __device__ __forceinline__ void lite_thread_bwd(const float* in, const float* dh
     orow[D::kN] = rs * rs * kap * inv_nC;
 }
 
-template <int N_>
-__global__ void __launch_bounds__(kActThreads, 3) lite_tailpre_t_k(
+template <int N_, bool STREAM, int THREADS, int GROUP>
+__global__ void __launch_bounds__(THREADS) lite_tailpre_t_k(
     int64_t T, int C8, float inv_nC, const uint4* __restrict__ x, const uint4* __restrict__ du,
+    const float* __restrict__ dH_pre_in,
     const float* __restrict__ a_saved, const float* __restrict__ p, const float* __restrict__ rstd,
     const float* __restrict__ alpha, const float* __restrict__ H_pre, const float* __restrict__ H_post,
     const float* __restrict__ dH_res, const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa,
     float* db, float* dalpha) {
     using D = LiteDims<N_>;
     __shared__ uint8_t sigma_s[D::kFact * N_];
-    __shared__ float in_s[kTokGroup][D::kIn + 1];
-    __shared__ float dhp_s[kTokGroup][N_];
-    __shared__ float og[kTokGroup][2 * D::kN + 3];
+    __shared__ float in_s[GROUP][D::kIn + 1];
+    __shared__ float dhp_s[GROUP][N_];
+    __shared__ float og[GROUP][2 * D::kN + 3];
     __shared__ float dal_s[3];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    for (int i = tid; i < D::kFact * N_; i += kActThreads) sigma_s[i] = c_perm[N_].sigma[i];
+    for (int i = tid; i < D::kFact * N_; i += THREADS) sigma_s[i] = c_perm[N_].sigma[i];
     if (tid < 3) dal_s[tid] = 0.f;
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
     float db_col = 0.f, dal_col = 0.f;             // thread c < kN: column c of db, and sum_t dz[t,c] p[t,c]
     constexpr int o_p = D::kFact, o_dhres = o_p + D::kN, o_hpre = o_dhres + D::kNN, o_hpost = o_hpre + N_,
                   o_dhpost = o_hpost + N_, o_rstd = o_dhpost + N_;
     __syncthreads();
-    const int64_t ngroups = (T + kTokGroup - 1) / kTokGroup;
+    const int64_t ngroups = (T + GROUP - 1) / GROUP;
     for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
-        const int64_t t0 = grp * kTokGroup;
-        const int nt = (T - t0 < kTokGroup) ? (int)(T - t0) : kTokGroup;
+        const int64_t t0 = grp * GROUP;
+        const int nt = (T - t0 < GROUP) ? (int)(T - t0) : GROUP;
         // L: stage the per-token inputs with cp.async (they arrive while D streams)
-        for (int i = tid; i < nt * D::kIn; i += kActThreads) {
+        for (int i = tid; i < nt * D::kIn; i += THREADS) {
             const int tl = i / D::kIn, c = i - tl * D::kIn;
             const int64_t t = t0 + tl;
             const float* src;
@@ -646,8 +678,11 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_tailpre_t_k(
             asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&in_s[tl][c])), "l"(src) : "memory");
         }
         cp_async_commit();
-        // D: dH_pre[j] = <du, x_j>, one warp per token
-        for (int tl = w; tl < nt; tl += kActWarps) {
+        // D: dH_pre[j] = <du, x_j>, one warp per token (or taken from a preceding premix_bwd call)
+        if (!STREAM) {
+            for (int i = tid; i < nt * N_; i += THREADS) dhp_s[i / N_][i % N_] = __ldg(dH_pre_in + t0 * N_ + i);
+        }
+        for (int tl = w; STREAM && tl < nt; tl += (THREADS / 32)) {
             const int64_t t = t0 + tl;
             float r[N_];
 #pragma unroll
@@ -697,7 +732,7 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_tailpre_t_k(
         }
         // W: e as a bf16 pair (and / or fp32), kappa
         const int cols = eo.ehi ? eo.Kp : eo.Npad;
-        for (int i = tid; i < nt * cols; i += kActThreads) {
+        for (int i = tid; i < nt * cols; i += THREADS) {
             const int tl = i / cols, c = i - tl * cols;
             const float v = (c < D::kN) ? og[tl][c] : 0.f;
             const int64_t t = t0 + tl;
@@ -952,15 +987,20 @@ void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp,
 
 void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const void* du, const float* a, const float* p,
                          const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
-                         const float* dH_res, const float* dH_post, float* e, int Npad, void* ehi, void* elo, int Kp,
-                         float* kappa, float* db, float* dalpha, cudaStream_t s) {
+                         const float* dH_res, const float* dH_post, float* dH_pre_ws, float* e, int Npad, void* ehi,
+                         void* elo, int Kp, float* kappa, float* db, float* dalpha, cudaStream_t s) {
     c->launches += 1;
     KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_PRE, s);
     const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
     const int C8 = c->C / 8;
     const float inv = 1.f / (float)(c->n * c->C);
-#define MHCL_TP_T(N_) lite_tailpre_t_k<N_><<<group_grid(T, kTokGroup, c->sm_count), kActThreads, 0, s>>>( \
-        T, C8, inv, (const uint4*)x, (const uint4*)du, a, p, rstd, alpha, H_pre, H_post, dH_res, dH_post, eo, kappa, db, dalpha)
+    // n <= 4: a streaming pass for dH_pre (premix_bwd without dx), then the thread-per-token activation backward;
+    // measured faster than one kernel doing both, whose per-token phase stalls the streaming warps
+#define MHCL_TP_T(N_) do { \
+        launch_premix_bwd(c, T, x, H_pre, du, dH_pre_ws, nullptr, 0, s); \
+        lite_tailpre_t_k<N_, false, 256, 64><<<group_grid(T, 64, c->sm_count), 256, 0, s>>>( \
+            T, C8, inv, (const uint4*)x, (const uint4*)du, dH_pre_ws, a, p, rstd, alpha, H_pre, H_post, dH_res, dH_post, \
+            eo, kappa, db, dalpha); } while (0)
     switch (c->n) {
         case 2: MHCL_TP_T(2); break;
         case 3: MHCL_TP_T(3); break;

@@ -343,7 +343,7 @@ int mhclite_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, c
     rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
     if (rc) return rc;
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
-    launch_lite_tailpre(ctx, T, x, du, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_post,
+    launch_lite_tailpre(ctx, T, x, du, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_post, w.dH_pre,
                         tp.supported ? nullptr : w.e, w.Npad, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db,
                         dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_tailpre");
