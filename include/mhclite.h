@@ -261,6 +261,11 @@ typedef enum mhclite_kernel {
 MHCLITE_API int mhclite_set_kernel_timing(mhclite_ctx* ctx, int on);
 MHCLITE_API int mhclite_kernel_time_ms(mhclite_ctx* ctx, int kernel, float* ms);
 
+/* Synchronous check of the device status word: kernels that wait on hardware barriers do so with a bound
+ * and, instead of hanging, record MHCLITE_ERR_TIMEOUT there and return.  Copies one int device->host
+ * (synchronises the device); returns MHCLITE_OK or the recorded status. */
+MHCLITE_API int mhclite_device_status(mhclite_ctx* ctx);
+
 /* Number of kernels this context has launched since it was created (for accounting; host counter). */
 MHCLITE_API int64_t mhclite_kernel_launches(const mhclite_ctx* ctx);
 

@@ -60,6 +60,7 @@ SIGNATURES = {
     "mhclite_step_host": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p, _i,
                                _p, _sz, _p]),
     "mhclite_kernel_launches": (_i64, [_p]),
+    "mhclite_device_status": (_i, [_p]),
     "mhclite_set_kernel_timing": (_i, [_p, _i]),
     "mhclite_kernel_time_ms": (_i, [_p, _i, C.POINTER(_f)]),
 }
@@ -277,6 +278,10 @@ class MhcLite:
         ms = _f()
         self._check(self.lib.mhclite_kernel_time_ms(self._h, kernel, C.byref(ms)), "mhclite_kernel_time_ms")
         return float(ms.value)
+
+    def device_status(self):
+        """Raises if a kernel recorded a timed-out wait (synchronises the device)."""
+        self._check(self.lib.mhclite_device_status(self._h), "mhclite_device_status")
 
     def kernel_launches(self) -> int:
         return int(self.lib.mhclite_kernel_launches(self._h))

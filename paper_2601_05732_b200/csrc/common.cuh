@@ -24,6 +24,7 @@ struct mhclite_ctx {
     void* ws;
     size_t ws_bytes;
     mutable int64_t launches;     // kernels launched through this context
+    int* status_word;             // device status word inside the attached workspace (null until first used)
     bool timing;                  // record CUDA events around the main kernels (mhclite_set_kernel_timing)
     cudaEvent_t ev[MHCLITE_KERNEL_COUNT][2];
     char err[256];
@@ -83,6 +84,8 @@ struct Workspace {
     float* ssq;      // [kMaxKSplit][T]          partial sums of squares
     void *ehi, *elo; // [T rounded up to 32][Kp] bf16 pair hi + lo = e
     float* Gpart;    // [splits][nC][Kp] partial G of each token range
+    void* Wt;        // [2 nq][Kpad] bf16: W' hi rows then lo rows, K-major (tcgen05 projection)
+    int* status;     // device status word (0, or a negative mhclite_status raised by a kernel)
     size_t bytes;
     int Npad;
 };

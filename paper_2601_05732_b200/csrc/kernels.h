@@ -32,6 +32,14 @@ void launch_proj_bwd_dw(const mhclite_ctx* c, int64_t T, int N, int Npad, const 
                         const float* gain, const float* e, float* G, float* dW, float* dgain, int acc,
                         cudaStream_t s);
 
+// proj_tc.cu : the same projection on tcgen05 / TMA / tensor memory (N <= 128 columns)
+bool proj_tc_supported(int n, int C, int N);
+int proj_tc_nq(int N);
+void launch_pack_wt(const mhclite_ctx* c, const ProjPlan& p, int N, const float* W, const float* gain, void* Wt,
+                    cudaStream_t s);
+bool launch_proj_fwd_tc(const mhclite_ctx* c, int64_t T, int N, const ProjPlan& p, const void* x, const void* Wt,
+                        float* qpart, float* ssq, int* status, cudaStream_t s);
+
 // act_kernels.cu : per-token activations, H_res assembly and their gradients
 void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, const float* qpart, const float* ssq,
                          float eps, const float* b, const float* alpha, float* H_res, float* H_pre, float* H_post,

@@ -43,6 +43,8 @@ Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base) {
     w.ehi = p + off;             off += align256(erows * tp.Kp * 2);
     w.elo = p + off;             off += align256(erows * tp.Kp * 2);
     w.Gpart = (float*)(p + off); off += align256(tp.supported ? (size_t)tp.splits * n * C * tp.Kp * sizeof(float) : 0);
+    w.Wt = p + off;              off += align256((size_t)2 * round_up(N, 8) * pp.nchunks * 64 * 2);
+    w.status = (int*)(p + off);  off += 256;
     w.bytes = off;
     return w;
 }
@@ -86,6 +88,32 @@ static int need_workspace(mhclite_ctx* ctx, int64_t T, int kind, Workspace* w) {
     if (!ctx->ws || ctx->ws_bytes < need)
         return fail(ctx, MHCLITE_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu attached", need, ctx->ws ? ctx->ws_bytes : (size_t)0);
     *w = plan_workspace(ctx->n, ctx->C, T, kind, ctx->ws);
+    // one status word per workspace, at its very end, cleared when first used
+    w->status = (int*)((char*)ctx->ws + ((ctx->ws_bytes - sizeof(int)) & ~(size_t)255));
+    if (ctx->status_word != w->status) {
+        DeviceGuard g(ctx->device);
+        if (cudaMemset(w->status, 0, sizeof(int)) != cudaSuccess) return fail(ctx, MHCLITE_ERR_CUDA, "clearing the status word");
+        ctx->status_word = w->status;
+    }
+    return MHCLITE_OK;
+}
+
+// RMSNorm statistics + projection partials of every entry point's forward: tcgen05 / TMA kernel when the
+// projection fits one UMMA tile (N <= 128 columns), the mma.sync kernel otherwise.
+static int proj_forward(mhclite_ctx* ctx, int64_t T, int N, const Workspace& w, const ProjPlan& pp, const mhclite_bf16* x,
+                        const float* W, const float* gain, cudaStream_t s) {
+    if (proj_tc_supported(ctx->n, ctx->C, N)) {
+        launch_pack_wt(ctx, pp, N, W, gain, w.Wt, s);
+        MHCL_LAUNCH_CHECK(ctx, "pack_wt");
+        if (launch_proj_fwd_tc(ctx, T, N, pp, x, w.Wt, w.qpart, w.ssq, w.status, s)) {
+            MHCL_LAUNCH_CHECK(ctx, "proj_fwd_tc");
+            return MHCLITE_OK;
+        }
+    }
+    launch_pack_w(ctx, pp, N, W, gain, w.Wp, s);
+    MHCL_LAUNCH_CHECK(ctx, "pack_w");
+    launch_proj_fwd_mma(ctx, T, pp, x, w.Wp, w.qpart, w.ssq, s);
+    MHCL_LAUNCH_CHECK(ctx, "proj_fwd_mma");
     return MHCLITE_OK;
 }
 
@@ -138,7 +166,7 @@ int mhclite_create(mhclite_ctx** out, int n, int C, int device) {
     mhclite_ctx* ctx = new (std::nothrow) mhclite_ctx();
     if (!ctx) return MHCLITE_ERR_CUDA;
     ctx->n = n; ctx->C = C; ctx->device = device; ctx->nfact = ipow_fact(n);
-    ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->err[0] = 0; ctx->launches = 0; ctx->timing = false;
+    ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->err[0] = 0; ctx->launches = 0; ctx->timing = false; ctx->status_word = nullptr;
     for (int k = 0; k < MHCLITE_KERNEL_COUNT; ++k) ctx->ev[k][0] = ctx->ev[k][1] = nullptr;
     {
         DeviceGuard g(device);
@@ -185,6 +213,7 @@ int mhclite_set_workspace(mhclite_ctx* ctx, void* workspace, size_t bytes) {
     if (workspace && ((uintptr_t)workspace & 255)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "workspace not 256-byte aligned");
     ctx->ws = workspace;
     ctx->ws_bytes = workspace ? bytes : 0;
+    ctx->status_word = nullptr;
     return MHCLITE_OK;
 }
 
@@ -205,10 +234,8 @@ int mhclite_coeffs_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     cudaStream_t s = (cudaStream_t)stream;
     const int N = n_cols(ctx->n, 0);
     const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
-    launch_pack_w(ctx, pp, N, W, gain, w.Wp, s);
-    MHCL_LAUNCH_CHECK(ctx, "pack_w");
-    launch_proj_fwd_mma(ctx, T, pp, x, w.Wp, w.qpart, w.ssq, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_fwd_mma");
+    rc = proj_forward(ctx, T, N, w, pp, x, W, gain, s);
+    if (rc) return rc;
     launch_lite_act_fwd(ctx, T, pp, w.qpart, w.ssq, eps, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_act_fwd");
     return MHCLITE_OK;
@@ -252,10 +279,8 @@ int mhclite_pre_fwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, co
     cudaStream_t s = (cudaStream_t)stream;
     const int N = n_cols(ctx->n, 0);
     const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
-    launch_pack_w(ctx, pp, N, W, gain, w.Wp, s);
-    MHCL_LAUNCH_CHECK(ctx, "pack_w");
-    launch_proj_fwd_mma(ctx, T, pp, x, w.Wp, w.qpart, w.ssq, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_fwd_mma");
+    rc = proj_forward(ctx, T, N, w, pp, x, W, gain, s);
+    if (rc) return rc;
     launch_lite_act_premix(ctx, T, pp, w.qpart, w.ssq, eps, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, x, u, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_act_premix");
     return MHCLITE_OK;
@@ -367,10 +392,8 @@ int mhc_sk20_coeffs_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
     cudaStream_t s = (cudaStream_t)stream;
     const int N = n_cols(ctx->n, 1);
     const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
-    launch_pack_w(ctx, pp, N, W_sk, gain, w.Wp, s);
-    MHCL_LAUNCH_CHECK(ctx, "pack_w");
-    launch_proj_fwd_mma(ctx, T, pp, x, w.Wp, w.qpart, w.ssq, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_fwd_mma");
+    rc = proj_forward(ctx, T, N, w, pp, x, W_sk, gain, s);
+    if (rc) return rc;
     launch_sk_act_fwd(ctx, T, iters, pp, w.qpart, w.ssq, eps, b_sk, alpha, H_res, H_pre, H_post, p_saved, rstd, s);
     MHCL_LAUNCH_CHECK(ctx, "sk_act_fwd");
     return MHCLITE_OK;
@@ -518,6 +541,17 @@ int mhclite_step_host(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x_host, c
 }
 
 int64_t mhclite_kernel_launches(const mhclite_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int mhclite_device_status(mhclite_ctx* ctx) {
+    MHCL_REQUIRE_CTX(ctx);
+    if (!ctx->status_word) return MHCLITE_OK;
+    MHCL_DEVICE(ctx);
+    int v = 0;
+    int rc = check_cuda(ctx, cudaMemcpy(&v, ctx->status_word, sizeof(int), cudaMemcpyDeviceToHost), "read status word");
+    if (rc) return rc;
+    if (v != 0) return fail(ctx, v, "a kernel gave up on a bounded wait (status %d)", v);
+    return MHCLITE_OK;
+}
 
 int mhclite_set_kernel_timing(mhclite_ctx* ctx, int on) {
     MHCL_REQUIRE_CTX(ctx);

@@ -1,0 +1,309 @@
+// Blackwell-native forward projection of paper Eq. (4): q = x W' (W' = diag(gain) W) and the RMSNorm sum of
+// squares, in one pass over x, on the 5th-generation tensor cores.
+//
+//   TMA (cp.async.bulk.tensor, 128-byte swizzle) streams x tiles [128 tokens x 64 k] and W' tiles
+//   [2 Nq x 64 k] into a shared-memory ring; one thread issues tcgen05.mma (M = 128 tokens, N = 2 Nq,
+//   K = 16 per instruction) with the fp32 accumulator [128 x 2 Nq] in tensor memory; the bf16 pair
+//   hi | lo of W' sits side by side in N, so x is read from shared memory once per k-step and the two
+//   partial products are added in the epilogue.  Four warps read the same x tiles from shared memory for
+//   the sum of squares, then fetch the accumulator with tcgen05.ld (thread = token) and store the K slice's
+//   partial result.  The tensor work is a small fraction of the time the bytes take to arrive: the
+//   kernel is bound by HBM.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (owns the tensor-memory
+// allocation), warps 2..5 = sum of squares + epilogue (TMEM lane quadrant = warp % 4).
+// Every wait on an mbarrier is bounded: when the bound is hit the CTA raises an abort flag, records a status
+// word in global memory, lets in-flight copies land, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "kernels.h"
+#include "mma.cuh"
+
+namespace mhcl {
+
+constexpr int kTcTok = 128;                 // tokens per CTA = UMMA M
+constexpr int kTcK = 64;                    // k per stage = one 128-byte swizzle row of bf16
+constexpr int kTcXBytes = kTcTok * kTcK * 2;
+constexpr uint32_t kWaitLimit = 1u << 22;   // bounded mbarrier polling
+
+// ---- PTX wrappers -----------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Waits for the phase with the given parity; gives up (and raises *abort) after kWaitLimit polls or when
+// another role has raised it.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort) return false;
+    }
+    *abort = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, bf16 x bf16 -> f32
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) with the 128-byte
+// swizzle: 8-row groups 1024 bytes apart; descriptor version 1 (Blackwell), layout type 2 (SWIZZLE_128B).
+__device__ __forceinline__ uint64_t smem_desc_k128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);          // start address
+    d |= (uint64_t)1 << 16;                          // leading byte offset (16 B units; fixed for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                          // descriptor version
+    d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor: D f32, A and B bf16, both K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t umma_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTcTok >> 4) << 24);
+}
+
+struct TcSmem {                       // control block placed after the stage ring
+    uint64_t full[8], empty[8], accum;
+    uint32_t tmem_base;
+    int abort;
+};
+
+__global__ void __launch_bounds__(192, 1)
+proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw, int64_t T, int nchunks,
+              int chunks_per_split, int umma_n, int n_out, int stages, int tmem_cols, float* __restrict__ qpart,
+              float* __restrict__ ssq, int* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    // the ring must start on a 1024-byte boundary (swizzle atoms)
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int w_bytes = umma_n * 128;
+    const int stage_bytes = kTcXBytes + w_bytes;
+    TcSmem* ctl = reinterpret_cast<TcSmem*>(smem + stages * stage_bytes);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t t0 = (int64_t)blockIdx.x * kTcTok;
+    const int split = blockIdx.y;
+    const int c_begin = split * chunks_per_split;
+    const int c_end = (c_begin + chunks_per_split < nchunks) ? c_begin + chunks_per_split : nchunks;
+    const int nloc = c_end - c_begin;
+    volatile int* abort = &ctl->abort;
+
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 5); }
+        mbar_init(smem_u32(&ctl->accum), 1);
+        ctl->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {      // tensor-memory allocation (whole warp), address lands in shared memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int i = 0; i < nloc; ++i) {
+                const int s = i % stages;
+                if (!mbar_wait(smem_u32(&ctl->empty[s]), ((i / stages) & 1) ^ 1, abort)) break;
+                const uint32_t full = smem_u32(&ctl->full[s]);
+                mbar_expect_tx(full, stage_bytes);
+                const uint32_t dst = smem_u32(smem + s * stage_bytes);
+                const int k = (c_begin + i) * kTcK;
+                tma_load_2d(dst, &tmx, full, k, (int)t0);
+                tma_load_2d(dst + kTcXBytes, &tmw, full, k, 0);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc(umma_n);
+            bool ok = true;
+            for (int i = 0; i < nloc && ok; ++i) {
+                const int s = i % stages;
+                ok = mbar_wait(smem_u32(&ctl->full[s]), (i / stages) & 1, abort);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t xa = smem_u32(smem + s * stage_bytes);
+                const uint64_t ad = smem_desc_k128(xa), bd = smem_desc_k128(xa + kTcXBytes);
+#pragma unroll
+                for (int kk = 0; kk < kTcK / 16; ++kk)      // 32 bytes further along the swizzled row per k-step
+                    tc_mma(tmem, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                tc_commit(smem_u32(&ctl->empty[s]));        // frees the stage when these MMAs have read it
+            }
+            if (ok) tc_commit(smem_u32(&ctl->accum));       // accumulator complete
+        }
+    } else {
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;                   // this thread's token within the tile
+        float sq = 0.f;
+        bool ok = true;
+        for (int i = 0; i < nloc && ok; ++i) {
+            const int s = i % stages;
+            ok = mbar_wait(smem_u32(&ctl->full[s]), (i / stages) & 1, abort);
+            if (!ok) break;
+            const unsigned char* xr = smem + s * stage_bytes + row * 128;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                float f[8];
+                unpack8(*reinterpret_cast<const uint4*>(xr + ((c ^ (row & 7)) << 4)), f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) sq = fmaf(f[e], f[e], sq);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->empty[s]));
+        }
+        if (ok) ok = mbar_wait(smem_u32(&ctl->accum), 0, abort);
+        ok = __all_sync(0xffffffffu, ok);                   // the tensor-memory loads below are warp-wide
+        if (ok) {
+            tc_fence_after();
+            const int nq = umma_n >> 1;                     // = n_out: hi columns [0, nq), lo columns [nq, 2 nq)
+            const int64_t t = t0 + row;
+            float* qrow = qpart + ((int64_t)split * T + t) * n_out;
+            const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
+            for (int c0 = 0; c0 < nq; c0 += 16) {
+                float hi[16], lo[16];
+                tc_ld16(lane_base + c0, hi);
+                tc_ld16(lane_base + nq + c0, lo);
+                if (t < T) {
+#pragma unroll
+                    for (int e = 0; e < 16; e += 4)
+                        if (c0 + e < nq)
+                            *reinterpret_cast<float4*>(qrow + c0 + e) =
+                                make_float4(hi[e] + lo[e], hi[e + 1] + lo[e + 1], hi[e + 2] + lo[e + 2], hi[e + 3] + lo[e + 3]);
+                }
+            }
+            if (t < T) ssq[(int64_t)split * T + t] = sq;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (ctl->abort) {
+        // let copies that may still be in flight land before the CTA's shared memory is released
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        if (tid == 0) atomicExch(status, MHCLITE_ERR_TIMEOUT);
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
+    }
+}
+
+// ---- W' as two stacked K-major bf16 matrices: rows [0, nq) = hi, rows [nq, 2 nq) = lo, row length Kpad ----
+__global__ void __launch_bounds__(256) pack_wt_k(int nC, int N, int nq, int Kpad, const float* __restrict__ W,
+                                                 const float* __restrict__ gain, __nv_bfloat16* __restrict__ Wt) {
+    const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;       // over nq x Kpad, k fastest
+    if (idx >= (int64_t)nq * Kpad) return;
+    const int c = (int)(idx / Kpad), k = (int)(idx - (int64_t)c * Kpad);
+    const float w = (k < nC && c < N) ? __ldg(W + (int64_t)k * N + c) * __ldg(gain + k) : 0.f;
+    __nv_bfloat16 hi, lo;
+    split_bf16(w, hi, lo);
+    Wt[(int64_t)c * Kpad + k] = hi;
+    Wt[(int64_t)(nq + c) * Kpad + k] = lo;
+}
+
+// ---- host side -------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor map: `rows` rows of `cols` elements (row pitch `pitch_elems`), box = 64 columns x box_rows rows.
+static bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t pitch_elems, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {pitch_elems * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool proj_tc_supported(int n, int C, int N) {
+    const int nq = round_up(N, 8);
+    return 2 * nq <= 256 && ((n * C) % 8) == 0 && encode_tiled_fn() != nullptr;
+}
+
+int proj_tc_nq(int N) { return round_up(N, 8); }
+
+void launch_pack_wt(const mhclite_ctx* c, const ProjPlan& p, int N, const float* W, const float* gain, void* Wt,
+                    cudaStream_t s) {
+    c->launches += 1;
+    const int nq = proj_tc_nq(N), Kpad = p.nchunks * kTcK;
+    const int64_t total = (int64_t)nq * Kpad;
+    pack_wt_k<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(c->n * c->C, N, nq, Kpad, W, gain, (__nv_bfloat16*)Wt);
+}
+
+// Returns false when the tensor maps could not be built (the caller then uses the mma.sync kernel).
+bool launch_proj_fwd_tc(const mhclite_ctx* c, int64_t T, int N, const ProjPlan& p, const void* x, const void* Wt,
+                        float* qpart, float* ssq, int* status, cudaStream_t s) {
+    const int nC = c->n * c->C, nq = proj_tc_nq(N), umma_n = 2 * nq, Kpad = p.nchunks * kTcK;
+    CUtensorMap tmx, tmw;
+    if (!make_map(&tmx, x, (uint64_t)nC, (uint64_t)T, (uint64_t)nC, kTcTok)) return false;
+    if (!make_map(&tmw, Wt, (uint64_t)Kpad, (uint64_t)umma_n, (uint64_t)Kpad, (uint32_t)umma_n)) return false;
+    const int stage_bytes = kTcXBytes + umma_n * 128;
+    int stages = 100 * 1024 / stage_bytes;                   // two CTAs per SM when the stages are small enough
+    if (stages > 6) stages = 6;
+    if (stages < 3) stages = (200 * 1024 / stage_bytes < 4) ? 200 * 1024 / stage_bytes : 4;
+    if (stages > 8) stages = 8;
+    const int smem = stages * stage_bytes + (int)sizeof(TcSmem) + 1024;
+    int tmem_cols = 32;
+    while (tmem_cols < umma_n) tmem_cols *= 2;
+    c->launches += 1;
+    KernelTimer timer_(c, MHCLITE_KERNEL_PROJ_FWD, s);
+    cudaFuncSetAttribute(proj_fwd_tc_k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    dim3 grid((unsigned)((T + kTcTok - 1) / kTcTok), p.ksplit);
+    proj_fwd_tc_k<<<grid, 192, smem, s>>>(tmx, tmw, T, p.nchunks, p.chunks_per_split, umma_n, p.Npad, stages, tmem_cols,
+                                          qpart, ssq, status);
+    return true;
+}
+
+}  // namespace mhcl
