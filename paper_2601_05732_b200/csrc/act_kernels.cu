@@ -998,7 +998,7 @@ void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const v
     // measured faster than one kernel doing both, whose per-token phase stalls the streaming warps
 #define MHCL_TP_T(N_) do { \
         launch_premix_bwd(c, T, x, H_pre, du, dH_pre_ws, nullptr, 0, s); \
-        lite_tailpre_t_k<N_, false, 256, 64><<<group_grid(T, 64, c->sm_count), 256, 0, s>>>( \
+        lite_tailpre_t_k<N_, false, 128, 32><<<group_grid(T, 32, c->sm_count), 128, 0, s>>>( \
             T, C8, inv, (const uint4*)x, (const uint4*)du, dH_pre_ws, a, p, rstd, alpha, H_pre, H_post, dH_res, dH_post, \
             eo, kappa, db, dalpha); } while (0)
     switch (c->n) {
