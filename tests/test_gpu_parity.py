@@ -183,3 +183,18 @@ def test_sk_gap_vs_lite_on_ill_conditioned_logits():
     GL = GpuLayer(lite); GL.forward()
     GL.ctx.ds_gap(GL.B.H_res, l1, cd); torch.cuda.synchronize()
     assert float(l1.max()) < 4e-6 and float(cd.max()) < 1e-6
+
+
+def test_kernel_timing_and_device_status():
+    # the library's own per-kernel events and its device status word (bounded waits record a status there)
+    n, C, T = 4, 256, 2048
+    inp = synth.make_layer_inputs(n, C, T, seed=8, bias_std=0.1)
+    G = GpuLayer(inp)
+    G.ctx.set_kernel_timing(True)
+    G.forward(True); G.backward(True)
+    torch.cuda.synchronize()
+    times = [G.ctx.kernel_time_ms(i) for i in range(len(G.ctx.KERNELS))]
+    assert all(0.0 < t < 50.0 for t in times), times
+    G.ctx.set_kernel_timing(False)
+    G.ctx.device_status()                      # raises if any kernel gave up on a wait
+    compare_forward(G, oracle_fwd(inp))
