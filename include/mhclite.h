@@ -248,7 +248,8 @@ MHCLITE_API int mhclite_step_host(mhclite_ctx* ctx, int64_t T,
 /* Per-kernel device time, for roofline accounting.  With timing on, the library records a pair of CUDA
  * events on the call's stream around each launch of the kernels below (a few microseconds of overhead
  * per launch: switch it off for throughput runs).  mhclite_kernel_time_ms returns the duration of the
- * most recent launch of that kernel; the caller must have synchronised the stream since. */
+ * most recent launch of that kernel; the caller must have synchronised the stream since.  A kernel that
+ * the problem size routes around (the fallbacks replace some of them) has no time: MHCLITE_ERR_BAD_ARG. */
 typedef enum mhclite_kernel {
     MHCLITE_KERNEL_PROJ_FWD = 0,     /* tensor-core projection + sum of squares        reads x            */
     MHCLITE_KERNEL_ACT_PREMIX = 1,   /* mappings + pre-mix                              reads x, writes u  */

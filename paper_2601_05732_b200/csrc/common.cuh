@@ -27,6 +27,7 @@ struct mhclite_ctx {
     int* status_word;             // device status word inside the attached workspace (null until first used)
     bool timing;                  // record CUDA events around the main kernels (mhclite_set_kernel_timing)
     cudaEvent_t ev[MHCLITE_KERNEL_COUNT][2];
+    mutable bool ev_recorded[MHCLITE_KERNEL_COUNT];   // the pair has bracketed at least one launch
     char err[256];
 };
 
@@ -46,7 +47,7 @@ struct KernelTimer {
     KernelTimer(const mhclite_ctx* c_, int id_, cudaStream_t s_) : c(c_), id(id_), s(s_) {
         if (c->timing) cudaEventRecord(c->ev[id][0], s);
     }
-    ~KernelTimer() { if (c->timing) cudaEventRecord(c->ev[id][1], s); }
+    ~KernelTimer() { if (c->timing) { cudaEventRecord(c->ev[id][1], s); c->ev_recorded[id] = true; } }
 };
 
 int fail(mhclite_ctx* ctx, int status, const char* fmt, ...);

@@ -167,7 +167,7 @@ int mhclite_create(mhclite_ctx** out, int n, int C, int device) {
     if (!ctx) return MHCLITE_ERR_CUDA;
     ctx->n = n; ctx->C = C; ctx->device = device; ctx->nfact = ipow_fact(n);
     ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->err[0] = 0; ctx->launches = 0; ctx->timing = false; ctx->status_word = nullptr;
-    for (int k = 0; k < MHCLITE_KERNEL_COUNT; ++k) ctx->ev[k][0] = ctx->ev[k][1] = nullptr;
+    for (int k = 0; k < MHCLITE_KERNEL_COUNT; ++k) { ctx->ev[k][0] = ctx->ev[k][1] = nullptr; ctx->ev_recorded[k] = false; }
     {
         DeviceGuard g(device);
         cudaError_t e = g.err;
@@ -572,6 +572,8 @@ int mhclite_kernel_time_ms(mhclite_ctx* ctx, int kernel, float* ms) {
     MHCL_REQUIRE_CTX(ctx);
     if (kernel < 0 || kernel >= MHCLITE_KERNEL_COUNT || !ms) return fail(ctx, MHCLITE_ERR_BAD_ARG, "bad kernel id");
     if (!ctx->ev[kernel][0]) return fail(ctx, MHCLITE_ERR_BAD_ARG, "kernel timing was never switched on");
+    if (!ctx->ev_recorded[kernel])
+        return fail(ctx, MHCLITE_ERR_BAD_ARG, "kernel %d has not been launched since timing was switched on", kernel);
     return check_cuda(ctx, cudaEventElapsedTime(ms, ctx->ev[kernel][0], ctx->ev[kernel][1]), "cudaEventElapsedTime");
 }
 

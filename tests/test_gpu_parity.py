@@ -198,3 +198,21 @@ def test_kernel_timing_and_device_status():
     G.ctx.set_kernel_timing(False)
     G.ctx.device_status()                      # raises if any kernel gave up on a wait
     compare_forward(G, oracle_fwd(inp))
+
+
+def test_kernel_timing_of_a_kernel_off_the_path_is_an_argument_error():
+    # n = 5 routes around the tensor-core tail: its time is refused cleanly and later calls still work
+    from paper_2601_05732_b200.binding import MhcLiteError
+    n, C, T = 5, 64, 200
+    inp = synth.make_layer_inputs(n, C, T, seed=9, bias_std=0.1)
+    G = GpuLayer(inp)
+    G.ctx.set_kernel_timing(True)
+    G.forward(True); G.backward(True)
+    torch.cuda.synchronize()
+    tail = G.ctx.KERNELS.index("tail_mma")
+    with pytest.raises(MhcLiteError) as ei:
+        G.ctx.kernel_time_ms(tail)
+    assert ei.value.status == -1
+    assert G.ctx.kernel_time_ms(0) > 0.0
+    G.forward(True); torch.cuda.synchronize()
+    compare_forward(G, oracle_fwd(inp))
