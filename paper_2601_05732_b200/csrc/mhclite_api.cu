@@ -43,7 +43,7 @@ Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base) {
     w.ehi = p + off;             off += align256(erows * tp.Kp * 2);
     w.elo = p + off;             off += align256(erows * tp.Kp * 2);
     w.Gpart = (float*)(p + off); off += align256(tp.supported ? (size_t)tp.splits * n * C * tp.Kp * sizeof(float) : 0);
-    w.Wt = p + off;              off += align256((size_t)2 * round_up(N, 8) * pp.nchunks * 64 * 2);
+    w.Wt = p + off;              off += align256((size_t)2 * proj_tc_nq(N) * pp.nchunks * 64 * 2);
     w.status = (int*)(p + off);  off += 256;
     w.bytes = off;
     return w;

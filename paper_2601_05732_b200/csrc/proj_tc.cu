@@ -5,7 +5,9 @@
 //   [2 Nq x 64 k] into a shared-memory ring; one thread issues tcgen05.mma (M = 128 tokens, N = 2 Nq,
 //   K = 16 per instruction) with the fp32 accumulator [128 x 2 Nq] in tensor memory; the bf16 pair
 //   hi | lo of W' sits side by side in N, so x is read from shared memory once per k-step and the two
-//   partial products are added in the epilogue.  Four warps read the same x tiles from shared memory for
+//   partial products are added in the epilogue.  When 2 Nq exceeds the 256 columns of one instruction
+//   (n = 5: 130 columns) the hi and lo halves run as two instructions of N = Nq that accumulate into the
+//   same [128 x Nq] accumulator.  Four warps read the same x tiles from shared memory for
 //   the sum of squares, then fetch the accumulator with tcgen05.ld (thread = token) and store the K slice's
 //   partial result.  The tensor work is a small fraction of the time the bytes take to arrive: the
 //   kernel is bound by HBM.
@@ -103,12 +105,13 @@ struct TcSmem {                       // control block placed after the stage ri
 
 __global__ void __launch_bounds__(192, 1)
 proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw, int64_t T, int nchunks,
-              int chunks_per_split, int umma_n, int n_out, int stages, int tmem_cols, float* __restrict__ qpart,
-              float* __restrict__ ssq, int* __restrict__ status) {
+              int chunks_per_split, int nq, int two_pass, int n_out, int stages, int tmem_cols,
+              float* __restrict__ qpart, float* __restrict__ ssq, int* __restrict__ status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     // the ring must start on a 1024-byte boundary (swizzle atoms)
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const int w_bytes = umma_n * 128;
+    const int w_bytes = 2 * nq * 128;                       // hi rows then lo rows
+    const int umma_n = two_pass ? nq : 2 * nq;
     const int stage_bytes = kTcXBytes + w_bytes;
     TcSmem* ctl = reinterpret_cast<TcSmem*>(smem + stages * stage_bytes);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -146,6 +149,7 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
                 const int k = (c_begin + i) * kTcK;
                 tma_load_2d(dst, &tmx, full, k, (int)t0);
                 tma_load_2d(dst + kTcXBytes, &tmw, full, k, 0);
+                if (two_pass) tma_load_2d(dst + kTcXBytes + nq * 128, &tmw, full, k, nq);   // box = Nq rows
             }
         }
     } else if (warp == 1) {
@@ -159,9 +163,12 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
                 tc_fence_after();
                 const uint32_t xa = smem_u32(smem + s * stage_bytes);
                 const uint64_t ad = smem_desc_k128(xa), bd = smem_desc_k128(xa + kTcXBytes);
+                const uint64_t bl = smem_desc_k128(xa + kTcXBytes + nq * 128);
 #pragma unroll
-                for (int kk = 0; kk < kTcK / 16; ++kk)      // 32 bytes further along the swizzled row per k-step
+                for (int kk = 0; kk < kTcK / 16; ++kk) {    // 32 bytes further along the swizzled row per k-step
                     tc_mma(tmem, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                    if (two_pass) tc_mma(tmem, ad + (uint64_t)(kk * 2), bl + (uint64_t)(kk * 2), idesc, 1u);
+                }
                 tc_commit(smem_u32(&ctl->empty[s]));        // frees the stage when these MMAs have read it
             }
             if (ok) tc_commit(smem_u32(&ctl->accum));       // accumulator complete
@@ -190,14 +197,19 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
         ok = __all_sync(0xffffffffu, ok);                   // the tensor-memory loads below are warp-wide
         if (ok) {
             tc_fence_after();
-            const int nq = umma_n >> 1;                     // = n_out: hi columns [0, nq), lo columns [nq, 2 nq)
+            // hi columns [0, nq), lo columns [nq, 2 nq) (already added when the two halves share the accumulator)
             const int64_t t = t0 + row;
             float* qrow = qpart + ((int64_t)split * T + t) * n_out;
             const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
             for (int c0 = 0; c0 < nq; c0 += 16) {
                 float hi[16], lo[16];
                 tc_ld16(lane_base + c0, hi);
-                tc_ld16(lane_base + nq + c0, lo);
+                if (two_pass) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) lo[e] = 0.f;
+                } else {
+                    tc_ld16(lane_base + nq + c0, lo);
+                }
                 if (t < T) {
 #pragma unroll
                     for (int e = 0; e < 16; e += 4)
@@ -267,12 +279,13 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t r
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-bool proj_tc_supported(int n, int C, int N) {
-    const int nq = round_up(N, 8);
-    return 2 * nq <= 256 && ((n * C) % 8) == 0 && encode_tiled_fn() != nullptr;
-}
+// Columns of one half of W' in the packed operand: a multiple of 8 while both halves fit one instruction
+// (2 Nq <= 256), else a multiple of 16 (the instruction's N granularity at M = 128).
+int proj_tc_nq(int N) { return 2 * round_up(N, 8) <= 256 ? round_up(N, 8) : round_up(N, 16); }
 
-int proj_tc_nq(int N) { return round_up(N, 8); }
+bool proj_tc_supported(int n, int C, int N) {
+    return proj_tc_nq(N) <= 256 && ((n * C) % 8) == 0 && encode_tiled_fn() != nullptr;
+}
 
 void launch_pack_wt(const mhclite_ctx* c, const ProjPlan& p, int N, const float* W, const float* gain, void* Wt,
                     cudaStream_t s) {
@@ -285,11 +298,14 @@ void launch_pack_wt(const mhclite_ctx* c, const ProjPlan& p, int N, const float*
 // Returns false when the tensor maps could not be built (the caller then uses the mma.sync kernel).
 bool launch_proj_fwd_tc(const mhclite_ctx* c, int64_t T, int N, const ProjPlan& p, const void* x, const void* Wt,
                         float* qpart, float* ssq, int* status, cudaStream_t s) {
-    const int nC = c->n * c->C, nq = proj_tc_nq(N), umma_n = 2 * nq, Kpad = p.nchunks * kTcK;
+    const int nC = c->n * c->C, nq = proj_tc_nq(N), Kpad = p.nchunks * kTcK;
+    const int two_pass = 2 * nq > 256;
+    const int umma_n = two_pass ? nq : 2 * nq;
+    if (nq > p.Npad) return false;                            // the rows of qpart hold Npad columns
     CUtensorMap tmx, tmw;
     if (!make_map(&tmx, x, (uint64_t)nC, (uint64_t)T, (uint64_t)nC, kTcTok)) return false;
-    if (!make_map(&tmw, Wt, (uint64_t)Kpad, (uint64_t)umma_n, (uint64_t)Kpad, (uint32_t)umma_n)) return false;
-    const int stage_bytes = kTcXBytes + umma_n * 128;
+    if (!make_map(&tmw, Wt, (uint64_t)Kpad, (uint64_t)(2 * nq), (uint64_t)Kpad, (uint32_t)umma_n)) return false;
+    const int stage_bytes = kTcXBytes + 2 * nq * 128;
     int stages = 100 * 1024 / stage_bytes;                   // two CTAs per SM when the stages are small enough
     if (stages > 6) stages = 6;
     if (stages < 3) stages = (200 * 1024 / stage_bytes < 4) ? 200 * 1024 / stage_bytes : 4;
@@ -301,8 +317,8 @@ bool launch_proj_fwd_tc(const mhclite_ctx* c, int64_t T, int N, const ProjPlan& 
     KernelTimer timer_(c, MHCLITE_KERNEL_PROJ_FWD, s);
     cudaFuncSetAttribute(proj_fwd_tc_k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     dim3 grid((unsigned)((T + kTcTok - 1) / kTcTok), p.ksplit);
-    proj_fwd_tc_k<<<grid, 192, smem, s>>>(tmx, tmw, T, p.nchunks, p.chunks_per_split, umma_n, p.Npad, stages, tmem_cols,
-                                          qpart, ssq, status);
+    proj_fwd_tc_k<<<grid, 192, smem, s>>>(tmx, tmw, T, p.nchunks, p.chunks_per_split, nq, two_pass, p.Npad, stages,
+                                          tmem_cols, qpart, ssq, status);
     return true;
 }
 
