@@ -25,16 +25,27 @@ __device__ __forceinline__ void store_e(const EOut& o, int64_t t, int c, float v
     if (o.ehi) {
         __nv_bfloat16 h, l;
         split_bf16(v, h, l);
-        o.ehi[t * o.Kp + c] = h;
-        o.elo[t * o.Kp + c] = l;
+        const int64_t i = e_tiled_index(o.Kp, t, c);
+        o.ehi[i] = h;
+        o.elo[i] = l;
     }
 }
 __device__ __forceinline__ void pad_e(const EOut& o, int64_t t, int N, int first, int step) {
     if (o.e) for (int c = N + first; c < o.Npad; c += step) o.e[t * o.Npad + c] = 0.f;
     if (o.ehi) for (int c = N + first; c < o.Kp; c += step) {
-        o.ehi[t * o.Kp + c] = __float2bfloat16_rn(0.f);
-        o.elo[t * o.Kp + c] = __float2bfloat16_rn(0.f);
+        const int64_t i = e_tiled_index(o.Kp, t, c);
+        o.ehi[i] = __float2bfloat16_rn(0.f);
+        o.elo[i] = __float2bfloat16_rn(0.f);
     }
+}
+
+// Tokens past T in the last 128-token granule of the tiled e buffers are read by the tensor-core kernels:
+// the granule is cleared before the activation backward fills its valid part.
+static void clear_e_tail(int64_t T, void* ehi, void* elo, int Kp, cudaStream_t s) {
+    if (!ehi || (T % kEGranule) == 0) return;
+    const size_t gbytes = (size_t)Kp * kEGranule * 2, off = (size_t)(T / kEGranule) * gbytes;
+    cudaMemsetAsync((char*)ehi + off, 0, gbytes, s);
+    cudaMemsetAsync((char*)elo + off, 0, gbytes, s);
 }
 
 constexpr int kActThreads = 256;
@@ -730,19 +741,32 @@ __global__ void __launch_bounds__(THREADS) lite_tailpre_t_k(
                 dal_col = fmaf(dz, in_s[tl][o_p + tid], dal_col);
             }
         }
-        // W: e as a bf16 pair (and / or fp32), kappa
-        const int cols = eo.ehi ? eo.Kp : eo.Npad;
-        for (int i = tid; i < nt * cols; i += THREADS) {
-            const int tl = i / cols, c = i - tl * cols;
-            const float v = (c < D::kN) ? og[tl][c] : 0.f;
-            const int64_t t = t0 + tl;
-            if (eo.ehi) {
-                __nv_bfloat16 h, l;
-                split_bf16(v, h, l);
-                eo.ehi[t * eo.Kp + c] = h;
-                eo.elo[t * eo.Kp + c] = l;
+        // W: e as a bf16 pair (one 16-byte piece of 8 columns per thread, consecutive tokens side by side in
+        // the tiled layout) and / or fp32 rows; kappa
+        if (eo.ehi) {
+            for (int i = tid; i < nt * (eo.Kp >> 3); i += THREADS) {
+                const int cg = i / nt, tl = i - cg * nt;
+                uint32_t hw[4], lw[4];
+#pragma unroll
+                for (int e2 = 0; e2 < 4; ++e2) {
+                    const int c = cg * 8 + 2 * e2;
+                    const float v0 = (c < D::kN) ? og[tl][c] : 0.f, v1 = (c + 1 < D::kN) ? og[tl][c + 1] : 0.f;
+                    __nv_bfloat16 h0, l0, h1, l1;
+                    split_bf16(v0, h0, l0);
+                    split_bf16(v1, h1, l1);
+                    hw[e2] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                    lw[e2] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                }
+                const int64_t o = e_tiled_index(eo.Kp, t0 + tl, cg * 8);
+                *reinterpret_cast<uint4*>(eo.ehi + o) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                *reinterpret_cast<uint4*>(eo.elo + o) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
             }
-            if (eo.e && c < eo.Npad) eo.e[t * eo.Npad + c] = v;
+        }
+        if (eo.e) {
+            for (int i = tid; i < nt * eo.Npad; i += THREADS) {
+                const int tl = i / eo.Npad, c = i - tl * eo.Npad;
+                eo.e[(t0 + tl) * eo.Npad + c] = (c < D::kN) ? og[tl][c] : 0.f;
+            }
         }
         if (tid < nt) kappa[t0 + tid] = og[tid][D::kN];
         __syncthreads();
@@ -953,6 +977,7 @@ void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float*
                          const float* dH_pre, const float* dH_post, float* e, void* ehi, void* elo, int Kp,
                          float* kappa, float* db, float* dalpha, cudaStream_t s) {
     const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
+    clear_e_tail(T, ehi, elo, Kp, s);
     c->launches += 1;
     // fewer, longer-lived blocks: the parameter-gradient partials are reduced once per block
     int64_t blocks = (T + kActWarps * 8 - 1) / (kActWarps * 8);
@@ -992,6 +1017,7 @@ void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const v
     c->launches += 1;
     KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_PRE, s);
     const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
+    clear_e_tail(T, ehi, elo, Kp, s);
     const int C8 = c->C / 8;
     const float inv = 1.f / (float)(c->n * c->C);
     // n <= 4: a streaming pass for dH_pre (premix_bwd without dx), then the thread-per-token activation backward;
@@ -1028,6 +1054,7 @@ void launch_sk_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, int iters, con
                        const float* dH_res, const float* dH_pre, const float* dH_post, float* e, void* ehi, void* elo,
                        int Kp, float* kappa, float* db, float* dalpha, cudaStream_t s) {
     const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
+    clear_e_tail(T, ehi, elo, Kp, s);
     c->launches += 1;
     const int grid = (int)((T + 127) / 128);
     const float inv = 1.f / (float)(c->n * c->C);

@@ -37,6 +37,17 @@ inline int ipow_fact(int n) { int f = 1; for (int i = 2; i <= n; ++i) f *= i; re
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 inline int64_t round_up64(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 
+// Layout of e = rstd * alpha (.) dz as a bf16 pair (hi, lo) for the tensor-core backward, Kp columns per
+// token (a multiple of 16).  Tokens are grouped in granules of 128; inside a granule the columns are
+// grouped by 8, and inside a column group the 16-byte pieces of the 128 tokens lie back to back:
+//   element (t, c)  ->  ((t / 128) * (Kp / 8) + c / 8) * 1024 + (t % 128) * 8 + c % 8.
+// A granule is then a ready-made shared-memory operand without swizzle (8 x 16-byte core matrices) both
+// with tokens as the M dimension and columns as K, and with columns as N and tokens as K.
+constexpr int kEGranule = 128;
+__host__ __device__ inline int64_t e_tiled_index(int Kp, int64_t t, int c) {
+    return ((t >> 7) * (Kp >> 3) + (c >> 3)) * 1024 + (t & 127) * 8 + (c & 7);
+}
+
 // Number of projection columns. kind 0: n!+2n (mHC-lite); kind 1: n*n+2n (SK path).
 inline int n_res_cols(int n, int kind) { return kind == 0 ? ipow_fact(n) : n * n; }
 inline int n_cols(int n, int kind) { return n_res_cols(n, kind) + 2 * n; }
@@ -70,7 +81,12 @@ struct TailPlan {
     int Kp, KS;             // projection columns padded to 16, and Kp / 16
     int slices, splits;     // 64-channel slices x token ranges = the grid
     int64_t tok_per_split;  // multiple of 32
-    bool supported;         // KS <= 3 (N <= 48); wider projections use the CUDA-core kernels
+    bool supported;         // KS <= 3 (N <= 48): the fused mma.sync kernel
+    // wider projections: tcgen05 kernels (tail_tc.cu) when the shape allows, else the CUDA-core kernels
+    bool tc;                // Kp <= 256 and rows of x a multiple of 16 bytes
+    int g_mt;               // G kernel: 128-row accumulators per CTA (g_mt * Kp <= 512 tensor-memory columns)
+    int g_groups, g_splits; // its grid: row groups of 128 * g_mt x token ranges
+    int64_t g_tok_per_split;   // multiple of 128
 };
 TailPlan plan_tail(int n, int C, int64_t T, int N, int sm_count);
 
@@ -84,7 +100,7 @@ struct Workspace {
     float* qpart;    // [kMaxKSplit][T][NTpad*8] partial x W' of each K slice
     float* ssq;      // [kMaxKSplit][T]          partial sums of squares
     void *ehi, *elo; // [T rounded up to 32][Kp] bf16 pair hi + lo = e
-    float* Gpart;    // [splits][nC][Kp] partial G of each token range
+    float* Gpart;    // [splits or g_splits][nC][Kp] partial G of each token range
     void* Wt;        // [2 nq][Kpad] bf16: W' hi rows then lo rows, K-major (tcgen05 projection)
     int* status;     // device status word (0, or a negative mhclite_status raised by a kernel)
     size_t bytes;

@@ -33,6 +33,11 @@ void launch_proj_bwd_dw(const mhclite_ctx* c, int64_t T, int N, int Npad, const 
                         cudaStream_t s);
 
 // proj_tc.cu : the same projection on tcgen05 / TMA / tensor memory (N <= 128 columns)
+bool tensor_maps_available();
+bool launch_tail_g_tc(const mhclite_ctx* c, int64_t T, const TailPlan& p, const void* x, const void* ehi,
+                      const void* elo, float* Gpart, int* status, cudaStream_t s);
+void launch_tail_finish(const mhclite_ctx* c, int N, int Kp, int splits, const float* W, const float* gain,
+                        const float* Gpart, float* dW, float* dgain, int acc_params, cudaStream_t s);
 bool proj_tc_supported(int n, int C, int N);
 int proj_tc_nq(int N);
 void launch_pack_wt(const mhclite_ctx* c, const ProjPlan& p, int N, const float* W, const float* gain, void* Wt,

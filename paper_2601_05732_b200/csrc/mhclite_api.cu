@@ -39,10 +39,11 @@ Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base) {
     w.qpart = (float*)(p + off); off += align256((size_t)kMaxKSplit * T * pp.Npad * sizeof(float));
     w.ssq = (float*)(p + off);   off += align256((size_t)kMaxKSplit * T * sizeof(float));
     const TailPlan tp = plan_tail(n, C, T, N, 148);
-    const size_t erows = (size_t)round_up64(T, 32);
+    const size_t erows = (size_t)round_up64(T, kEGranule);
     w.ehi = p + off;             off += align256(erows * tp.Kp * 2);
     w.elo = p + off;             off += align256(erows * tp.Kp * 2);
-    w.Gpart = (float*)(p + off); off += align256(tp.supported ? (size_t)tp.splits * n * C * tp.Kp * sizeof(float) : 0);
+    const int gparts = tp.supported ? tp.splits : (tp.tc ? tp.g_splits : 0);
+    w.Gpart = (float*)(p + off); off += align256((size_t)gparts * n * C * tp.Kp * sizeof(float));
     w.Wt = p + off;              off += align256((size_t)2 * proj_tc_nq(N) * pp.nchunks * 64 * 2);
     w.status = (int*)(p + off);  off += 256;
     w.bytes = off;
@@ -117,6 +118,9 @@ static int proj_forward(mhclite_ctx* ctx, int64_t T, int N, const Workspace& w, 
     return MHCLITE_OK;
 }
 
+// True when the activation backward must leave e as the tiled bf16 pair (a tensor-core kernel reads it).
+static bool tail_pair(const TailPlan& tp) { return tp.supported || (tp.tc && tensor_maps_available()); }
+
 // The part of the backward shared by every entry point, after the activation backward has produced e and
 // kappa: projection / RMSNorm backward into dx (fused with H_res^T g + H_pre du when g is given) and the
 // parameter gradients dW, dgain.  Tensor cores when the projection is narrow enough, CUDA cores otherwise.
@@ -137,6 +141,13 @@ static int proj_backward(mhclite_ctx* ctx, int64_t T, int N, const Workspace& w,
     }
     launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W, gain, w.e, w.kappa, dx, accumulate_dx, s);
     MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dx");
+    if (tail_pair(tp) && launch_tail_g_tc(ctx, T, tp, x, w.ehi, w.elo, w.Gpart, w.status, s)) {
+        MHCL_LAUNCH_CHECK(ctx, "tail_g_tc");
+        ctx->launches += 1;
+        launch_tail_finish(ctx, N, tp.Kp, tp.g_splits, W, gain, w.Gpart, dW, dgain, accumulate_params, s);
+        MHCL_LAUNCH_CHECK(ctx, "tail_finish");
+        return MHCLITE_OK;
+    }
     launch_proj_bwd_dw(ctx, T, N, w.Npad, x, W, gain, w.e, w.G, dW, dgain, accumulate_params, s);
     MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dw");
     return MHCLITE_OK;
@@ -341,7 +352,7 @@ int mhclite_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     if (rc) return rc;
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
     launch_lite_act_bwd(ctx, T, w.Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post,
-                        tp.supported ? nullptr : w.e, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
+                        tp.supported ? nullptr : w.e, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_act_bwd");
     return proj_backward(ctx, T, N, w, tp, x, nullptr, nullptr, nullptr, nullptr, W, gain, dx, accumulate_dx, dW, dgain,
                          accumulate_params, s);
@@ -369,7 +380,7 @@ int mhclite_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, c
     if (rc) return rc;
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
     launch_lite_tailpre(ctx, T, x, du, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_post, w.dH_pre,
-                        tp.supported ? nullptr : w.e, w.Npad, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db,
+                        tp.supported ? nullptr : w.e, w.Npad, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db,
                         dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_tailpre");
     return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W, gain, dx, 0, dW, dgain, accumulate_params, s);
@@ -422,7 +433,7 @@ int mhc_sk20_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
     if (rc) return rc;
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
     launch_sk_act_bwd(ctx, T, w.Npad, iters, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post,
-                      tp.supported ? nullptr : w.e, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
+                      tp.supported ? nullptr : w.e, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "sk_act_bwd");
     return proj_backward(ctx, T, N, w, tp, x, nullptr, nullptr, nullptr, nullptr, W_sk, gain, dx, accumulate_dx, dW,
                          dgain, accumulate_params, s);
@@ -454,7 +465,7 @@ int mhc_sk20_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, 
     launch_premix_bwd(ctx, T, x, H_pre, du, w.dH_pre, nullptr, 0, s);
     MHCL_LAUNCH_CHECK(ctx, "premix_bwd");
     launch_sk_act_bwd(ctx, T, w.Npad, iters, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, w.dH_pre, dH_post,
-                      tp.supported ? nullptr : w.e, tp.supported ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
+                      tp.supported ? nullptr : w.e, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "sk_act_bwd");
     return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W_sk, gain, dx, 0, dW, dgain, accumulate_params, s);
 }

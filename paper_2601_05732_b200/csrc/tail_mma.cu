@@ -39,7 +39,7 @@ struct TailArgs {
     int64_t T, tok_per_split;
     int C, N, Kp;                                  // channels per stream, projection columns, padded to 16
     const __nv_bfloat16 *x, *g, *du;               // g, du only when FUSED
-    const __nv_bfloat16 *ehi, *elo;                // [T][Kp]
+    const __nv_bfloat16 *ehi, *elo;                // Kp columns per token, tiled (e_tiled_index)
     const float *kappa, *H_res, *H_pre;            // H_* only when FUSED
     const float *W, *gain;
     __nv_bfloat16* dx;
@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(256, 2) tail_mma_k(const TailArgs a) {
             const int tl = i / (KS * 2), pc = i - tl * (KS * 2);
             const int64_t t = tt0 + tl;
             const bool ok = t < t_end;
-            const int64_t off = t * a.Kp + pc * 8;
+            const int64_t off = ok ? e_tiled_index(a.Kp, t, pc * 8) : 0;
             cp_async16(sb + Cfg::oEh + tl * Cfg::kEStride + pc * 16, ok ? a.ehi + off : a.x, ok ? 16 : 0);
             cp_async16(sb + Cfg::oEl + tl * Cfg::kEStride + pc * 16, ok ? a.elo + off : a.x, ok ? 16 : 0);
         }
@@ -353,6 +353,20 @@ TailPlan plan_tail(int n, int C, int64_t T, int N, int sm_count) {
     if (p.tok_per_split < kTT) p.tok_per_split = kTT;
     p.splits = (int)((T + p.tok_per_split - 1) / p.tok_per_split);
     if (p.splits < 1) p.splits = 1;
+    // tcgen05 kernels for the wide case
+    p.tc = !p.supported && p.Kp <= 256 && ((n * C) % 8) == 0;
+    p.g_mt = 512 / p.Kp; if (p.g_mt > 3) p.g_mt = 3;
+    const int nC = n * C;
+    if ((nC + 127) / 128 < p.g_mt) p.g_mt = (nC + 127) / 128;
+    p.g_groups = (nC + 128 * p.g_mt - 1) / (128 * p.g_mt);
+    int64_t gs = sm_count / p.g_groups;
+    const int64_t max_gs = (T + kEGranule - 1) / kEGranule;
+    if (gs > max_gs) gs = max_gs;
+    if (gs < 1) gs = 1;
+    p.g_tok_per_split = round_up64((T + gs - 1) / gs, kEGranule);
+    if (p.g_tok_per_split < kEGranule) p.g_tok_per_split = kEGranule;
+    p.g_splits = (int)((T + p.g_tok_per_split - 1) / p.g_tok_per_split);
+    if (p.g_splits < 1) p.g_splits = 1;
     return p;
 }
 
@@ -394,10 +408,16 @@ void launch_tail_mma(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, 
         MHCL_DISPATCH_N(c->n, MHCL_TAIL_KS(N_));
     }
 #undef MHCL_TAIL_KS
+    launch_tail_finish(c, N, p.Kp, p.splits, W, gain, Gpart, dW, dgain, acc_params, s);
+}
+
+// Counted by the caller.
+void launch_tail_finish(const mhclite_ctx* c, int N, int Kp, int splits, const float* W, const float* gain,
+                        const float* Gpart, float* dW, float* dgain, int acc_params, cudaStream_t s) {
     const int nC = c->n * c->C;
     const int fg = (nC + 7) / 8;
-    if (acc_params) tail_finish_k<true><<<fg, 256, 0, s>>>(nC, N, p.Kp, p.splits, W, gain, Gpart, dW, dgain);
-    else tail_finish_k<false><<<fg, 256, 0, s>>>(nC, N, p.Kp, p.splits, W, gain, Gpart, dW, dgain);
+    if (acc_params) tail_finish_k<true><<<fg, 256, 0, s>>>(nC, N, Kp, splits, W, gain, Gpart, dW, dgain);
+    else tail_finish_k<false><<<fg, 256, 0, s>>>(nC, N, Kp, splits, W, gain, Gpart, dW, dgain);
 }
 
 }  // namespace mhcl
