@@ -101,6 +101,7 @@ struct Workspace {
     float* ssq;      // [kMaxKSplit][T]          partial sums of squares
     void *ehi, *elo; // [T rounded up to 32][Kp] bf16 pair hi + lo = e
     float* Gpart;    // [splits or g_splits][nC][Kp] partial G of each token range
+    void* Wb;        // bf16 W' blocks of the tcgen05 dx kernel (wide projections only)
     void* Wt;        // [2 nq][Kpad] bf16: W' hi rows then lo rows, K-major (tcgen05 projection)
     int* status;     // device status word (0, or a negative mhclite_status raised by a kernel)
     size_t bytes;

@@ -45,6 +45,7 @@ Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base) {
     const int gparts = tp.supported ? tp.splits : (tp.tc ? tp.g_splits : 0);
     w.Gpart = (float*)(p + off); off += align256((size_t)gparts * n * C * tp.Kp * sizeof(float));
     w.Wt = p + off;              off += align256((size_t)2 * proj_tc_nq(N) * pp.nchunks * 64 * 2);
+    w.Wb = p + off;              off += align256(tp.tc ? tail_wb_bytes(n, C, tp.Kp) : 0);
     w.status = (int*)(p + off);  off += 256;
     w.bytes = off;
     return w;
@@ -134,13 +135,21 @@ static int proj_backward(mhclite_ctx* ctx, int64_t T, int N, const Workspace& w,
         MHCL_LAUNCH_CHECK(ctx, "tail_mma");
         return MHCLITE_OK;
     }
-    if (g) {
+    bool dx_done = false;
+    if (tail_pair(tp)) {
+        dx_done = launch_tail_dx_tc(ctx, T, N, tp, x, g, du, w.ehi, w.kappa, H_res, H_pre, W, gain, w.Wb, dx,
+                                    accumulate_dx, w.status, s);
+        if (dx_done) MHCL_LAUNCH_CHECK(ctx, "tail_dx_tc");
+    }
+    if (!dx_done && g) {
         launch_tail_mix(ctx, T, x, g, du, H_res, H_pre, nullptr, dx, s);
         MHCL_LAUNCH_CHECK(ctx, "tail_mix");
         accumulate_dx = 1;
     }
-    launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W, gain, w.e, w.kappa, dx, accumulate_dx, s);
-    MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dx");
+    if (!dx_done) {
+        launch_proj_bwd_dx(ctx, T, N, w.Npad, x, W, gain, w.e, w.kappa, dx, accumulate_dx, s);
+        MHCL_LAUNCH_CHECK(ctx, "proj_bwd_dx");
+    }
     if (tail_pair(tp) && launch_tail_g_tc(ctx, T, tp, x, w.ehi, w.elo, w.Gpart, w.status, s)) {
         MHCL_LAUNCH_CHECK(ctx, "tail_g_tc");
         ctx->launches += 1;

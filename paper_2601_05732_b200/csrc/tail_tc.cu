@@ -153,6 +153,293 @@ tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __nv_bfloat16* __rest
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+//   tail_dx_tc_k : dxhat[t,m] = sum_c e[t,c] W'[m,c] - x[t,m] kappa_t, fused with the rest of dx:
+//                    FUSED:  dx[t,j,c] = sum_i H_res[t,i,j] g[t,i,c] + H_pre[t,j] du[t,c] + dxhat[t,j*C+c]
+//                    else :  dx (+)= dxhat
+//   A CTA keeps the e tile of 128 tokens (hi part, one granule of the tiled buffer) in shared memory and
+//   walks over blocks of 32 channels: per block and stream j one small W' operand (packed by pack_wb_k,
+//   K-major without swizzle) streams through a ring, tcgen05.mma (M = 128 tokens, N = 32 channels,
+//   K = Kp) leaves dxhat of all n streams in one of two tensor-memory buffers, and the four epilogue
+//   warps (thread = token) combine it with x, g and du, which TMA delivers per 32-token quadrant
+//   (64-byte swizzle) through a second ring, and store dx.  Work items (token tile, channel block) are
+//   dealt out in contiguous runs, one run per CTA, so that the e tile is reloaded only at tile changes.
+constexpr int kDTok = 128;                      // tokens per tile (UMMA M)
+constexpr int kDCh = 32;                        // channels per block (UMMA N)
+constexpr int kDBox = 32 * 64;                  // one TMA box: 32 tokens x 32 channels of bf16
+constexpr int kDWSlots = 4;
+constexpr int kDDSlots = 5;
+
+struct DCtl {
+    uint64_t e_full, e_empty, w_full[kDWSlots], w_empty[kDWSlots], d_full[kDDSlots], d_empty[kDDSlots],
+        acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+struct DxArgs {
+    int64_t T;
+    int C, Kp, ncb;                 // channels per stream, padded projection columns, channel blocks per stream
+    int64_t items, per_cta;         // work items = token tiles x channel blocks
+    int tmem_cols;
+    const __nv_bfloat16* ehi;       // tiled
+    const __nv_bfloat16* Wb;        // [n][ncb][Kp/8][32][8]
+    const float *kappa, *H_res, *H_pre;
+    __nv_bfloat16* dx;
+    int* status;
+};
+
+__device__ __forceinline__ void tc_ld8_nowait(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+}
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Ties the registers of an earlier tcgen05.ld to a point after the wait, so that no use is scheduled before it.
+__device__ __forceinline__ void tc_ld_settle(uint32_t (&r)[8]) {
+    asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]) :: "memory");
+}
+
+template <int N_, bool FUSED, bool ACC>
+__global__ void __launch_bounds__(192, 1)
+tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmg,
+             const __grid_constant__ CUtensorMap tmdu, const DxArgs a) {
+    constexpr int kBoxes = FUSED ? 2 * N_ + 1 : N_;
+    constexpr int kDSlot = kBoxes * kDBox;
+    constexpr int kDW = N_ * kDCh;                             // tensor-memory columns of one dxhat buffer
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int e_bytes = a.Kp * kDTok * 2;
+    const int w_bytes = a.Kp * kDCh * 2;
+    unsigned char* e_s = smem;
+    unsigned char* w_s = e_s + e_bytes;                        // e_bytes is a multiple of 4096
+    unsigned char* d_s = w_s + ((kDWSlots * w_bytes + 1023) & ~1023);
+    DCtl* ctl = reinterpret_cast<DCtl*>(d_s + kDDSlots * kDSlot);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t it_begin = (int64_t)blockIdx.x * a.per_cta;
+    const int64_t it_end = (it_begin + a.per_cta < a.items) ? it_begin + a.per_cta : a.items;
+    const int nit = it_end > it_begin ? (int)(it_end - it_begin) : 0;
+    volatile int* abort = &ctl->abort;
+
+    if (tid == 0) {
+        mbar_init(smem_u32(&ctl->e_full), 1); mbar_init(smem_u32(&ctl->e_empty), 1);
+        for (int s = 0; s < kDWSlots; ++s) { mbar_init(smem_u32(&ctl->w_full[s]), 1); mbar_init(smem_u32(&ctl->w_empty[s]), 1); }
+        for (int s = 0; s < kDDSlots; ++s) { mbar_init(smem_u32(&ctl->d_full[s]), 1); mbar_init(smem_u32(&ctl->d_empty[s]), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->acc_full[s]), 1); mbar_init(smem_u32(&ctl->acc_empty[s]), 4); }
+        ctl->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(a.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ---- producer -------------------------------------------------------------------------------
+        if (lane == 0) {
+            int64_t cur_tile = -1;
+            int ec = 0;
+            bool ok = true;
+            for (int li = 0; li < nit && ok; ++li) {
+                const int64_t item = it_begin + li;
+                const int64_t tile = item / a.ncb;
+                const int cb = (int)(item - tile * a.ncb);
+                if (tile != cur_tile) {
+                    ok = mbar_wait(smem_u32(&ctl->e_empty), (ec & 1) ^ 1, abort);
+                    if (!ok) break;
+                    mbar_expect_tx(smem_u32(&ctl->e_full), e_bytes);
+                    bulk_load(smem_u32(e_s), a.ehi + tile * (int64_t)a.Kp * kDTok, e_bytes, smem_u32(&ctl->e_full));
+                    cur_tile = tile;
+                    ++ec;
+                }
+                for (int j = 0; j < N_ && ok; ++j) {
+                    const int wi = li * N_ + j, ws = wi % kDWSlots;
+                    ok = mbar_wait(smem_u32(&ctl->w_empty[ws]), ((wi / kDWSlots) & 1) ^ 1, abort);
+                    if (!ok) break;
+                    mbar_expect_tx(smem_u32(&ctl->w_full[ws]), w_bytes);
+                    bulk_load(smem_u32(w_s + ws * w_bytes), a.Wb + ((int64_t)j * a.ncb + cb) * a.Kp * kDCh, w_bytes,
+                              smem_u32(&ctl->w_full[ws]));
+                }
+                for (int q = 0; q < 4 && ok; ++q) {
+                    const int si = li * 4 + q, ds = si % kDDSlots;
+                    ok = mbar_wait(smem_u32(&ctl->d_empty[ds]), ((si / kDDSlots) & 1) ^ 1, abort);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&ctl->d_full[ds]);
+                    mbar_expect_tx(full, kDSlot);
+                    const uint32_t dst = smem_u32(d_s + ds * kDSlot);
+                    const int row = (int)(tile * kDTok + q * 32);
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) {
+                        tma_load_2d(dst + j * kDBox, &tmx, full, j * a.C + cb * kDCh, row);
+                        if (FUSED) tma_load_2d(dst + (N_ + j) * kDBox, &tmg, full, j * a.C + cb * kDCh, row);
+                    }
+                    if (FUSED) tma_load_2d(dst + 2 * N_ * kDBox, &tmdu, full, cb * kDCh, row);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer -----------------------------------------------------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_mn(128, kDCh, 0, 0);
+            const int ksteps = a.Kp >> 4;
+            int64_t cur_tile = -1;
+            int ec = 0;
+            bool ok = true;
+            for (int li = 0; li < nit && ok; ++li) {
+                const int64_t item = it_begin + li;
+                const int64_t tile = item / a.ncb;
+                const int buf = li & 1;
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[buf]), ((li >> 1) & 1) ^ 1, abort);
+                if (!ok) break;
+                if (tile != cur_tile) {
+                    ok = mbar_wait(smem_u32(&ctl->e_full), ec & 1, abort);
+                    if (!ok) break;
+                    cur_tile = tile;
+                    ++ec;
+                }
+                for (int j = 0; j < N_ && ok; ++j) {
+                    const int wi = li * N_ + j, ws = wi % kDWSlots;
+                    ok = mbar_wait(smem_u32(&ctl->w_full[ws]), (wi / kDWSlots) & 1, abort);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t ea = smem_u32(e_s), wa = smem_u32(w_s + ws * w_bytes);
+                    for (int ks = 0; ks < ksteps; ++ks) {
+                        // A: tokens x columns, K-major, no swizzle: column groups 2 KB apart, 8-token groups 128 B apart
+                        // B: channels x columns, K-major, no swizzle: column groups 512 B apart, 8-channel groups 128 B apart
+                        tc_mma(tmem + buf * kDW + j * kDCh, smem_desc(ea + ks * 4096, 2048, 128, 0),
+                               smem_desc(wa + ks * 1024, 512, 128, 0), idesc, ks > 0 ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&ctl->w_empty[ws]));
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&ctl->acc_full[buf]));
+                const bool last_of_tile = (li + 1 == nit) || ((item + 1) / a.ncb != tile);
+                if (last_of_tile) tc_commit(smem_u32(&ctl->e_empty));
+            }
+        }
+    } else {
+        // ---- epilogue: thread = token ---------------------------------------------------------------
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;                         // token within the tile
+        float kap = 0.f, hp[N_], hr[N_][N_];
+        int64_t cur_tile = -1;
+        bool ok = true;
+        for (int li = 0; li < nit; ++li) {
+            const int64_t item = it_begin + li;
+            const int64_t tile = item / a.ncb;
+            const int cb = (int)(item - tile * a.ncb);
+            const int64_t t = tile * kDTok + r;
+            const bool live = t < a.T;
+            if (tile != cur_tile) {
+                cur_tile = tile;
+                kap = live ? __ldg(a.kappa + t) : 0.f;
+                if (FUSED) {
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) hp[j] = live ? __ldg(a.H_pre + t * N_ + j) : 0.f;
+#pragma unroll
+                    for (int i = 0; i < N_; ++i)
+#pragma unroll
+                        for (int j = 0; j < N_; ++j) hr[i][j] = live ? __ldg(a.H_res + t * N_ * N_ + i * N_ + j) : 0.f;
+                }
+            }
+            const int buf = li & 1;
+            const int si = li * 4 + quad, ds = si % kDDSlots;
+            ok = mbar_wait(smem_u32(&ctl->acc_full[buf]), (li >> 1) & 1, abort);
+            if (ok) ok = mbar_wait(smem_u32(&ctl->d_full[ds]), (si / kDDSlots) & 1, abort);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const unsigned char* slot = d_s + ds * kDSlot;
+            const int rsw = (lane >> 1) & 3;                    // 64-byte swizzle: piece ^= (row / 2) % 4
+            const uint32_t tbase = tmem + ((uint32_t)(quad * 32) << 16) + buf * kDW;
+#pragma unroll
+            for (int pc = 0; pc < 4; ++pc) {
+                const int po = lane * 64 + ((pc ^ rsw) << 4);
+                uint32_t acc[N_][8];
+#pragma unroll
+                for (int j = 0; j < N_; ++j) tc_ld8_nowait(tbase + j * kDCh + pc * 8, acc[j]);
+                float gf[FUSED ? N_ : 1][8], df[8];
+                if (FUSED) {
+#pragma unroll
+                    for (int i = 0; i < N_; ++i) unpack8(*reinterpret_cast<const uint4*>(slot + (N_ + i) * kDBox + po), gf[i]);
+                    unpack8(*reinterpret_cast<const uint4*>(slot + 2 * N_ * kDBox + po), df);
+                }
+                tc_ld_wait();
+#pragma unroll
+                for (int j = 0; j < N_; ++j) tc_ld_settle(acc[j]);
+                const int ch = cb * kDCh + pc * 8;
+#pragma unroll
+                for (int j = 0; j < N_; ++j) {
+                    float xf[8], o[8];
+                    unpack8(*reinterpret_cast<const uint4*>(slot + j * kDBox + po), xf);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) o[e] = fmaf(-xf[e], kap, __uint_as_float(acc[j][e]));
+                    if (FUSED) {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) o[e] = fmaf(hp[j], df[e], o[e]);
+#pragma unroll
+                        for (int i = 0; i < N_; ++i)
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) o[e] = fmaf(hr[i][j], gf[i][e], o[e]);
+                    }
+                    if (live && ch < a.C) {
+                        __nv_bfloat16* dst = a.dx + (t * N_ + j) * a.C + ch;
+                        if (ACC) {
+                            float old[8];
+                            unpack8(*reinterpret_cast<const uint4*>(dst), old);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) o[e] += old[e];
+                        }
+                        st_stream(dst, pack8(o));
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&ctl->d_empty[ds]));
+                mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (ctl->abort) {
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        if (tid == 0) atomicExch(a.status, MHCLITE_ERR_TIMEOUT);
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(a.tmem_cols) : "memory");
+    }
+}
+
+// W' = diag(gain) W in bf16 as the B operand of tail_dx_tc_k: per (stream j, channel block cb) a block
+// [Kp/8 column groups][32 channels][8 columns]; zero beyond N columns and beyond C channels.
+__global__ void __launch_bounds__(256) pack_wb_k(int n, int C, int N, int Kp, int ncb, const float* __restrict__ W,
+                                                 const float* __restrict__ gain, __nv_bfloat16* __restrict__ Wb) {
+    const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int64_t total = (int64_t)n * ncb * Kp * kDCh;
+    if (idx >= total) return;
+    const int c8 = (int)(idx & 7), chl = (int)((idx >> 3) & 31);
+    const int64_t rest = idx >> 8;                             // (j * ncb + cb) * (Kp / 8) + cg
+    const int cg = (int)(rest % (Kp >> 3));
+    const int64_t jb = rest / (Kp >> 3);
+    const int cb = (int)(jb % ncb), j = (int)(jb / ncb);
+    const int ch = cb * kDCh + chl, col = cg * 8 + c8;
+    float w = 0.f;
+    if (ch < C && col < N) {
+        const int m = j * C + ch;
+        w = __ldg(W + (int64_t)m * N + col) * __ldg(gain + m);
+    }
+    Wb[idx] = __float2bfloat16_rn(w);
+}
+
 // ---- host side -------------------------------------------------------------------------------------
 template <int MT>
 static void launch_g_t(const TailPlan& p, const CUtensorMap& tmx, const void* ehi, const void* elo, int64_t T, int nC,
@@ -179,6 +466,60 @@ bool launch_tail_g_tc(const mhclite_ctx* c, int64_t T, const TailPlan& p, const 
         case 2: launch_g_t<2>(p, tmx, ehi, elo, T, nC, Gpart, status, s); break;
         default: launch_g_t<3>(p, tmx, ehi, elo, T, nC, Gpart, status, s); break;
     }
+    return true;
+}
+
+size_t tail_wb_bytes(int n, int C, int Kp) { return (size_t)n * ((C + kDCh - 1) / kDCh) * Kp * kDCh * 2; }
+
+template <int N_>
+static void launch_dx_t(int grid, int smem, const CUtensorMap& tmx, const CUtensorMap& tmg, const CUtensorMap& tmdu,
+                        const DxArgs& a, bool fused, bool acc, cudaStream_t s) {
+#define MHCL_DX(F, A)                                                                                        \
+    do {                                                                                                     \
+        cudaFuncSetAttribute(tail_dx_tc_k<N_, F, A>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);     \
+        tail_dx_tc_k<N_, F, A><<<grid, 192, smem, s>>>(tmx, tmg, tmdu, a);                                   \
+    } while (0)
+    if (fused) MHCL_DX(true, false);
+    else if (acc) MHCL_DX(false, true);
+    else MHCL_DX(false, false);
+#undef MHCL_DX
+}
+
+// dx of the projection / RMSNorm backward, fused with H_res^T g + H_pre du when g is given.  Packs W' first.
+// False (nothing launched) when the shape does not fit shared memory or no tensor map could be made.
+bool launch_tail_dx_tc(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, const void* x, const void* g,
+                       const void* du, const void* ehi, const float* kappa, const float* H_res, const float* H_pre,
+                       const float* W, const float* gain, void* Wb, void* dx, int acc_dx, int* status, cudaStream_t s) {
+    const int n = c->n, C = c->C, nC = n * C;
+    const bool fused = g != nullptr;
+    const int boxes = fused ? 2 * n + 1 : n;
+    const int e_bytes = p.Kp * kDTok * 2, w_bytes = p.Kp * kDCh * 2;
+    const int smem = e_bytes + ((kDWSlots * w_bytes + 1023) & ~1023) + kDDSlots * boxes * kDBox + (int)sizeof(DCtl) + 1024;
+    if (smem > 227 * 1024) return false;
+    CUtensorMap tmx, tmg, tmdu;
+    if (!make_tensor_map_2d(&tmx, x, (uint64_t)nC, (uint64_t)T, (uint64_t)nC, kDCh, 32, 64)) return false;
+    tmg = tmx; tmdu = tmx;
+    if (fused) {
+        if (!make_tensor_map_2d(&tmg, g, (uint64_t)nC, (uint64_t)T, (uint64_t)nC, kDCh, 32, 64)) return false;
+        if (!make_tensor_map_2d(&tmdu, du, (uint64_t)C, (uint64_t)T, (uint64_t)C, kDCh, 32, 64)) return false;
+    }
+    DxArgs a;
+    a.T = T; a.C = C; a.Kp = p.Kp; a.ncb = (C + kDCh - 1) / kDCh;
+    a.items = ((T + kDTok - 1) / kDTok) * a.ncb;
+    int grid = c->sm_count;
+    if ((int64_t)grid > a.items) grid = (int)a.items;
+    if (grid < 1) return false;
+    a.per_cta = (a.items + grid - 1) / grid;
+    grid = (int)((a.items + a.per_cta - 1) / a.per_cta);
+    a.tmem_cols = 32;
+    while (a.tmem_cols < 2 * n * kDCh) a.tmem_cols *= 2;
+    a.ehi = (const __nv_bfloat16*)ehi; a.Wb = (const __nv_bfloat16*)Wb;
+    a.kappa = kappa; a.H_res = H_res; a.H_pre = H_pre; a.dx = (__nv_bfloat16*)dx; a.status = status;
+    c->launches += 2;
+    const int64_t total = (int64_t)n * a.ncb * p.Kp * kDCh;
+    pack_wb_k<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(n, C, N, p.Kp, a.ncb, W, gain, (__nv_bfloat16*)Wb);
+    KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_MMA, s);
+    MHCL_DISPATCH_N(n, (launch_dx_t<N_>(grid, smem, tmx, tmg, tmdu, a, fused, acc_dx != 0, s)));
     return true;
 }
 
