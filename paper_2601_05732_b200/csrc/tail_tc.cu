@@ -160,15 +160,15 @@ tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __nv_bfloat16* __rest
 //   A CTA keeps the e tile of 128 tokens (hi part, one granule of the tiled buffer) in shared memory and
 //   walks over blocks of 32 channels: per block and stream j one small W' operand (packed by pack_wb_k,
 //   K-major without swizzle) streams through a ring, tcgen05.mma (M = 128 tokens, N = 32 channels,
-//   K = Kp) leaves dxhat of all n streams in one of two tensor-memory buffers, and the four epilogue
-//   warps (thread = token) combine it with x, g and du, which TMA delivers per 32-token quadrant
+//   K = Kp) leaves dxhat of all n streams in one of two tensor-memory buffers, and the eight epilogue
+//   warps (thread = token, two warps per lane quadrant) combine it with x, g and du, which TMA delivers per 32-token quadrant
 //   (64-byte swizzle) through a second ring, and store dx.  Work items (token tile, channel block) are
 //   dealt out in contiguous runs, one run per CTA, so that the e tile is reloaded only at tile changes.
 constexpr int kDTok = 128;                      // tokens per tile (UMMA M)
 constexpr int kDCh = 32;                        // channels per block (UMMA N)
 constexpr int kDBox = 32 * 64;                  // one TMA box: 32 tokens x 32 channels of bf16
 constexpr int kDWSlots = 4;
-constexpr int kDDSlots = 5;
+constexpr int kDDSlots = 6;
 
 struct DCtl {
     uint64_t e_full, e_empty, w_full[kDWSlots], w_empty[kDWSlots], d_full[kDDSlots], d_empty[kDDSlots],
@@ -200,8 +200,10 @@ __device__ __forceinline__ void tc_ld_settle(uint32_t (&r)[8]) {
     asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]) :: "memory");
 }
 
+constexpr int kDThreads = 64 + 256;              // producer warp, MMA warp, 8 epilogue warps
+
 template <int N_, bool FUSED, bool ACC>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kDThreads, 1)
 tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmg,
              const __grid_constant__ CUtensorMap tmdu, const DxArgs a) {
     constexpr int kBoxes = FUSED ? 2 * N_ + 1 : N_;
@@ -224,8 +226,8 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
     if (tid == 0) {
         mbar_init(smem_u32(&ctl->e_full), 1); mbar_init(smem_u32(&ctl->e_empty), 1);
         for (int s = 0; s < kDWSlots; ++s) { mbar_init(smem_u32(&ctl->w_full[s]), 1); mbar_init(smem_u32(&ctl->w_empty[s]), 1); }
-        for (int s = 0; s < kDDSlots; ++s) { mbar_init(smem_u32(&ctl->d_full[s]), 1); mbar_init(smem_u32(&ctl->d_empty[s]), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->acc_full[s]), 1); mbar_init(smem_u32(&ctl->acc_empty[s]), 4); }
+        for (int s = 0; s < kDDSlots; ++s) { mbar_init(smem_u32(&ctl->d_full[s]), 1); mbar_init(smem_u32(&ctl->d_empty[s]), 2); }
+        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->acc_full[s]), 1); mbar_init(smem_u32(&ctl->acc_empty[s]), 8); }
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -323,8 +325,9 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
             }
         }
     } else {
-        // ---- epilogue: thread = token ---------------------------------------------------------------
+        // ---- epilogue: thread = token; the two warps of a lane quadrant take 16 channels each ---------
         const int quad = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int r = quad * 32 + lane;                         // token within the tile
         float kap = 0.f, hp[N_], hr[N_][N_];
         int64_t cur_tile = -1;
@@ -358,7 +361,8 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
             const int rsw = (lane >> 1) & 3;                    // 64-byte swizzle: piece ^= (row / 2) % 4
             const uint32_t tbase = tmem + ((uint32_t)(quad * 32) << 16) + buf * kDW;
 #pragma unroll
-            for (int pc = 0; pc < 4; ++pc) {
+            for (int pp = 0; pp < 2; ++pp) {
+                const int pc = half * 2 + pp;
                 const int po = lane * 64 + ((pc ^ rsw) << 4);
                 uint32_t acc[N_][8];
 #pragma unroll
@@ -477,7 +481,7 @@ static void launch_dx_t(int grid, int smem, const CUtensorMap& tmx, const CUtens
 #define MHCL_DX(F, A)                                                                                        \
     do {                                                                                                     \
         cudaFuncSetAttribute(tail_dx_tc_k<N_, F, A>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);     \
-        tail_dx_tc_k<N_, F, A><<<grid, 192, smem, s>>>(tmx, tmg, tmdu, a);                                   \
+        tail_dx_tc_k<N_, F, A><<<grid, kDThreads, smem, s>>>(tmx, tmg, tmdu, a);                                   \
     } while (0)
     if (fused) MHCL_DX(true, false);
     else if (acc) MHCL_DX(false, true);

@@ -16,6 +16,7 @@ pytestmark = pytest.mark.gpu
 
 CASES = [  # (n, C, T): ragged token tails (T not a multiple of 32/64/128) and ragged channel tails
     (4, 256, 333), (4, 264, 130), (2, 8, 77), (3, 72, 200), (5, 136, 161), (4, 1024, 257), (3, 1536, 65),
+    (5, 320, 700),
 ]
 
 
