@@ -90,11 +90,12 @@ static int need_workspace(mhclite_ctx* ctx, int64_t T, int kind, Workspace* w) {
     if (!ctx->ws || ctx->ws_bytes < need)
         return fail(ctx, MHCLITE_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu attached", need, ctx->ws ? ctx->ws_bytes : (size_t)0);
     *w = plan_workspace(ctx->n, ctx->C, T, kind, ctx->ws);
-    // one status word per workspace, at its very end, cleared when first used
-    w->status = (int*)((char*)ctx->ws + ((ctx->ws_bytes - sizeof(int)) & ~(size_t)255));
+    // status words of the workspace (status + four words describing the first report), at its very end,
+    // cleared when first used
+    w->status = (int*)((char*)ctx->ws + ((ctx->ws_bytes - 32) & ~(size_t)255));
     if (ctx->status_word != w->status) {
         DeviceGuard g(ctx->device);
-        if (cudaMemset(w->status, 0, sizeof(int)) != cudaSuccess) return fail(ctx, MHCLITE_ERR_CUDA, "clearing the status word");
+        if (cudaMemset(w->status, 0, 32) != cudaSuccess) return fail(ctx, MHCLITE_ERR_CUDA, "clearing the status word");
         ctx->status_word = w->status;
     }
     return MHCLITE_OK;
@@ -566,10 +567,12 @@ int mhclite_device_status(mhclite_ctx* ctx) {
     MHCL_REQUIRE_CTX(ctx);
     if (!ctx->status_word) return MHCLITE_OK;
     MHCL_DEVICE(ctx);
-    int v = 0;
-    int rc = check_cuda(ctx, cudaMemcpy(&v, ctx->status_word, sizeof(int), cudaMemcpyDeviceToHost), "read status word");
+    int v[5] = {0, 0, 0, 0, 0};
+    int rc = check_cuda(ctx, cudaMemcpy(v, ctx->status_word, sizeof(v), cudaMemcpyDeviceToHost), "read status word");
     if (rc) return rc;
-    if (v != 0) return fail(ctx, v, "a kernel gave up on a bounded wait (status %d)", v);
+    if (v[0] != 0)
+        return fail(ctx, v[0], "a kernel gave up on a bounded wait (kernel %d, wait %d, block %d, index %d)", v[1], v[2],
+                    v[3], v[4]);
     return MHCLITE_OK;
 }
 

@@ -46,7 +46,7 @@ __host__ __device__ constexpr uint32_t umma_idesc(int n) {
 struct TcSmem {                       // control block placed after the stage ring
     uint64_t full[8], empty[8], accum;
     uint32_t tmem_base;
-    int abort;
+    int abort[3];
 };
 
 __global__ void __launch_bounds__(192, 1)
@@ -66,12 +66,12 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
     const int c_begin = split * chunks_per_split;
     const int c_end = (c_begin + chunks_per_split < nchunks) ? c_begin + chunks_per_split : nchunks;
     const int nloc = c_end - c_begin;
-    volatile int* abort = &ctl->abort;
+    volatile int* abort = ctl->abort;
 
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 5); }
         mbar_init(smem_u32(&ctl->accum), 1);
-        ctl->abort = 0;
+        ctl->abort[0] = ctl->abort[1] = ctl->abort[2] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -169,11 +169,7 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
     }
     tc_fence_before();
     __syncthreads();
-    if (ctl->abort) {
-        // let copies that may still be in flight land before the CTA's shared memory is released
-        for (int i = 0; i < 64; ++i) __nanosleep(2000);
-        if (tid == 0) atomicExch(status, MHCLITE_ERR_TIMEOUT);
-    }
+    if (ctl->abort[0]) report_abort(abort, status, 1);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");

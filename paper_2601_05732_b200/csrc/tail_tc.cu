@@ -27,7 +27,7 @@ constexpr int kGXBox = kGTok * 128;             // one TMA box: 64 tokens x 64 c
 struct GCtl {
     uint64_t full[kGStages], empty[kGStages], accum;
     uint32_t tmem_base;
-    int abort;
+    int abort[3];
 };
 
 template <int MT>
@@ -47,12 +47,12 @@ tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __nv_bfloat16* __rest
     const int64_t t_begin = (int64_t)blockIdx.y * tok_per_split;       // multiple of 128
     const int64_t t_end = (t_begin + tok_per_split < T) ? t_begin + tok_per_split : T;
     const int nblk = (t_end > t_begin) ? (int)((t_end - t_begin + kGTok - 1) / kGTok) : 0;
-    volatile int* abort = &ctl->abort;
+    volatile int* abort = ctl->abort;
 
     if (tid == 0) {
         for (int s = 0; s < kGStages; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
         mbar_init(smem_u32(&ctl->accum), 1);
-        ctl->abort = 0;
+        ctl->abort[0] = ctl->abort[1] = ctl->abort[2] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -69,7 +69,7 @@ tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __nv_bfloat16* __rest
         if (lane == 0) {
             for (int i = 0; i < nblk; ++i) {
                 const int s = i % kGStages;
-                if (!mbar_wait(smem_u32(&ctl->empty[s]), ((i / kGStages) & 1) ^ 1, abort)) break;
+                if (!mbar_wait(smem_u32(&ctl->empty[s]), ((i / kGStages) & 1) ^ 1, abort, 1, i)) break;
                 const uint32_t full = smem_u32(&ctl->full[s]);
                 mbar_expect_tx(full, stage_bytes);
                 const uint32_t dst = smem_u32(smem + s * stage_bytes);
@@ -90,7 +90,7 @@ tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __nv_bfloat16* __rest
             bool ok = true;
             for (int i = 0; i < nblk && ok; ++i) {
                 const int s = i % kGStages;
-                ok = mbar_wait(smem_u32(&ctl->full[s]), (i / kGStages) & 1, abort);
+                ok = mbar_wait(smem_u32(&ctl->full[s]), (i / kGStages) & 1, abort, 2, i);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t xs = smem_u32(smem + s * stage_bytes), eh = xs + x_bytes, el = eh + e_bytes;
@@ -113,7 +113,7 @@ tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __nv_bfloat16* __rest
         }
     } else {
         const int quad = warp & 3;
-        bool ok = nblk == 0 || mbar_wait(smem_u32(&ctl->accum), 0, abort);
+        bool ok = nblk == 0 || mbar_wait(smem_u32(&ctl->accum), 0, abort, 3, 0);
         ok = __all_sync(0xffffffffu, ok);
         if (ok && nblk > 0) {
             tc_fence_after();
@@ -143,10 +143,7 @@ tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __nv_bfloat16* __rest
     }
     tc_fence_before();
     __syncthreads();
-    if (ctl->abort) {
-        for (int i = 0; i < 64; ++i) __nanosleep(2000);
-        if (tid == 0) atomicExch(status, MHCLITE_ERR_TIMEOUT);
-    }
+    if (ctl->abort[0]) report_abort(abort, status, 2);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
@@ -167,14 +164,18 @@ tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __nv_bfloat16* __rest
 constexpr int kDTok = 128;                      // tokens per tile (UMMA M)
 constexpr int kDCh = 32;                        // channels per block (UMMA N)
 constexpr int kDBox = 32 * 64;                  // one TMA box: 32 tokens x 32 channels of bf16
-constexpr int kDWSlots = 4;
-constexpr int kDDSlots = 6;
+constexpr int kDWSlots = 6;
+// Data slots: a multiple of 4, so that a slot always serves the same lane quadrant.  (A parity wait is only
+// safe for a waiter that has seen every earlier phase of its barrier; with slots shared between quadrants
+// a warp could take the phase before last for its own.)
+constexpr int kDDSlots = 4;
+static_assert(kDDSlots % 4 == 0, "a data slot must always serve the same lane quadrant");
 
 struct DCtl {
     uint64_t e_full, e_empty, w_full[kDWSlots], w_empty[kDWSlots], d_full[kDDSlots], d_empty[kDDSlots],
         acc_full[2], acc_empty[2];
     uint32_t tmem_base;
-    int abort;
+    int abort[3];
 };
 
 struct DxArgs {
@@ -200,7 +201,7 @@ __device__ __forceinline__ void tc_ld_settle(uint32_t (&r)[8]) {
     asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]) :: "memory");
 }
 
-constexpr int kDThreads = 64 + 256;              // producer warp, MMA warp, 8 epilogue warps
+constexpr int kDThreads = 96 + 256;              // operand producer, MMA issuer, data producer, 8 epilogue warps
 
 template <int N_, bool FUSED, bool ACC>
 __global__ void __launch_bounds__(kDThreads, 1)
@@ -221,14 +222,14 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
     const int64_t it_begin = (int64_t)blockIdx.x * a.per_cta;
     const int64_t it_end = (it_begin + a.per_cta < a.items) ? it_begin + a.per_cta : a.items;
     const int nit = it_end > it_begin ? (int)(it_end - it_begin) : 0;
-    volatile int* abort = &ctl->abort;
+    volatile int* abort = ctl->abort;
 
     if (tid == 0) {
         mbar_init(smem_u32(&ctl->e_full), 1); mbar_init(smem_u32(&ctl->e_empty), 1);
         for (int s = 0; s < kDWSlots; ++s) { mbar_init(smem_u32(&ctl->w_full[s]), 1); mbar_init(smem_u32(&ctl->w_empty[s]), 1); }
         for (int s = 0; s < kDDSlots; ++s) { mbar_init(smem_u32(&ctl->d_full[s]), 1); mbar_init(smem_u32(&ctl->d_empty[s]), 2); }
         for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->acc_full[s]), 1); mbar_init(smem_u32(&ctl->acc_empty[s]), 8); }
-        ctl->abort = 0;
+        ctl->abort[0] = ctl->abort[1] = ctl->abort[2] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -242,7 +243,7 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
     const uint32_t tmem = ctl->tmem_base;
 
     if (warp == 0) {
-        // ---- producer -------------------------------------------------------------------------------
+        // ---- producer of the MMA operands: e tile at tile changes, W' blocks ---------------------------
         if (lane == 0) {
             int64_t cur_tile = -1;
             int ec = 0;
@@ -252,7 +253,7 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
                 const int64_t tile = item / a.ncb;
                 const int cb = (int)(item - tile * a.ncb);
                 if (tile != cur_tile) {
-                    ok = mbar_wait(smem_u32(&ctl->e_empty), (ec & 1) ^ 1, abort);
+                    ok = mbar_wait(smem_u32(&ctl->e_empty), (ec & 1) ^ 1, abort, 1, li);
                     if (!ok) break;
                     mbar_expect_tx(smem_u32(&ctl->e_full), e_bytes);
                     bulk_load(smem_u32(e_s), a.ehi + tile * (int64_t)a.Kp * kDTok, e_bytes, smem_u32(&ctl->e_full));
@@ -261,15 +262,25 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
                 }
                 for (int j = 0; j < N_ && ok; ++j) {
                     const int wi = li * N_ + j, ws = wi % kDWSlots;
-                    ok = mbar_wait(smem_u32(&ctl->w_empty[ws]), ((wi / kDWSlots) & 1) ^ 1, abort);
+                    ok = mbar_wait(smem_u32(&ctl->w_empty[ws]), ((wi / kDWSlots) & 1) ^ 1, abort, 2, wi);
                     if (!ok) break;
                     mbar_expect_tx(smem_u32(&ctl->w_full[ws]), w_bytes);
                     bulk_load(smem_u32(w_s + ws * w_bytes), a.Wb + ((int64_t)j * a.ncb + cb) * a.Kp * kDCh, w_bytes,
                               smem_u32(&ctl->w_full[ws]));
                 }
+            }
+        }
+    } else if (warp == 2) {
+        // ---- producer of the epilogue's data: x, g, du per 32-token quadrant, as far ahead as the ring allows
+        if (lane == 0) {
+            bool ok = true;
+            for (int li = 0; li < nit && ok; ++li) {
+                const int64_t item = it_begin + li;
+                const int64_t tile = item / a.ncb;
+                const int cb = (int)(item - tile * a.ncb);
                 for (int q = 0; q < 4 && ok; ++q) {
                     const int si = li * 4 + q, ds = si % kDDSlots;
-                    ok = mbar_wait(smem_u32(&ctl->d_empty[ds]), ((si / kDDSlots) & 1) ^ 1, abort);
+                    ok = mbar_wait(smem_u32(&ctl->d_empty[ds]), ((si / kDDSlots) & 1) ^ 1, abort, 3, si);
                     if (!ok) break;
                     const uint32_t full = smem_u32(&ctl->d_full[ds]);
                     mbar_expect_tx(full, kDSlot);
@@ -296,17 +307,17 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
                 const int64_t item = it_begin + li;
                 const int64_t tile = item / a.ncb;
                 const int buf = li & 1;
-                ok = mbar_wait(smem_u32(&ctl->acc_empty[buf]), ((li >> 1) & 1) ^ 1, abort);
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[buf]), ((li >> 1) & 1) ^ 1, abort, 4, li);
                 if (!ok) break;
                 if (tile != cur_tile) {
-                    ok = mbar_wait(smem_u32(&ctl->e_full), ec & 1, abort);
+                    ok = mbar_wait(smem_u32(&ctl->e_full), ec & 1, abort, 5, li);
                     if (!ok) break;
                     cur_tile = tile;
                     ++ec;
                 }
                 for (int j = 0; j < N_ && ok; ++j) {
                     const int wi = li * N_ + j, ws = wi % kDWSlots;
-                    ok = mbar_wait(smem_u32(&ctl->w_full[ws]), (wi / kDWSlots) & 1, abort);
+                    ok = mbar_wait(smem_u32(&ctl->w_full[ws]), (wi / kDWSlots) & 1, abort, 6, wi);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t ea = smem_u32(e_s), wa = smem_u32(w_s + ws * w_bytes);
@@ -327,7 +338,7 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
     } else {
         // ---- epilogue: thread = token; the two warps of a lane quadrant take 16 channels each ---------
         const int quad = warp & 3;
-        const int half = (warp - 2) >> 2;
+        const int half = (warp - 3) >> 2;
         const int r = quad * 32 + lane;                         // token within the tile
         float kap = 0.f, hp[N_], hr[N_][N_];
         int64_t cur_tile = -1;
@@ -352,8 +363,8 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
             }
             const int buf = li & 1;
             const int si = li * 4 + quad, ds = si % kDDSlots;
-            ok = mbar_wait(smem_u32(&ctl->acc_full[buf]), (li >> 1) & 1, abort);
-            if (ok) ok = mbar_wait(smem_u32(&ctl->d_full[ds]), (si / kDDSlots) & 1, abort);
+            ok = mbar_wait(smem_u32(&ctl->acc_full[buf]), (li >> 1) & 1, abort, 7, li);
+            if (ok) ok = mbar_wait(smem_u32(&ctl->d_full[ds]), (si / kDDSlots) & 1, abort, 8, si);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -413,10 +424,7 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
     }
     tc_fence_before();
     __syncthreads();
-    if (ctl->abort) {
-        for (int i = 0; i < 64; ++i) __nanosleep(2000);
-        if (tid == 0) atomicExch(a.status, MHCLITE_ERR_TIMEOUT);
-    }
+    if (ctl->abort[0]) report_abort(abort, a.status, 3);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(a.tmem_cols) : "memory");

@@ -23,15 +23,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Waits for the phase with the given parity; gives up (and raises *abort) after kWaitLimit polls or when
-// another role has raised it.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+// Waits for the phase with the given parity; gives up after kWaitLimit polls or when another role of the CTA
+// has given up.  `abort` points at three ints in shared memory: flag, and for the first wait that ran out,
+// a code naming it and a progress index (reported through the status words).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, int where = 0, int index = 0) {
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort) return false;
+        if (abort[0]) return false;
     }
-    *abort = 1;
+    if (abort[0] == 0) { abort[1] = where; abort[2] = index; }
+    abort[0] = 1;
     return false;
+}
+// End of a kernel whose CTA gave up: lets copies in flight land, then records the first report in the status
+// words (status[0] = MHCLITE_ERR_TIMEOUT, [1] = kernel, [2] = wait code, [3] = block, [4] = progress index).
+__device__ __forceinline__ void report_abort(volatile int* abort, int* status, int kernel_id) {
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);
+    if (threadIdx.x == 0 && atomicCAS(status, 0, MHCLITE_ERR_TIMEOUT) == 0) {
+        status[1] = kernel_id; status[2] = abort[1];
+        status[3] = (int)(blockIdx.x | (blockIdx.y << 16)); status[4] = abort[2];
+    }
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
