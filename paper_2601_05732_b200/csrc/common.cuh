@@ -87,6 +87,10 @@ struct TailPlan {
     int g_mt;               // G kernel: 128-row accumulators per CTA (g_mt * Kp <= 512 tensor-memory columns)
     int g_groups, g_splits; // its grid: row groups of 128 * g_mt x token ranges
     int64_t g_tok_per_split;   // multiple of 128
+    // narrow projections: the fused tcgen05 kernel (tail_ftc.cu) when C is a multiple of 64
+    bool ftc;
+    int f_slices, f_splits;  // its grid: 64-channel slices x ranges of 128-token tiles
+    int f_ring;              // dxhat buffers in tensor memory
 };
 TailPlan plan_tail(int n, int C, int64_t T, int N, int sm_count);
 
@@ -101,7 +105,7 @@ struct Workspace {
     float* ssq;      // [kMaxKSplit][T]          partial sums of squares
     void *ehi, *elo; // [T rounded up to 32][Kp] bf16 pair hi + lo = e
     float* Gpart;    // [splits or g_splits][nC][Kp] partial G of each token range
-    void* Wb;        // bf16 W' blocks of the tcgen05 dx kernel (wide projections only)
+    void* Wb;        // bf16 W' blocks of the tcgen05 dx kernels
     void* Wt;        // [2 nq][Kpad] bf16: W' hi rows then lo rows, K-major (tcgen05 projection)
     int* status;     // device status word (0, or a negative mhclite_status raised by a kernel)
     size_t bytes;

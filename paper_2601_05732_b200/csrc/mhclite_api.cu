@@ -42,10 +42,11 @@ Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base) {
     const size_t erows = (size_t)round_up64(T, kEGranule);
     w.ehi = p + off;             off += align256(erows * tp.Kp * 2);
     w.elo = p + off;             off += align256(erows * tp.Kp * 2);
-    const int gparts = tp.supported ? tp.splits : (tp.tc ? tp.g_splits : 0);
+    int gparts = tp.supported ? tp.splits : (tp.tc ? tp.g_splits : 0);
+    if (tp.ftc && tp.f_splits > gparts) gparts = tp.f_splits;
     w.Gpart = (float*)(p + off); off += align256((size_t)gparts * n * C * tp.Kp * sizeof(float));
     w.Wt = p + off;              off += align256((size_t)2 * proj_tc_nq(N) * pp.nchunks * 64 * 2);
-    w.Wb = p + off;              off += align256(tp.tc ? tail_wb_bytes(n, C, tp.Kp) : 0);
+    w.Wb = p + off;              off += align256((tp.tc || tp.ftc) ? tail_wb_bytes(n, C, tp.Kp) : 0);
     w.status = (int*)(p + off);  off += 256;
     w.bytes = off;
     return w;
@@ -130,6 +131,14 @@ static int proj_backward(mhclite_ctx* ctx, int64_t T, int N, const Workspace& w,
                          const mhclite_bf16* x, const mhclite_bf16* g, const mhclite_bf16* du, const float* H_res,
                          const float* H_pre, const float* W, const float* gain, mhclite_bf16* dx, int accumulate_dx,
                          float* dW, float* dgain, int accumulate_params, cudaStream_t s) {
+    if (tp.ftc && launch_tail_ftc(ctx, T, N, tp, x, g, du, w.ehi, w.elo, w.kappa, H_res, H_pre, W, gain, w.Wb, dx,
+                                  accumulate_dx, w.Gpart, w.status, s)) {
+        MHCL_LAUNCH_CHECK(ctx, "tail_ftc");
+        ctx->launches += 1;
+        launch_tail_finish(ctx, N, tp.Kp, tp.f_splits, W, gain, w.Gpart, dW, dgain, accumulate_params, s);
+        MHCL_LAUNCH_CHECK(ctx, "tail_finish");
+        return MHCLITE_OK;
+    }
     if (tp.supported) {
         launch_tail_mma(ctx, T, N, tp, x, g, du, w.ehi, w.elo, w.kappa, H_res, H_pre, W, gain, dx, accumulate_dx,
                         w.Gpart, dW, dgain, accumulate_params, s);

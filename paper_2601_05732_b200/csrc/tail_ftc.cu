@@ -1,0 +1,436 @@
+// Blackwell tensor-core backward tail for narrow projections (n <= 4: at most 32 columns): the projection /
+// RMSNorm backward of paper Eq. (4) fused with the gradient of Eq. (1), one pass over x, g and du.
+//
+//   dxhat[t,m] = sum_c e[t,c] W'[m,c] - x[t,m] kappa_t            (W' = diag(gain) W, e = rstd alpha (.) dz)
+//   dx[t,j,c]  = sum_i H_res[t,i,j] g[t,i,c] + H_pre[t,j] du[t,c] + dxhat[t,j*C+c]
+//   G[m,c]     = sum_t x[t,m] e[t,c]                              (dW = gain (.) G, dgain = sum_c W G)
+//
+// A CTA owns a slice of 64 channels of all n streams and walks over a range of 128-token tiles.
+//   * x, g and du arrive by TMA (128-byte swizzle) per 32-token quadrant into four slots, one per lane
+//     quadrant of the tensor memory; the tiled e buffers (hi, lo) of a tile arrive as two bulk copies; the
+//     CTA's rows of W' stay in shared memory.
+//   * One thread issues tcgen05.mma: dxhat of a tile half (M = 128 tokens, N = n x 32 channels, K = Kp) into a
+//     ring of tensor-memory buffers, and per arrived quadrant G += x^T e (M = 128 rows of the slice, N = Kp,
+//     K = 32 tokens, x as the MN-major operand straight from its slot, e as hi + lo) into accumulators that
+//     stay in tensor memory over the whole token range.
+//   * Eight epilogue warps (thread = token, two warps per quadrant) combine dxhat with x, g, du and the
+//     token's H_res, H_pre and kappa, write dx over the x boxes of the slot, and one thread per quadrant
+//     sends the boxes to global memory with a TMA store before it hands the slot back.
+//   * At the end the G accumulators go to this token range's partial (no atomics).
+// Every mbarrier wait is bounded; on a time-out the CTA raises its abort flag, records MHCLITE_ERR_TIMEOUT in
+// the status word, lets copies in flight land, frees its tensor memory and returns.
+#include "common.cuh"
+#include "kernels.h"
+#include "mma.cuh"
+#include "tc.cuh"
+
+namespace mhcl {
+
+constexpr int kFTok = 128;                      // tokens per tile (UMMA M)
+constexpr int kFCs = 64;                        // channels per slice = one 128-byte swizzle row
+constexpr int kFBox = 32 * 128;                 // one TMA box: 32 tokens x 64 channels of bf16
+constexpr int kFEpiWarps = 8;
+constexpr int kFThreads = 96 + 32 * kFEpiWarps; // operand producer, MMA issuer, data producer, epilogue
+constexpr int kFMaxRing = 3;
+
+struct FCtl {
+    uint64_t w_full, e_full[2], e_empty[2], d_full[4], d_empty[4], g_done[4], q_done[4], acc_full[kFMaxRing],
+        acc_empty[kFMaxRing], g_final;
+    uint32_t tmem_base;
+    int abort[3];
+};
+
+struct FArgs {
+    int64_t T;
+    int C, Kp;
+    int ntiles, splits;             // 128-token tiles in all, token ranges (grid y)
+    int ring, tmem_cols;            // dxhat buffers in tensor memory, columns allocated
+    const __nv_bfloat16 *ehi, *elo; // tiled (see e_tiled_index)
+    const __nv_bfloat16* Wf;        // [slice][half][Kp/8][n][32][8]
+    const float *kappa, *H_res, *H_pre;
+    float* Gpart;                   // [splits][nC][Kp]
+    int* status;
+};
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void ftc_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+}
+__device__ __forceinline__ void ftc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Ties the registers of an earlier tcgen05.ld to a point after the wait, so that no use is scheduled before it.
+__device__ __forceinline__ void ftc_settle(uint32_t (&r)[8]) {
+    asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]) :: "memory");
+}
+
+// MODE 0: dx = dxhat (x only);  1: fused with H_res^T g + H_pre du;  2: dx += dxhat (x and the old dx).
+template <int N_, int MODE>
+__global__ void __launch_bounds__(kFThreads, 1)
+tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmg,
+           const __grid_constant__ CUtensorMap tmdu, const __grid_constant__ CUtensorMap tmdx, const FArgs a) {
+    constexpr int kBoxes = MODE == 1 ? 2 * N_ + 1 : (MODE == 2 ? 2 * N_ : N_);
+    constexpr int kSlot = kBoxes * kFBox;
+    constexpr int kNA = (N_ + 1) / 2;                          // G accumulators: 128 rows = two streams' 64 channels
+    constexpr int kDW = N_ * 32;                               // tensor-memory columns of one dxhat buffer
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int e_bytes = a.Kp * kFTok * 2;                      // one of hi / lo of a tile; a multiple of 4096
+    const int w_bytes = a.Kp * N_ * kFCs * 2;
+    unsigned char* slots = smem;
+    unsigned char* e_s = slots + 4 * kSlot;                    // [2 buffers][hi | lo]
+    unsigned char* w_s = e_s + 4 * e_bytes;
+    FCtl* ctl = reinterpret_cast<FCtl*>(w_s + ((w_bytes + 1023) & ~1023));
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int c0 = blockIdx.x * kFCs;
+    const int tile_begin = (int)(((int64_t)a.ntiles * blockIdx.y) / a.splits);
+    const int tile_end = (int)(((int64_t)a.ntiles * (blockIdx.y + 1)) / a.splits);
+    const int nt = tile_end - tile_begin;
+    const int64_t t0 = (int64_t)tile_begin * kFTok;
+    volatile int* abort = ctl->abort;
+
+    if (tid == 0) {
+        mbar_init(smem_u32(&ctl->w_full), 1);
+        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->e_full[s]), 1); mbar_init(smem_u32(&ctl->e_empty[s]), 1); }
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(smem_u32(&ctl->d_full[s]), 1); mbar_init(smem_u32(&ctl->d_empty[s]), 1);
+            mbar_init(smem_u32(&ctl->g_done[s]), 1); mbar_init(smem_u32(&ctl->q_done[s]), 2);
+        }
+        for (int s = 0; s < kFMaxRing; ++s) { mbar_init(smem_u32(&ctl->acc_full[s]), 1); mbar_init(smem_u32(&ctl->acc_empty[s]), kFEpiWarps); }
+        mbar_init(smem_u32(&ctl->g_final), 1);
+        ctl->abort[0] = ctl->abort[1] = ctl->abort[2] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(a.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+    const uint32_t tmem_g = tmem;                              // kNA accumulators of Kp columns
+    const uint32_t tmem_d = tmem + kNA * a.Kp;                 // ring of dxhat buffers
+
+    if (warp == 0) {
+        // ---- producer of the MMA operands: W' rows of the slice once, then the e tiles ------------------
+        if (lane == 0 && nt > 0) {
+            mbar_expect_tx(smem_u32(&ctl->w_full), w_bytes);
+            bulk_load(smem_u32(w_s), a.Wf + (int64_t)blockIdx.x * (w_bytes / 2), w_bytes, smem_u32(&ctl->w_full));
+            for (int ti = 0; ti < nt; ++ti) {
+                const int buf = ti & 1;
+                if (!mbar_wait(smem_u32(&ctl->e_empty[buf]), ((ti >> 1) & 1) ^ 1, abort, 1, ti)) break;
+                const uint32_t full = smem_u32(&ctl->e_full[buf]);
+                mbar_expect_tx(full, 2 * e_bytes);
+                const int64_t off = (int64_t)(tile_begin + ti) * a.Kp * kFTok;       // elements
+                bulk_load(smem_u32(e_s + buf * 2 * e_bytes), a.ehi + off, e_bytes, full);
+                bulk_load(smem_u32(e_s + buf * 2 * e_bytes + e_bytes), a.elo + off, e_bytes, full);
+            }
+        }
+    } else if (warp == 2) {
+        // ---- producer of the data: x (and g, du, or the old dx) per 32-token quadrant --------------------
+        if (lane == 0) {
+            bool ok = true;
+            for (int ti = 0; ti < nt && ok; ++ti) {
+                for (int q = 0; q < 4 && ok; ++q) {
+                    ok = mbar_wait(smem_u32(&ctl->d_empty[q]), (ti & 1) ^ 1, abort, 2, ti * 4 + q);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&ctl->d_full[q]);
+                    mbar_expect_tx(full, kSlot);
+                    const uint32_t dst = smem_u32(slots + q * kSlot);
+                    const int row = (int)(t0 + (int64_t)ti * kFTok + q * 32);
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) {
+                        tma_load_2d(dst + j * kFBox, &tmx, full, j * a.C + c0, row);
+                        if (MODE != 0) tma_load_2d(dst + (N_ + j) * kFBox, &tmg, full, j * a.C + c0, row);
+                    }
+                    if (MODE == 1) tma_load_2d(dst + 2 * N_ * kFBox, &tmdu, full, c0, row);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer ------------------------------------------------------------------------------
+        if (lane == 0 && nt > 0) {
+            const uint32_t idesc_d = umma_idesc_mn(128, kDW, 0, 0);
+            const uint32_t idesc_g = umma_idesc_mn(128, a.Kp, 1, 1);
+            const int ksteps = a.Kp >> 4;
+            const uint32_t w_half = (uint32_t)(a.Kp >> 3) * (kDW * 16);          // bytes of one channel half of W'
+            bool ok = mbar_wait(smem_u32(&ctl->w_full), 0, abort, 3, 0);
+            for (int ti = 0; ti < nt && ok; ++ti) {
+                const int buf = ti & 1;
+                ok = mbar_wait(smem_u32(&ctl->e_full[buf]), (ti >> 1) & 1, abort, 4, ti);
+                if (!ok) break;
+                const uint32_t eh = smem_u32(e_s + buf * 2 * e_bytes), el = eh + e_bytes;
+                for (int half = 0; half < 2 && ok; ++half) {
+                    const int u = 2 * ti + half, rr = u % a.ring;
+                    ok = mbar_wait(smem_u32(&ctl->acc_empty[rr]), ((u / a.ring) & 1) ^ 1, abort, 5, u);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t wa = smem_u32(w_s) + half * w_half;
+                    for (int ks = 0; ks < ksteps; ++ks) {
+                        // A: tokens x columns, K-major, no swizzle: column groups 2 KB apart, 8-token groups 128 B apart
+                        // B: channels x columns, K-major, no swizzle: column groups kDW * 16 B apart, 8-channel groups 128 B apart
+                        tc_mma(tmem_d + rr * kDW, smem_desc(eh + ks * 4096, 2048, 128, 0),
+                               smem_desc(wa + ks * 2 * (kDW * 16), kDW * 16, 128, 0), idesc_d, ks > 0 ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&ctl->acc_full[rr]));
+                }
+                for (int q = 0; q < 4 && ok; ++q) {
+                    ok = mbar_wait(smem_u32(&ctl->d_full[q]), ti & 1, abort, 6, ti * 4 + q);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t xs = smem_u32(slots + q * kSlot);
+#pragma unroll
+                    for (int ks = 0; ks < 2; ++ks) {
+                        // B: columns = N (8-column groups 2 KB apart), tokens = K (8-token groups 128 B apart)
+                        const uint32_t eo = (uint32_t)(q * 32 + ks * 16) * 16;
+                        const uint64_t bh = smem_desc(eh + eo, 128, 2048, 0), bl = smem_desc(el + eo, 128, 2048, 0);
+#pragma unroll
+                        for (int ac = 0; ac < kNA; ++ac) {
+                            // A: 128 rows = the 64 channels of two streams (boxes 4 KB apart), 8-token groups 1 KB apart
+                            const uint64_t ad = smem_desc(xs + ac * 2 * kFBox + ks * 2048, kFBox, 1024, 2);
+                            tc_mma(tmem_g + ac * a.Kp, ad, bh, idesc_g, (ti > 0 || q > 0 || ks > 0) ? 1u : 0u);
+                            tc_mma(tmem_g + ac * a.Kp, ad, bl, idesc_g, 1u);
+                        }
+                    }
+                    tc_commit(smem_u32(&ctl->g_done[q]));
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&ctl->e_empty[buf]));
+            }
+            if (ok) tc_commit(smem_u32(&ctl->g_final));
+        }
+    } else {
+        // ---- epilogue: thread = token; the two warps of a lane quadrant take 16 channels of each half ----
+        const int quad = warp & 3;
+        const int hw = (warp - 3) >> 2;
+        unsigned char* slot = slots + quad * kSlot;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        float kap = 0.f, hp[N_], hr[N_][N_];
+        bool ok = true;
+        for (int ti = 0; ti < nt; ++ti) {
+            const int64_t row0 = t0 + (int64_t)ti * kFTok + quad * 32;
+            const int64_t t = row0 + lane;
+            const bool live = t < a.T;
+            kap = live ? __ldg(a.kappa + t) : 0.f;
+            if (MODE == 1) {
+#pragma unroll
+                for (int j = 0; j < N_; ++j) hp[j] = live ? __ldg(a.H_pre + t * N_ + j) : 0.f;
+#pragma unroll
+                for (int i = 0; i < N_; ++i)
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) hr[i][j] = live ? __ldg(a.H_res + t * N_ * N_ + i * N_ + j) : 0.f;
+            }
+            ok = mbar_wait(smem_u32(&ctl->d_full[quad]), ti & 1, abort, 7, ti);
+            if (ok) ok = mbar_wait(smem_u32(&ctl->g_done[quad]), ti & 1, abort, 8, ti);
+            for (int half = 0; half < 2; ++half) {
+                const int u = 2 * ti + half, rr = u % a.ring;
+                if (ok) ok = mbar_wait(smem_u32(&ctl->acc_full[rr]), (u / a.ring) & 1, abort, 9, u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t tbase = tmem_d + lane_base + rr * kDW;
+#pragma unroll
+                for (int pp = 0; pp < 2; ++pp) {
+                    const int pcl = hw * 2 + pp;                       // 8-channel group within the half
+                    const int pc = half * 4 + pcl;                     // 16-byte piece within the 128-byte row
+                    const int po = lane * 128 + ((pc ^ (lane & 7)) << 4);
+                    uint32_t acc[N_][8];
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) ftc_ld8(tbase + j * 32 + pcl * 8, acc[j]);
+                    float gf[MODE == 1 ? N_ : 1][8], df[8];
+                    if (MODE == 1) {
+#pragma unroll
+                        for (int i = 0; i < N_; ++i) unpack8(*reinterpret_cast<const uint4*>(slot + (N_ + i) * kFBox + po), gf[i]);
+                        unpack8(*reinterpret_cast<const uint4*>(slot + 2 * N_ * kFBox + po), df);
+                    }
+                    ftc_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) ftc_settle(acc[j]);
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) {
+                        float xf[8], o[8];
+                        uint4* xp = reinterpret_cast<uint4*>(slot + j * kFBox + po);
+                        unpack8(*xp, xf);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) o[e] = fmaf(-xf[e], kap, __uint_as_float(acc[j][e]));
+                        if (MODE == 1) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) o[e] = fmaf(hp[j], df[e], o[e]);
+#pragma unroll
+                            for (int i = 0; i < N_; ++i)
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) o[e] = fmaf(hr[i][j], gf[i][e], o[e]);
+                        }
+                        if (MODE == 2) {
+                            float old[8];
+                            unpack8(*reinterpret_cast<const uint4*>(slot + (N_ + j) * kFBox + po), old);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) o[e] += old[e];
+                        }
+                        *xp = pack8(o);                                // dx takes the place of x in the slot
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[rr]));
+            }
+            if (!ok) break;
+            // the slot's x boxes now hold dx: make the writes visible to the TMA unit, then one thread stores them
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&ctl->q_done[quad]));
+                if (hw == 0 && mbar_wait(smem_u32(&ctl->q_done[quad]), ti & 1, abort, 10, ti)) {
+                    if (row0 < a.T) {
+#pragma unroll
+                        for (int j = 0; j < N_; ++j) tma_store_2d(&tmdx, smem_u32(slot + j * kFBox), j * a.C + c0, (int)row0);
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    }
+                    mbar_arrive(smem_u32(&ctl->d_empty[quad]));
+                }
+            }
+            __syncwarp();
+        }
+        if (hw == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        // ---- G of this token range -> its partial -----------------------------------------------------
+        if (nt > 0) {
+            if (ok) ok = mbar_wait(smem_u32(&ctl->g_final), 0, abort, 11, 0);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after();
+                float* Gp = a.Gpart + (int64_t)blockIdx.y * (N_ * a.C) * a.Kp;
+                for (int ac = hw; ac < kNA; ac += 2) {
+                    const int j = 2 * ac + (quad >> 1);
+                    const int ch = c0 + (quad & 1) * 32 + lane;
+                    for (int cc = 0; cc < a.Kp; cc += 16) {
+                        float v[16];
+                        tc_ld16(tmem_g + lane_base + ac * a.Kp + cc, v);
+                        if (j < N_) {
+                            float* rowp = Gp + ((int64_t)j * a.C + ch) * a.Kp + cc;
+#pragma unroll
+                            for (int e = 0; e < 16; e += 4)
+                                *reinterpret_cast<float4*>(rowp + e) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (ctl->abort[0]) report_abort(abort, a.status, 4);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(a.tmem_cols) : "memory");
+    }
+}
+
+// W' = diag(gain) W in bf16 as the B operand of tail_ftc_k: per slice of 64 channels and per half of it a
+// block [Kp/8 column groups][n streams][32 channels][8 columns]; zero beyond the N columns.
+__global__ void __launch_bounds__(256) pack_wf_k(int n, int C, int N, int Kp, const float* __restrict__ W,
+                                                 const float* __restrict__ gain, __nv_bfloat16* __restrict__ Wf) {
+    const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int64_t total = (int64_t)n * C * Kp;
+    if (idx >= total) return;
+    const int c8 = (int)(idx & 7), chl = (int)((idx >> 3) & 31);
+    int64_t rest = idx >> 8;
+    const int j = (int)(rest % n); rest /= n;
+    const int cg = (int)(rest % (Kp >> 3)); rest /= (Kp >> 3);
+    const int half = (int)(rest & 1);
+    const int slice = (int)(rest >> 1);
+    const int ch = slice * kFCs + half * 32 + chl, col = cg * 8 + c8;
+    float w = 0.f;
+    if (col < N) {
+        const int m = j * C + ch;
+        w = __ldg(W + (int64_t)m * N + col) * __ldg(gain + m);
+    }
+    Wf[idx] = __float2bfloat16_rn(w);
+}
+
+// ---- host side -------------------------------------------------------------------------------------
+static int ftc_smem_bytes(int n, int Kp, int mode) {
+    const int boxes = mode == 1 ? 2 * n + 1 : (mode == 2 ? 2 * n : n);
+    const int w_bytes = Kp * n * kFCs * 2;
+    return 4 * boxes * kFBox + 4 * (Kp * kFTok * 2) + ((w_bytes + 1023) & ~1023) + (int)sizeof(FCtl) + 1024;
+}
+
+// Fills the plan's fields of this kernel: usable when the slices are whole (C a multiple of 64), the G
+// accumulators and two dxhat buffers fit the 512 columns of tensor memory, and the slots fit shared memory.
+void plan_tail_ftc(int n, int C, int64_t T, int sm_count, TailPlan* p) {
+    const int na = (n + 1) / 2;
+    p->ftc = p->supported && (C % kFCs) == 0 && na * p->Kp + 2 * n * 32 <= 512 && ftc_smem_bytes(n, p->Kp, 1) <= 227 * 1024;
+    p->f_slices = C / kFCs;
+    const int64_t ntiles = (T + kFTok - 1) / kFTok;
+    int64_t splits = p->f_slices > 0 ? sm_count / p->f_slices : 1;
+    if (splits > ntiles) splits = ntiles;
+    if (splits < 1) splits = 1;
+    p->f_splits = (int)splits;
+    int ring = (512 - na * p->Kp) / (n * 32);
+    p->f_ring = ring > kFMaxRing ? kFMaxRing : ring;
+}
+
+template <int N_>
+static void launch_ftc_t(dim3 grid, int smem, const CUtensorMap& tmx, const CUtensorMap& tmg, const CUtensorMap& tmdu,
+                         const CUtensorMap& tmdx, const FArgs& a, int mode, cudaStream_t s) {
+#define MHCL_FTC(M)                                                                                      \
+    do {                                                                                                 \
+        cudaFuncSetAttribute(tail_ftc_k<N_, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);      \
+        tail_ftc_k<N_, M><<<grid, kFThreads, smem, s>>>(tmx, tmg, tmdu, tmdx, a);                         \
+    } while (0)
+    if (mode == 1) MHCL_FTC(1);
+    else if (mode == 2) MHCL_FTC(2);
+    else MHCL_FTC(0);
+#undef MHCL_FTC
+}
+
+// dx and the G partials [f_splits][nC][Kp] in one pass; packs W' first.  False (nothing launched) when no
+// tensor map could be made.
+bool launch_tail_ftc(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, const void* x, const void* g,
+                     const void* du, const void* ehi, const void* elo, const float* kappa, const float* H_res,
+                     const float* H_pre, const float* W, const float* gain, void* Wf, void* dx, int acc_dx,
+                     float* Gpart, int* status, cudaStream_t s) {
+    const int n = c->n, C = c->C, nC = n * C;
+    if (n > 4 || !p.ftc) return false;
+    const int mode = g ? 1 : (acc_dx ? 2 : 0);
+    CUtensorMap tmx, tmg, tmdu, tmdx;
+    if (!make_tensor_map_2d(&tmx, x, (uint64_t)nC, (uint64_t)T, (uint64_t)nC, kFCs, 32, 128)) return false;
+    if (!make_tensor_map_2d(&tmdx, dx, (uint64_t)nC, (uint64_t)T, (uint64_t)nC, kFCs, 32, 128)) return false;
+    tmg = mode == 2 ? tmdx : tmx; tmdu = tmx;
+    if (mode == 1) {
+        if (!make_tensor_map_2d(&tmg, g, (uint64_t)nC, (uint64_t)T, (uint64_t)nC, kFCs, 32, 128)) return false;
+        if (!make_tensor_map_2d(&tmdu, du, (uint64_t)C, (uint64_t)T, (uint64_t)C, kFCs, 32, 128)) return false;
+    }
+    FArgs a;
+    a.T = T; a.C = C; a.Kp = p.Kp;
+    a.ntiles = (int)((T + kFTok - 1) / kFTok); a.splits = p.f_splits; a.ring = p.f_ring;
+    const int smem = ftc_smem_bytes(n, p.Kp, mode);
+    const int cols = ((n + 1) / 2) * p.Kp + a.ring * n * 32;
+    a.tmem_cols = 32;
+    while (a.tmem_cols < cols) a.tmem_cols *= 2;
+    if (2 * smem <= 227 * 1024 && a.tmem_cols > 256) {        // two CTAs may share an SM: halve the claim
+        a.ring = 2;
+        a.tmem_cols = 256;
+        if (((n + 1) / 2) * p.Kp + 2 * n * 32 > 256) return false;
+    }
+    a.ehi = (const __nv_bfloat16*)ehi; a.elo = (const __nv_bfloat16*)elo; a.Wf = (const __nv_bfloat16*)Wf;
+    a.kappa = kappa; a.H_res = H_res; a.H_pre = H_pre; a.Gpart = Gpart; a.status = status;
+    c->launches += 2;
+    const int64_t total = (int64_t)nC * p.Kp;
+    pack_wf_k<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(n, C, N, p.Kp, W, gain, (__nv_bfloat16*)Wf);
+    KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_MMA, s);
+    dim3 grid(p.f_slices, p.f_splits);
+    switch (n) {
+        case 2: launch_ftc_t<2>(grid, smem, tmx, tmg, tmdu, tmdx, a, mode, s); break;
+        case 3: launch_ftc_t<3>(grid, smem, tmx, tmg, tmdu, tmdx, a, mode, s); break;
+        default: launch_ftc_t<4>(grid, smem, tmx, tmg, tmdu, tmdx, a, mode, s); break;
+    }
+    return true;
+}
+
+}  // namespace mhcl

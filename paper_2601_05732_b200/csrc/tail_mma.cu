@@ -367,6 +367,7 @@ TailPlan plan_tail(int n, int C, int64_t T, int N, int sm_count) {
     if (p.g_tok_per_split < kEGranule) p.g_tok_per_split = kEGranule;
     p.g_splits = (int)((T + p.g_tok_per_split - 1) / p.g_tok_per_split);
     if (p.g_splits < 1) p.g_splits = 1;
+    plan_tail_ftc(n, C, T, sm_count, &p);
     return p;
 }
 
