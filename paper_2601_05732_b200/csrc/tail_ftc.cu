@@ -11,11 +11,12 @@
 //     CTA's rows of W' stay in shared memory.
 //   * One thread issues tcgen05.mma: dxhat of a tile half (M = 128 tokens, N = n x 32 channels, K = Kp) into a
 //     ring of tensor-memory buffers, and per arrived quadrant G += x^T e (M = 128 rows of the slice, N = Kp,
-//     K = 32 tokens, x as the MN-major operand straight from its slot, e as hi + lo) into accumulators that
-//     stay in tensor memory over the whole token range.
+//     K = 32 tokens, x as the MN-major operand straight from its slot, e as hi | lo side by side in N) into
+//     accumulators that stay in tensor memory over the whole token range.
 //   * Eight epilogue warps (thread = token, two warps per quadrant) combine dxhat with x, g, du and the
-//     token's H_res, H_pre and kappa, write dx over the x boxes of the slot, and one thread per quadrant
-//     sends the boxes to global memory with a TMA store before it hands the slot back.
+//     token's H_res, H_pre and kappa, write dx over the g boxes of the slot (a thread has read all of g at
+//     its position before it writes there), and one thread per quadrant sends the boxes to global memory
+//     with a TMA store before it hands the slot back.
 //   * At the end the G accumulators go to this token range's partial (no atomics).
 // Every mbarrier wait is bounded; on a time-out the CTA raises its abort flag, records MHCLITE_ERR_TIMEOUT in
 // the status word, lets copies in flight land, frees its tensor memory and returns.
@@ -74,6 +75,7 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
            const __grid_constant__ CUtensorMap tmdu, const __grid_constant__ CUtensorMap tmdx, const FArgs a) {
     constexpr int kBoxes = MODE == 1 ? 2 * N_ + 1 : (MODE == 2 ? 2 * N_ : N_);
     constexpr int kSlot = kBoxes * kFBox;
+    constexpr int kOut = MODE == 0 ? 0 : N_;                   // first of the boxes that dx is written over
     constexpr int kNA = (N_ + 1) / 2;                          // G accumulators: 128 rows = two streams' 64 channels
     constexpr int kDW = N_ * 32;                               // tensor-memory columns of one dxhat buffer
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -113,8 +115,8 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = ctl->tmem_base;
-    const uint32_t tmem_g = tmem;                              // kNA accumulators of Kp columns
-    const uint32_t tmem_d = tmem + kNA * a.Kp;                 // ring of dxhat buffers
+    const uint32_t tmem_g = tmem;                              // kNA accumulators of 2 Kp columns (hi | lo parts)
+    const uint32_t tmem_d = tmem + kNA * 2 * a.Kp;             // ring of dxhat buffers
 
     if (warp == 0) {
         // ---- producer of the MMA operands: W' rows of the slice once, then the e tiles ------------------
@@ -156,15 +158,16 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
         // ---- MMA issuer ------------------------------------------------------------------------------
         if (lane == 0 && nt > 0) {
             const uint32_t idesc_d = umma_idesc_mn(128, kDW, 0, 0);
-            const uint32_t idesc_g = umma_idesc_mn(128, a.Kp, 1, 1);
+            const uint32_t idesc_g = umma_idesc_mn(128, 2 * a.Kp, 1, 1);
             const int ksteps = a.Kp >> 4;
             const uint32_t w_half = (uint32_t)(a.Kp >> 3) * (kDW * 16);          // bytes of one channel half of W'
             bool ok = mbar_wait(smem_u32(&ctl->w_full), 0, abort, 3, 0);
+            bool g_started = false;
             for (int ti = 0; ti < nt && ok; ++ti) {
                 const int buf = ti & 1;
                 ok = mbar_wait(smem_u32(&ctl->e_full[buf]), (ti >> 1) & 1, abort, 4, ti);
                 if (!ok) break;
-                const uint32_t eh = smem_u32(e_s + buf * 2 * e_bytes), el = eh + e_bytes;
+                const uint32_t eh = smem_u32(e_s + buf * 2 * e_bytes);        // e_lo follows e_hi
                 for (int half = 0; half < 2 && ok; ++half) {
                     const int u = 2 * ti + half, rr = u % a.ring;
                     ok = mbar_wait(smem_u32(&ctl->acc_empty[rr]), ((u / a.ring) & 1) ^ 1, abort, 5, u);
@@ -179,25 +182,35 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                     }
                     tc_commit(smem_u32(&ctl->acc_full[rr]));
                 }
-                for (int q = 0; q < 4 && ok; ++q) {
-                    ok = mbar_wait(smem_u32(&ctl->d_full[q]), ti & 1, abort, 6, ti * 4 + q);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t xs = smem_u32(slots + q * kSlot);
-#pragma unroll
-                    for (int ks = 0; ks < 2; ++ks) {
-                        // B: columns = N (8-column groups 2 KB apart), tokens = K (8-token groups 128 B apart)
-                        const uint32_t eo = (uint32_t)(q * 32 + ks * 16) * 16;
-                        const uint64_t bh = smem_desc(eh + eo, 128, 2048, 0), bl = smem_desc(el + eo, 128, 2048, 0);
-#pragma unroll
-                        for (int ac = 0; ac < kNA; ++ac) {
-                            // A: 128 rows = the 64 channels of two streams (boxes 4 KB apart), 8-token groups 1 KB apart
-                            const uint64_t ad = smem_desc(xs + ac * 2 * kFBox + ks * 2048, kFBox, 1024, 2);
-                            tc_mma(tmem_g + ac * a.Kp, ad, bh, idesc_g, (ti > 0 || q > 0 || ks > 0) ? 1u : 0u);
-                            tc_mma(tmem_g + ac * a.Kp, ad, bl, idesc_g, 1u);
-                        }
+                // G += x^T e per quadrant, in the order in which the quadrants' data arrive
+                uint32_t pending = 0xFu;
+                for (uint32_t polls = 0; pending && ok; ++polls) {
+                    if (polls > kWaitLimit || abort[0]) {
+                        if (abort[0] == 0) { abort[1] = 6; abort[2] = ti; }
+                        abort[0] = 1;
+                        ok = false;
+                        break;
                     }
-                    tc_commit(smem_u32(&ctl->g_done[q]));
+                    for (int q = 0; q < 4; ++q) {
+                        if (!(pending & (1u << q)) || !mbar_try_wait(smem_u32(&ctl->d_full[q]), ti & 1)) continue;
+                        pending &= ~(1u << q);
+                        tc_fence_after();
+                        const uint32_t xs = smem_u32(slots + q * kSlot);
+#pragma unroll
+                        for (int ks = 0; ks < 2; ++ks) {
+                            // B: columns of e_hi then of e_lo = N (8-column groups 2 KB apart), tokens = K (8-token
+                            // groups 128 B apart)
+                            const uint64_t bd = smem_desc(eh + (uint32_t)(q * 32 + ks * 16) * 16, 128, 2048, 0);
+#pragma unroll
+                            for (int ac = 0; ac < kNA; ++ac) {
+                                // A: 128 rows = the 64 channels of two streams (boxes 4 KB apart), 8-token groups 1 KB apart
+                                const uint64_t ad = smem_desc(xs + ac * 2 * kFBox + ks * 2048, kFBox, 1024, 2);
+                                tc_mma(tmem_g + ac * 2 * a.Kp, ad, bd, idesc_g, g_started ? 1u : 0u);
+                            }
+                            g_started = true;
+                        }
+                        tc_commit(smem_u32(&ctl->g_done[q]));
+                    }
                 }
                 if (!ok) break;
                 tc_commit(smem_u32(&ctl->e_empty[buf]));
@@ -226,7 +239,8 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                     for (int j = 0; j < N_; ++j) hr[i][j] = live ? __ldg(a.H_res + t * N_ * N_ + i * N_ + j) : 0.f;
             }
             ok = mbar_wait(smem_u32(&ctl->d_full[quad]), ti & 1, abort, 7, ti);
-            if (ok) ok = mbar_wait(smem_u32(&ctl->g_done[quad]), ti & 1, abort, 8, ti);
+            // MODE 0 writes dx over x itself: the G MMAs must have read the boxes
+            if (MODE == 0 && ok) ok = mbar_wait(smem_u32(&ctl->g_done[quad]), ti & 1, abort, 8, ti);
             for (int half = 0; half < 2; ++half) {
                 const int u = 2 * ti + half, rr = u % a.ring;
                 if (ok) ok = mbar_wait(smem_u32(&ctl->acc_full[rr]), (u / a.ring) & 1, abort, 9, u);
@@ -254,8 +268,7 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
 #pragma unroll
                     for (int j = 0; j < N_; ++j) {
                         float xf[8], o[8];
-                        uint4* xp = reinterpret_cast<uint4*>(slot + j * kFBox + po);
-                        unpack8(*xp, xf);
+                        unpack8(*reinterpret_cast<const uint4*>(slot + j * kFBox + po), xf);
 #pragma unroll
                         for (int e = 0; e < 8; ++e) o[e] = fmaf(-xf[e], kap, __uint_as_float(acc[j][e]));
                         if (MODE == 1) {
@@ -272,7 +285,8 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
 #pragma unroll
                             for (int e = 0; e < 8; ++e) o[e] += old[e];
                         }
-                        *xp = pack8(o);                                // dx takes the place of x in the slot
+                        // dx takes the place of g (of the old dx; of x itself in MODE 0) in the slot
+                        *reinterpret_cast<uint4*>(slot + (kOut + j) * kFBox + po) = pack8(o);
                     }
                 }
                 tc_fence_before();
@@ -280,7 +294,7 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[rr]));
             }
             if (!ok) break;
-            // the slot's x boxes now hold dx: make the writes visible to the TMA unit, then one thread stores them
+            // the slot now holds dx: make the writes visible to the TMA unit, then one thread stores the boxes
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) {
@@ -288,11 +302,14 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                 if (hw == 0 && mbar_wait(smem_u32(&ctl->q_done[quad]), ti & 1, abort, 10, ti)) {
                     if (row0 < a.T) {
 #pragma unroll
-                        for (int j = 0; j < N_; ++j) tma_store_2d(&tmdx, smem_u32(slot + j * kFBox), j * a.C + c0, (int)row0);
+                        for (int j = 0; j < N_; ++j)
+                            tma_store_2d(&tmdx, smem_u32(slot + (kOut + j) * kFBox), j * a.C + c0, (int)row0);
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     }
-                    mbar_arrive(smem_u32(&ctl->d_empty[quad]));
+                    // the slot goes back once the G MMAs have read its x boxes (long done by now)
+                    if (MODE == 0 || mbar_wait(smem_u32(&ctl->g_done[quad]), ti & 1, abort, 8, ti))
+                        mbar_arrive(smem_u32(&ctl->d_empty[quad]));
                 }
             }
             __syncwarp();
@@ -309,8 +326,11 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                     const int j = 2 * ac + (quad >> 1);
                     const int ch = c0 + (quad & 1) * 32 + lane;
                     for (int cc = 0; cc < a.Kp; cc += 16) {
-                        float v[16];
-                        tc_ld16(tmem_g + lane_base + ac * a.Kp + cc, v);
+                        float v[16], lo[16];
+                        tc_ld16(tmem_g + lane_base + ac * 2 * a.Kp + cc, v);
+                        tc_ld16(tmem_g + lane_base + ac * 2 * a.Kp + a.Kp + cc, lo);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) v[e] += lo[e];
                         if (j < N_) {
                             float* rowp = Gp + ((int64_t)j * a.C + ch) * a.Kp + cc;
 #pragma unroll
@@ -361,17 +381,18 @@ static int ftc_smem_bytes(int n, int Kp, int mode) {
 }
 
 // Fills the plan's fields of this kernel: usable when the slices are whole (C a multiple of 64), the G
-// accumulators and two dxhat buffers fit the 512 columns of tensor memory, and the slots fit shared memory.
+// accumulators (hi | lo parts) and two dxhat buffers fit the 512 columns of tensor memory, and the slots fit
+// shared memory.
 void plan_tail_ftc(int n, int C, int64_t T, int sm_count, TailPlan* p) {
     const int na = (n + 1) / 2;
-    p->ftc = p->supported && (C % kFCs) == 0 && na * p->Kp + 2 * n * 32 <= 512 && ftc_smem_bytes(n, p->Kp, 1) <= 227 * 1024;
+    p->ftc = p->supported && (C % kFCs) == 0 && na * 2 * p->Kp + 2 * n * 32 <= 512 && ftc_smem_bytes(n, p->Kp, 1) <= 227 * 1024;
     p->f_slices = C / kFCs;
     const int64_t ntiles = (T + kFTok - 1) / kFTok;
     int64_t splits = p->f_slices > 0 ? sm_count / p->f_slices : 1;
     if (splits > ntiles) splits = ntiles;
     if (splits < 1) splits = 1;
     p->f_splits = (int)splits;
-    int ring = (512 - na * p->Kp) / (n * 32);
+    int ring = (512 - na * 2 * p->Kp) / (n * 32);
     p->f_ring = ring > kFMaxRing ? kFMaxRing : ring;
 }
 
@@ -410,13 +431,13 @@ bool launch_tail_ftc(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, 
     a.T = T; a.C = C; a.Kp = p.Kp;
     a.ntiles = (int)((T + kFTok - 1) / kFTok); a.splits = p.f_splits; a.ring = p.f_ring;
     const int smem = ftc_smem_bytes(n, p.Kp, mode);
-    const int cols = ((n + 1) / 2) * p.Kp + a.ring * n * 32;
+    const int cols = ((n + 1) / 2) * 2 * p.Kp + a.ring * n * 32;
     a.tmem_cols = 32;
     while (a.tmem_cols < cols) a.tmem_cols *= 2;
     if (2 * smem <= 227 * 1024 && a.tmem_cols > 256) {        // two CTAs may share an SM: halve the claim
         a.ring = 2;
         a.tmem_cols = 256;
-        if (((n + 1) / 2) * p.Kp + 2 * n * 32 > 256) return false;
+        if (((n + 1) / 2) * 2 * p.Kp + 2 * n * 32 > 256) return false;
     }
     a.ehi = (const __nv_bfloat16*)ehi; a.elo = (const __nv_bfloat16*)elo; a.Wf = (const __nv_bfloat16*)Wf;
     a.kappa = kappa; a.H_res = H_res; a.H_pre = H_pre; a.Gpart = Gpart; a.status = status;
