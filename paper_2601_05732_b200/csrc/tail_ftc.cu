@@ -57,6 +57,10 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
 }
+// Asks the L2 cache for a box ahead of the TMA load that will bring it to shared memory.
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
+}
 __device__ __forceinline__ void ftc_ld8(uint32_t taddr, uint32_t (&r)[8]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
@@ -134,23 +138,30 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
             }
         }
     } else if (warp == 2) {
-        // ---- producer of the data: x (and g, du, or the old dx) per 32-token quadrant --------------------
-        if (lane == 0) {
+        // ---- producer of the data: x (and g, du, or the old dx) per 32-token quadrant.  Lane b issues the
+        //      loads of box b (issuing a TMA instruction keeps a thread busy for ~100 cycles: nine in a row
+        //      from one thread would delay the slots behind it), lane 0 arms the barrier.
+        {
+            const int b = lane < kBoxes ? lane : 0;
+            const CUtensorMap* mp = b < N_ ? &tmx : (b < 2 * N_ ? &tmg : &tmdu);
+            if (MODE == 2 && b >= N_) mp = &tmg;
+            const int col = (b < N_ ? b * a.C : (b < 2 * N_ ? (b - N_) * a.C : 0)) + c0;
             bool ok = true;
             for (int ti = 0; ti < nt && ok; ++ti) {
                 for (int q = 0; q < 4 && ok; ++q) {
-                    ok = mbar_wait(smem_u32(&ctl->d_empty[q]), (ti & 1) ^ 1, abort, 2, ti * 4 + q);
+                    if (lane == 0) ok = mbar_wait(smem_u32(&ctl->d_empty[q]), (ti & 1) ^ 1, abort, 2, ti * 4 + q);
+                    ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     const uint32_t full = smem_u32(&ctl->d_full[q]);
-                    mbar_expect_tx(full, kSlot);
-                    const uint32_t dst = smem_u32(slots + q * kSlot);
+                    if (lane == 0) mbar_expect_tx(full, kSlot);
+                    __syncwarp();
                     const int row = (int)(t0 + (int64_t)ti * kFTok + q * 32);
-#pragma unroll
-                    for (int j = 0; j < N_; ++j) {
-                        tma_load_2d(dst + j * kFBox, &tmx, full, j * a.C + c0, row);
-                        if (MODE != 0) tma_load_2d(dst + (N_ + j) * kFBox, &tmg, full, j * a.C + c0, row);
+                    if (lane < kBoxes) {
+                        tma_load_2d(smem_u32(slots + q * kSlot) + b * kFBox, mp, full, col, row);
+                        // the quadrant's next boxes start their way from HBM to L2 now: a slot is busy for a
+                        // whole load + compute + store round, too long to hide the HBM latency with four slots
+                        if (ti + 1 < nt && row + kFTok < a.T) tma_prefetch_2d(mp, col, row + kFTok);
                     }
-                    if (MODE == 1) tma_load_2d(dst + 2 * N_ * kFBox, &tmdu, full, c0, row);
                 }
             }
         }
@@ -299,22 +310,23 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(smem_u32(&ctl->q_done[quad]));
-                if (hw == 0 && mbar_wait(smem_u32(&ctl->q_done[quad]), ti & 1, abort, 10, ti)) {
-                    if (row0 < a.T) {
-#pragma unroll
-                        for (int j = 0; j < N_; ++j)
-                            tma_store_2d(&tmdx, smem_u32(slot + (kOut + j) * kFBox), j * a.C + c0, (int)row0);
-                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                    }
-                    // the slot goes back once the G MMAs have read its x boxes (long done by now)
-                    if (MODE == 0 || mbar_wait(smem_u32(&ctl->g_done[quad]), ti & 1, abort, 8, ti))
-                        mbar_arrive(smem_u32(&ctl->d_empty[quad]));
+            }
+            if (hw == 0) {
+                // lane j stores box j once both warps of the quadrant have written their part
+                bool oks = lane >= N_ || mbar_wait(smem_u32(&ctl->q_done[quad]), ti & 1, abort, 10, ti);
+                if (oks && lane < N_ && row0 < a.T) {
+                    tma_store_2d(&tmdx, smem_u32(slot + (kOut + lane) * kFBox), lane * a.C + c0, (int)row0);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 }
+                // the slot goes back once the G MMAs have read its x boxes as well (long done by now)
+                if (MODE != 0 && lane == 0 && oks) oks = mbar_wait(smem_u32(&ctl->g_done[quad]), ti & 1, abort, 8, ti);
+                oks = __all_sync(0xffffffffu, oks);
+                if (oks && lane == 0) mbar_arrive(smem_u32(&ctl->d_empty[quad]));
             }
             __syncwarp();
         }
-        if (hw == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if (hw == 0 && lane < N_) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         // ---- G of this token range -> its partial -----------------------------------------------------
         if (nt > 0) {
             if (ok) ok = mbar_wait(smem_u32(&ctl->g_final), 0, abort, 11, 0);
