@@ -202,7 +202,8 @@ __global__ void __launch_bounds__(kActThreads) lite_act_premix_k(
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
     const int64_t ngroups = (T + kGroupTok - 1) / kGroupTok;
     for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
-        const int64_t t0 = grp * kGroupTok;
+        // descending: the projection kernel before this one read x in ascending order and left its last lines in L2
+        const int64_t t0 = (ngroups - 1 - grp) * kGroupTok;
         const int nt = (T - t0 < kGroupTok) ? (int)(T - t0) : kGroupTok;
         // L
         if (tid < nt) {
@@ -526,7 +527,8 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
     __syncthreads();
     const int64_t ngroups = (T + kTokGroup - 1) / kTokGroup;
     for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
-        const int64_t t0 = grp * kTokGroup;
+        // descending: the projection kernel before this one read x in ascending order and left its last lines in L2
+        const int64_t t0 = (ngroups - 1 - grp) * kTokGroup;
         const int nt = (T - t0 < kTokGroup) ? (int)(T - t0) : kTokGroup;
         // L: partials -> normalised projection rows in shared memory (and p_saved, rstd)
         if (tid < nt) {

@@ -92,10 +92,11 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
     FCtl* ctl = reinterpret_cast<FCtl*>(w_s + ((w_bytes + 1023) & ~1023));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int c0 = blockIdx.x * kFCs;
-    const int tile_begin = (int)(((int64_t)a.ntiles * blockIdx.y) / a.splits);
-    const int tile_end = (int)(((int64_t)a.ntiles * (blockIdx.y + 1)) / a.splits);
-    const int nt = tile_end - tile_begin;
-    const int64_t t0 = (int64_t)tile_begin * kFTok;
+    // Token range blockIdx.y takes the tiles ntiles - 1 - (blockIdx.y + splits * ti), ti = 0, 1, ...: all ranges walk
+    // down the token axis together, starting where the kernel before this one (it read x and du in ascending
+    // order) left its last lines in the L2 cache.
+    const int nt = (a.ntiles - (int)blockIdx.y + a.splits - 1) / a.splits;
+    auto tile_of = [&](int ti) { return a.ntiles - 1 - ((int)blockIdx.y + a.splits * ti); };
     volatile int* abort = ctl->abort;
 
     if (tid == 0) {
@@ -132,7 +133,7 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                 if (!mbar_wait(smem_u32(&ctl->e_empty[buf]), ((ti >> 1) & 1) ^ 1, abort, 1, ti)) break;
                 const uint32_t full = smem_u32(&ctl->e_full[buf]);
                 mbar_expect_tx(full, 2 * e_bytes);
-                const int64_t off = (int64_t)(tile_begin + ti) * a.Kp * kFTok;       // elements
+                const int64_t off = (int64_t)tile_of(ti) * a.Kp * kFTok;             // elements
                 bulk_load(smem_u32(e_s + buf * 2 * e_bytes), a.ehi + off, e_bytes, full);
                 bulk_load(smem_u32(e_s + buf * 2 * e_bytes + e_bytes), a.elo + off, e_bytes, full);
             }
@@ -155,12 +156,13 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                     const uint32_t full = smem_u32(&ctl->d_full[q]);
                     if (lane == 0) mbar_expect_tx(full, kSlot);
                     __syncwarp();
-                    const int row = (int)(t0 + (int64_t)ti * kFTok + q * 32);
+                    const int row = tile_of(ti) * kFTok + q * 32;
+                    const int next_row = tile_of(ti + 1) * kFTok + q * 32;
                     if (lane < kBoxes) {
                         tma_load_2d(smem_u32(slots + q * kSlot) + b * kFBox, mp, full, col, row);
                         // the quadrant's next boxes start their way from HBM to L2 now: a slot is busy for a
                         // whole load + compute + store round, too long to hide the HBM latency with four slots
-                        if (ti + 1 < nt && row + kFTok < a.T) tma_prefetch_2d(mp, col, row + kFTok);
+                        if (ti + 1 < nt) tma_prefetch_2d(mp, col, next_row);
                     }
                 }
             }
@@ -237,7 +239,7 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
         float kap = 0.f, hp[N_], hr[N_][N_];
         bool ok = true;
         for (int ti = 0; ti < nt; ++ti) {
-            const int64_t row0 = t0 + (int64_t)ti * kFTok + quad * 32;
+            const int64_t row0 = (int64_t)tile_of(ti) * kFTok + quad * 32;
             const int64_t t = row0 + lane;
             const bool live = t < a.T;
             kap = live ? __ldg(a.kappa + t) : 0.f;
