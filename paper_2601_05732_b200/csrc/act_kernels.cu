@@ -601,186 +601,116 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
     }
 }
 
-// Backward of one token by one thread.  in: a | p | dH_res | H_pre | H_post | dH_post | rstd (shared memory);
-// orow: e[0..kN) | kappa | dz[0..kN).
-template <int N_>
-__device__ __forceinline__ void lite_thread_bwd(const float* in, const float* dhpre, float* orow, const uint8_t* sigma_s,
-                                                float a_res, float a_pre, float a_post, float inv_nC) {
-    using D = LiteDims<N_>;
-    const float* a = in;
-    const float* pt = in + D::kFact;
-    const float* dh = pt + D::kN;
-    const float* hpre = dh + D::kNN;
-    const float* hpost = hpre + N_;
-    const float* dhpost = hpost + N_;
-    const float rs = dhpost[N_];
-    constexpr PermConst<N_> tab = make_perm_const<N_>();
-    (void)sigma_s;
-    float dhr[D::kNN], da[D::kFact], dot = 0.f;
-#pragma unroll
-    for (int e = 0; e < D::kNN; ++e) dhr[e] = dh[e];
-#pragma unroll
-    for (int k = 0; k < D::kFact; ++k) {
-        float d = 0.f;
-#pragma unroll
-        for (int i = 0; i < N_; ++i) d += dhr[i * N_ + tab.s[k][i]];                // Eq. (5): dL/da_k
-        da[k] = d;
-        dot = fmaf(a[k], d, dot);
-    }
-    float kap = 0.f;
-#pragma unroll
-    for (int k = 0; k < D::kFact; ++k) {
-        const float d = da[k];
-        const float dz = a[k] * (d - dot), ed = a_res * dz, pv = pt[k];
-        orow[k] = rs * ed;
-        orow[D::kN + 1 + k] = dz;
-        kap = fmaf(ed, pv, kap);
-    }
-#pragma unroll
-    for (int j = 0; j < N_; ++j) {
-        {
-            const float h = hpre[j], dz = dhpre[j] * h * (1.f - h), ed = a_pre * dz, pv = pt[D::kFact + j];
-            orow[D::kFact + j] = rs * ed; orow[D::kN + 1 + D::kFact + j] = dz; kap = fmaf(ed, pv, kap);
-        }
-        {
-            const float h = hpost[j], dz = dhpost[j] * h * (1.f - 0.5f * h), ed = a_post * dz, pv = pt[D::kFact + N_ + j];
-            orow[D::kFact + N_ + j] = rs * ed; orow[D::kN + 1 + D::kFact + N_ + j] = dz; kap = fmaf(ed, pv, kap);
-        }
-    }
-    orow[D::kN] = rs * rs * kap * inv_nC;
-}
+// ------------------------------------------------------------------------------------------------
+// First kernel of the fused backward tail for n <= 4 (n! + 2n <= 32 columns), one warp per token and one
+// lane per projection column.  The warp streams x and du of its token for dH_pre[j] = <du, x_j> (gradient of
+// Eq. (1) w.r.t. H_pre); the per-token inputs of the activation backward were requested before the stream
+// and have arrived by its end.  Lane c then holds column c of the gradient of Eq. (4), (5):
+//   res columns k: da_k = sum_i dH_res[i][sigma_k(i)], dz_k = a_k (da_k - <a, da>)   (the dot product is a warp sum)
+//   pre / post columns: the sigmoid derivatives, dH_pre taken from the warp's own reduction
+// e = rstd alpha (.) dz goes out as the tiled bf16 pair (and / or fp32 rows), kappa = rstd^2 sum_c alpha dz p / (nC)
+// is a second warp sum, and the lane keeps its column of db and of sum_t dz p in registers until the end.
+constexpr int kTpwVec = 2;      // 16-byte vectors per lane and tensor in flight
 
-template <int N_, bool STREAM, int THREADS, int GROUP>
-__global__ void __launch_bounds__(THREADS) lite_tailpre_t_k(
+template <int N_>
+__global__ void __launch_bounds__(256, 4) lite_tailpre_w_k(
     int64_t T, int C8, float inv_nC, const uint4* __restrict__ x, const uint4* __restrict__ du,
-    const float* __restrict__ dH_pre_in,
     const float* __restrict__ a_saved, const float* __restrict__ p, const float* __restrict__ rstd,
     const float* __restrict__ alpha, const float* __restrict__ H_pre, const float* __restrict__ H_post,
     const float* __restrict__ dH_res, const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa,
     float* db, float* dalpha) {
     using D = LiteDims<N_>;
-    __shared__ uint8_t sigma_s[D::kFact * N_];
-    __shared__ float in_s[GROUP][D::kIn + 1];
-    __shared__ float dhp_s[GROUP][N_];
-    __shared__ float og[GROUP][2 * D::kN + 3];
-    __shared__ float dal_s[3];
-    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    for (int i = tid; i < D::kFact * N_; i += THREADS) sigma_s[i] = c_perm[N_].sigma[i];
-    if (tid < 3) dal_s[tid] = 0.f;
-    const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
-    float db_col = 0.f, dal_col = 0.f;             // thread c < kN: column c of db, and sum_t dz[t,c] p[t,c]
-    constexpr int o_p = D::kFact, o_dhres = o_p + D::kN, o_hpre = o_dhres + D::kNN, o_hpost = o_hpre + N_,
-                  o_dhpost = o_hpost + N_, o_rstd = o_dhpost + N_;
-    __syncthreads();
-    const int64_t ngroups = (T + GROUP - 1) / GROUP;
-    for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
-        const int64_t t0 = grp * GROUP;
-        const int nt = (T - t0 < GROUP) ? (int)(T - t0) : GROUP;
-        // L: stage the per-token inputs with cp.async (they arrive while D streams)
-        for (int i = tid; i < nt * D::kIn; i += THREADS) {
-            const int tl = i / D::kIn, c = i - tl * D::kIn;
-            const int64_t t = t0 + tl;
-            const float* src;
-            if (c < o_p) src = a_saved + t * D::kFact + c;
-            else if (c < o_dhres) src = p + t * D::kN + (c - o_p);
-            else if (c < o_hpre) src = dH_res + t * D::kNN + (c - o_dhres);
-            else if (c < o_hpost) src = H_pre + t * N_ + (c - o_hpre);
-            else if (c < o_dhpost) src = H_post + t * N_ + (c - o_hpost);
-            else if (c < o_rstd) src = dH_post + t * N_ + (c - o_dhpost);
-            else src = rstd + t;
-            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&in_s[tl][c])), "l"(src) : "memory");
+    __shared__ float red[2][8][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int c = lane;
+    const bool is_res = c < D::kFact, is_pre = !is_res && c < D::kFact + N_, is_post = !is_res && !is_pre && c < D::kN;
+    const int jj = is_pre ? c - D::kFact : (is_post ? c - D::kFact - N_ : 0);
+    int sg[N_];
+#pragma unroll
+    for (int i = 0; i < N_; ++i) sg[i] = is_res ? i * N_ + c_perm[N_].sigma[c * N_ + i] : 0;
+    const float al = __ldg(alpha + (is_res ? 0 : (is_pre ? 1 : 2)));
+    float db_c = 0.f, dal_c = 0.f;
+    const int64_t warp0 = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * 256) >> 5;
+    for (int64_t t = warp0; t < T; t += nwarps) {
+        // per-token inputs of lane c, in flight during the stream
+        const float av = is_res ? __ldg(a_saved + t * D::kFact + c) : 0.f;
+        const float pv = c < D::kN ? __ldg(p + t * D::kN + c) : 0.f;
+        const float rs = __ldg(rstd + t);
+        float d = 0.f;
+        if (is_res) {
+#pragma unroll
+            for (int i = 0; i < N_; ++i) d += __ldg(dH_res + t * D::kNN + sg[i]);          // Eq. (5): dL/da_k
         }
-        cp_async_commit();
-        // D: dH_pre[j] = <du, x_j>, one warp per token (or taken from a preceding premix_bwd call)
-        if (!STREAM) {
-            for (int i = tid; i < nt * N_; i += THREADS) dhp_s[i / N_][i % N_] = __ldg(dH_pre_in + t0 * N_ + i);
-        }
-        for (int tl = w; STREAM && tl < nt; tl += (THREADS / 32)) {
-            const int64_t t = t0 + tl;
-            float r[N_];
+        const float h = is_pre ? __ldg(H_pre + t * N_ + jj) : (is_post ? __ldg(H_post + t * N_ + jj) : 0.f);
+        const float dhp = is_post ? __ldg(dH_post + t * N_ + jj) : 0.f;
+        float r[N_];
 #pragma unroll
-            for (int j = 0; j < N_; ++j) r[j] = 0.f;
-            for (int cv = lane; cv < C8; cv += 64) {               // two vectors per lane in flight
-                const int cw = cv + 32;
-                const bool has1 = cw < C8;
-                uint4 xv[N_], xw[N_], dv, dw = make_uint4(0, 0, 0, 0);
+        for (int j = 0; j < N_; ++j) r[j] = 0.f;
+        for (int cv0 = lane; cv0 < C8; cv0 += 32 * kTpwVec) {
+            uint4 xv[kTpwVec][N_], dv[kTpwVec];
 #pragma unroll
-                for (int j = 0; j < N_; ++j) xv[j] = ld_stream(x + (t * N_ + j) * C8 + cv);
-                dv = ld_stream(du + t * C8 + cv);
-                if (has1) {
+            for (int v = 0; v < kTpwVec; ++v) {
+                const int cv = cv0 + 32 * v;
+                if (cv < C8) {
 #pragma unroll
-                    for (int j = 0; j < N_; ++j) xw[j] = ld_stream(x + (t * N_ + j) * C8 + cw);
-                    dw = ld_stream(du + t * C8 + cw);
+                    for (int j = 0; j < N_; ++j) xv[v][j] = ld_stream(x + (t * N_ + j) * C8 + cv);
+                    dv[v] = ld_stream(du + t * C8 + cv);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) xv[v][j] = make_uint4(0, 0, 0, 0);
+                    dv[v] = make_uint4(0, 0, 0, 0);
                 }
-                float df[8], dg[8];
-                unpack8(dv, df);
-                unpack8(dw, dg);
+            }
+#pragma unroll
+            for (int v = 0; v < kTpwVec; ++v) {
+                float df[8];
+                unpack8(dv[v], df);
 #pragma unroll
                 for (int j = 0; j < N_; ++j) {
                     float xf[8];
-                    unpack8(xv[j], xf);
+                    unpack8(xv[v][j], xf);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) r[j] = fmaf(df[e], xf[e], r[j]);
-                    if (has1) {
-                        unpack8(xw[j], xf);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) r[j] = fmaf(dg[e], xf[e], r[j]);
-                    }
                 }
             }
+        }
+        float rj = 0.f;
 #pragma unroll
-            for (int j = 0; j < N_; ++j) { r[j] = warp_sum(r[j]); if (lane == j) dhp_s[tl][j] = r[j]; }
+        for (int j = 0; j < N_; ++j) { r[j] = warp_sum(r[j]); if (jj == j) rj = r[j]; }
+        const float dot = warp_sum(av * d);
+        float dz = 0.f;
+        if (is_res) dz = av * (d - dot);
+        else if (is_pre) dz = rj * h * (1.f - h);
+        else if (is_post) dz = dhp * h * (1.f - 0.5f * h);
+        const float ed = al * dz;
+        const float kap = warp_sum(ed * pv);
+        const float ev = rs * ed;
+        db_c += dz;
+        dal_c = fmaf(dz, pv, dal_c);
+        if (eo.ehi && c < eo.Kp) {
+            __nv_bfloat16 hi, lo;
+            split_bf16(ev, hi, lo);
+            const int64_t o = e_tiled_index(eo.Kp, t, c);
+            eo.ehi[o] = hi;
+            eo.elo[o] = lo;
         }
-        cp_async_wait<0>();
-        __syncthreads();
-        // A: one thread per token
-        if (tid < nt) lite_thread_bwd<N_>(in_s[tid], dhp_s[tid], og[tid], sigma_s, a_res, a_pre, a_post, inv_nC);
-        __syncthreads();
-        if (tid < D::kN) {
-            for (int tl = 0; tl < nt; ++tl) {
-                const float dz = og[tl][D::kN + 1 + tid];
-                db_col += dz;
-                dal_col = fmaf(dz, in_s[tl][o_p + tid], dal_col);
-            }
-        }
-        // W: e as a bf16 pair (one 16-byte piece of 8 columns per thread, consecutive tokens side by side in
-        // the tiled layout) and / or fp32 rows; kappa
-        if (eo.ehi) {
-            for (int i = tid; i < nt * (eo.Kp >> 3); i += THREADS) {
-                const int cg = i / nt, tl = i - cg * nt;
-                uint32_t hw[4], lw[4];
-#pragma unroll
-                for (int e2 = 0; e2 < 4; ++e2) {
-                    const int c = cg * 8 + 2 * e2;
-                    const float v0 = (c < D::kN) ? og[tl][c] : 0.f, v1 = (c + 1 < D::kN) ? og[tl][c + 1] : 0.f;
-                    __nv_bfloat16 h0, l0, h1, l1;
-                    split_bf16(v0, h0, l0);
-                    split_bf16(v1, h1, l1);
-                    hw[e2] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-                    lw[e2] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-                }
-                const int64_t o = e_tiled_index(eo.Kp, t0 + tl, cg * 8);
-                *reinterpret_cast<uint4*>(eo.ehi + o) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-                *reinterpret_cast<uint4*>(eo.elo + o) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-            }
-        }
-        if (eo.e) {
-            for (int i = tid; i < nt * eo.Npad; i += THREADS) {
-                const int tl = i / eo.Npad, c = i - tl * eo.Npad;
-                eo.e[(t0 + tl) * eo.Npad + c] = (c < D::kN) ? og[tl][c] : 0.f;
-            }
-        }
-        if (tid < nt) kappa[t0 + tid] = og[tid][D::kN];
-        __syncthreads();
+        if (eo.e && c < eo.Npad) eo.e[t * eo.Npad + c] = ev;
+        if (lane == 0) kappa[t] = rs * rs * kap * inv_nC;
     }
-    // parameter-gradient partials of this block
-    (void)lane; (void)w;
-    if (tid < D::kN) {
-        atomicAdd(db + tid, db_col);
-        atomicAdd(&dal_s[tid < D::kFact ? 0 : (tid < D::kFact + N_ ? 1 : 2)], dal_col);
-    }
+    // parameter-gradient partials of this block: columns over the warps, then one atomic per column
+    red[0][w][lane] = db_c;
+    red[1][w][lane] = dal_c;
     __syncthreads();
-    if (tid < 3) atomicAdd(dalpha + tid, dal_s[tid]);
+    if (w == 0) {
+        float sdb = 0.f, sdal = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { sdb += red[0][k][lane]; sdal += red[1][k][lane]; }
+        if (c < D::kN) atomicAdd(db + c, sdb);
+        const float s_res = warp_sum(is_res ? sdal : 0.f), s_pre = warp_sum(is_pre ? sdal : 0.f),
+                    s_post = warp_sum(is_post ? sdal : 0.f);
+        if (lane == 0) { atomicAdd(dalpha, s_res); atomicAdd(dalpha + 1, s_pre); atomicAdd(dalpha + 2, s_post); }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1022,13 +952,14 @@ void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const v
     clear_e_tail(T, ehi, elo, Kp, s);
     const int C8 = c->C / 8;
     const float inv = 1.f / (float)(c->n * c->C);
-    // n <= 4: a streaming pass for dH_pre (premix_bwd without dx), then the thread-per-token activation backward;
-    // measured faster than one kernel doing both, whose per-token phase stalls the streaming warps
-#define MHCL_TP_T(N_) do { \
-        launch_premix_bwd(c, T, x, H_pre, du, dH_pre_ws, nullptr, 0, s); \
-        lite_tailpre_t_k<N_, false, 128, 32><<<group_grid(T, 32, c->sm_count), 128, 0, s>>>( \
-            T, C8, inv, (const uint4*)x, (const uint4*)du, dH_pre_ws, a, p, rstd, alpha, H_pre, H_post, dH_res, dH_post, \
-            eo, kappa, db, dalpha); } while (0)
+    // n <= 4: one warp per token streams for dH_pre and then does the activation backward with a lane per column
+    int64_t blocks = (T * 32 + 255) / 256;
+    if (blocks > (int64_t)c->sm_count * 8) blocks = (int64_t)c->sm_count * 8;
+    if (blocks < 1) blocks = 1;
+    (void)dH_pre_ws;
+#define MHCL_TP_T(N_) lite_tailpre_w_k<N_><<<(int)blocks, 256, 0, s>>>( \
+        T, C8, inv, (const uint4*)x, (const uint4*)du, a, p, rstd, alpha, H_pre, H_post, dH_res, dH_post, eo, kappa, \
+        db, dalpha)
     switch (c->n) {
         case 2: MHCL_TP_T(2); break;
         case 3: MHCL_TP_T(3); break;
