@@ -42,10 +42,12 @@ bool launch_tail_dx_tc(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p
                        const float* W, const float* gain, void* Wb, void* dx, int acc_dx, int* status, cudaStream_t s);
 // tail_ftc.cu : narrow projections, dx and the G partials [f_splits][nC][Kp] in one tcgen05 kernel
 void plan_tail_ftc(int n, int C, int64_t T, int sm_count, TailPlan* p);
+bool launch_tail_ftc_prep(const mhclite_ctx* c, int N, const TailPlan& p, const float* W, const float* gain, void* Wf,
+                          float* zero_db, float* zero_dalpha, cudaStream_t s);
 bool launch_tail_ftc(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, const void* x, const void* g,
                      const void* du, const void* ehi, const void* elo, const float* kappa, const float* H_res,
-                     const float* H_pre, const float* W, const float* gain, void* Wf, void* dx, int acc_dx,
-                     float* Gpart, int* status, cudaStream_t s);
+                     const float* H_pre, const float* W, const float* gain, void* Wf, bool wf_packed, void* dx,
+                     int acc_dx, float* Gpart, int* status, cudaStream_t s);
 void launch_tail_finish(const mhclite_ctx* c, int N, int Kp, int splits, const float* W, const float* gain,
                         const float* Gpart, float* dW, float* dgain, int acc_params, cudaStream_t s);
 bool proj_tc_supported(int n, int C, int N);

@@ -129,10 +129,10 @@ static bool tail_pair(const TailPlan& tp) { return tp.supported || (tp.tc && ten
 // parameter gradients dW, dgain.  Tensor cores when the projection is narrow enough, CUDA cores otherwise.
 static int proj_backward(mhclite_ctx* ctx, int64_t T, int N, const Workspace& w, const TailPlan& tp,
                          const mhclite_bf16* x, const mhclite_bf16* g, const mhclite_bf16* du, const float* H_res,
-                         const float* H_pre, const float* W, const float* gain, mhclite_bf16* dx, int accumulate_dx,
-                         float* dW, float* dgain, int accumulate_params, cudaStream_t s) {
-    if (tp.ftc && launch_tail_ftc(ctx, T, N, tp, x, g, du, w.ehi, w.elo, w.kappa, H_res, H_pre, W, gain, w.Wb, dx,
-                                  accumulate_dx, w.Gpart, w.status, s)) {
+                         const float* H_pre, const float* W, const float* gain, bool wf_packed, mhclite_bf16* dx,
+                         int accumulate_dx, float* dW, float* dgain, int accumulate_params, cudaStream_t s) {
+    if (tp.ftc && launch_tail_ftc(ctx, T, N, tp, x, g, du, w.ehi, w.elo, w.kappa, H_res, H_pre, W, gain, w.Wb, wf_packed,
+                                  dx, accumulate_dx, w.Gpart, w.status, s)) {
         MHCL_LAUNCH_CHECK(ctx, "tail_ftc");
         ctx->launches += 1;
         launch_tail_finish(ctx, N, tp.Kp, tp.f_splits, W, gain, w.Gpart, dW, dgain, accumulate_params, s);
@@ -341,8 +341,14 @@ int mhclite_premix_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     return MHCLITE_OK;
 }
 
-// Zeroes the parameter-gradient accumulators that the kernels add into, unless the caller accumulates.
-static int prep_param_grads(mhclite_ctx* ctx, int N, float* db, float* dalpha, int accumulate, cudaStream_t s) {
+// Zeroes the parameter-gradient accumulators that the kernels add into, unless the caller accumulates.  When
+// the backward ends in the fused tcgen05 tail, the kernel that packs W' for it does the zeroing as well
+// (*wf_packed tells proj_backward that W' is ready).
+static int prep_param_grads(mhclite_ctx* ctx, int N, const TailPlan& tp, const Workspace& w, const float* W,
+                            const float* gain, float* db, float* dalpha, int accumulate, cudaStream_t s,
+                            bool* wf_packed) {
+    *wf_packed = launch_tail_ftc_prep(ctx, N, tp, W, gain, w.Wb, accumulate ? nullptr : db, accumulate ? nullptr : dalpha, s);
+    if (*wf_packed) return check_cuda(ctx, cudaGetLastError(), "pack_wf");
     if (accumulate) return MHCLITE_OK;
     int rc = check_cuda(ctx, cudaMemsetAsync(db, 0, (size_t)N * sizeof(float), s), "memset db");
     if (rc) return rc;
@@ -367,13 +373,14 @@ int mhclite_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
     const int N = n_cols(ctx->n, 0);
-    rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
-    if (rc) return rc;
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
+    bool wf_packed = false;
+    rc = prep_param_grads(ctx, N, tp, w, W, gain, db, dalpha, accumulate_params, s, &wf_packed);
+    if (rc) return rc;
     launch_lite_act_bwd(ctx, T, w.Npad, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post,
                         tp.supported ? nullptr : w.e, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_act_bwd");
-    return proj_backward(ctx, T, N, w, tp, x, nullptr, nullptr, nullptr, nullptr, W, gain, dx, accumulate_dx, dW, dgain,
+    return proj_backward(ctx, T, N, w, tp, x, nullptr, nullptr, nullptr, nullptr, W, gain, wf_packed, dx, accumulate_dx, dW, dgain,
                          accumulate_params, s);
 }
 
@@ -395,14 +402,15 @@ int mhclite_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, c
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
     const int N = n_cols(ctx->n, 0);
-    rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
-    if (rc) return rc;
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
+    bool wf_packed = false;
+    rc = prep_param_grads(ctx, N, tp, w, W, gain, db, dalpha, accumulate_params, s, &wf_packed);
+    if (rc) return rc;
     launch_lite_tailpre(ctx, T, x, du, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_post, w.dH_pre,
                         tp.supported ? nullptr : w.e, w.Npad, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db,
                         dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_tailpre");
-    return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W, gain, dx, 0, dW, dgain, accumulate_params, s);
+    return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W, gain, wf_packed, dx, 0, dW, dgain, accumulate_params, s);
 }
 
 // ---- SK comparison path --------------------------------------------------------------------------
@@ -448,13 +456,14 @@ int mhc_sk20_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
     const int N = n_cols(ctx->n, 1);
-    rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
-    if (rc) return rc;
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
+    bool wf_packed = false;
+    rc = prep_param_grads(ctx, N, tp, w, W_sk, gain, db, dalpha, accumulate_params, s, &wf_packed);
+    if (rc) return rc;
     launch_sk_act_bwd(ctx, T, w.Npad, iters, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, dH_pre, dH_post,
                       tp.supported ? nullptr : w.e, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "sk_act_bwd");
-    return proj_backward(ctx, T, N, w, tp, x, nullptr, nullptr, nullptr, nullptr, W_sk, gain, dx, accumulate_dx, dW,
+    return proj_backward(ctx, T, N, w, tp, x, nullptr, nullptr, nullptr, nullptr, W_sk, gain, wf_packed, dx, accumulate_dx, dW,
                          dgain, accumulate_params, s);
 }
 
@@ -478,15 +487,16 @@ int mhc_sk20_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, 
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
     const int N = n_cols(ctx->n, 1);
-    rc = prep_param_grads(ctx, N, db, dalpha, accumulate_params, s);
-    if (rc) return rc;
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
+    bool wf_packed = false;
+    rc = prep_param_grads(ctx, N, tp, w, W_sk, gain, db, dalpha, accumulate_params, s, &wf_packed);
+    if (rc) return rc;
     launch_premix_bwd(ctx, T, x, H_pre, du, w.dH_pre, nullptr, 0, s);
     MHCL_LAUNCH_CHECK(ctx, "premix_bwd");
     launch_sk_act_bwd(ctx, T, w.Npad, iters, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, w.dH_pre, dH_post,
                       tp.supported ? nullptr : w.e, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "sk_act_bwd");
-    return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W_sk, gain, dx, 0, dW, dgain, accumulate_params, s);
+    return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W_sk, gain, wf_packed, dx, 0, dW, dgain, accumulate_params, s);
 }
 
 int mhclite_ds_gap(mhclite_ctx* ctx, int64_t T, const float* H_res, float* l1_err, float* colsum_dev, void* stream) {

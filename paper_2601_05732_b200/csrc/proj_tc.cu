@@ -179,14 +179,24 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
 // ---- W' as two stacked K-major bf16 matrices: rows [0, nq) = hi, rows [nq, 2 nq) = lo, row length Kpad ----
 __global__ void __launch_bounds__(256) pack_wt_k(int nC, int N, int nq, int Kpad, const float* __restrict__ W,
                                                  const float* __restrict__ gain, __nv_bfloat16* __restrict__ Wt) {
-    const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;       // over nq x Kpad, k fastest
-    if (idx >= (int64_t)nq * Kpad) return;
-    const int c = (int)(idx / Kpad), k = (int)(idx - (int64_t)c * Kpad);
-    const float w = (k < nC && c < N) ? __ldg(W + (int64_t)k * N + c) * __ldg(gain + k) : 0.f;
-    __nv_bfloat16 hi, lo;
-    split_bf16(w, hi, lo);
-    Wt[(int64_t)c * Kpad + k] = hi;
-    Wt[(int64_t)(nq + c) * Kpad + k] = lo;
+    // a 32 (k) x 32 (column) tile through shared memory: W is read along its rows, Wt written along k
+    __shared__ float tile[32][33];
+    const int k0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int r = ty; r < 32; r += 8) {
+        const int k = k0 + r, c = c0 + tx;
+        tile[r][tx] = (k < nC && c < N) ? __ldg(W + (int64_t)k * N + c) * __ldg(gain + k) : 0.f;
+    }
+    __syncthreads();
+    for (int r = ty; r < 32; r += 8) {
+        const int c = c0 + r, k = k0 + tx;
+        if (c < nq && k < Kpad) {
+            __nv_bfloat16 hi, lo;
+            split_bf16(tile[tx][r], hi, lo);
+            Wt[(int64_t)c * Kpad + k] = hi;
+            Wt[(int64_t)(nq + c) * Kpad + k] = lo;
+        }
+    }
 }
 
 // ---- host side -------------------------------------------------------------------------------------
@@ -244,8 +254,8 @@ void launch_pack_wt(const mhclite_ctx* c, const ProjPlan& p, int N, const float*
                     cudaStream_t s) {
     c->launches += 1;
     const int nq = proj_tc_nq(N), Kpad = p.nchunks * kTcK;
-    const int64_t total = (int64_t)nq * Kpad;
-    pack_wt_k<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(c->n * c->C, N, nq, Kpad, W, gain, (__nv_bfloat16*)Wt);
+    dim3 grid((unsigned)((Kpad + 31) / 32), (unsigned)((nq + 31) / 32));
+    pack_wt_k<<<grid, 256, 0, s>>>(c->n * c->C, N, nq, Kpad, W, gain, (__nv_bfloat16*)Wt);
 }
 
 // Returns false when the tensor maps could not be built (the caller then uses the mma.sync kernel).

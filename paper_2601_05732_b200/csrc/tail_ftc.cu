@@ -366,10 +366,14 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
 }
 
 // W' = diag(gain) W in bf16 as the B operand of tail_ftc_k: per slice of 64 channels and per half of it a
-// block [Kp/8 column groups][n streams][32 channels][8 columns]; zero beyond the N columns.
+// block [Kp/8 column groups][n streams][32 channels][8 columns]; zero beyond the N columns.  The same launch
+// clears the accumulators db[N] and dalpha[3] when they are given (the backward's kernels add into them).
 __global__ void __launch_bounds__(256) pack_wf_k(int n, int C, int N, int Kp, const float* __restrict__ W,
-                                                 const float* __restrict__ gain, __nv_bfloat16* __restrict__ Wf) {
+                                                 const float* __restrict__ gain, __nv_bfloat16* __restrict__ Wf,
+                                                 float* zero_db, float* zero_dalpha) {
     const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (zero_db && idx < N) zero_db[idx] = 0.f;
+    if (zero_dalpha && idx < 3) zero_dalpha[idx] = 0.f;
     const int64_t total = (int64_t)n * C * Kp;
     if (idx >= total) return;
     const int c8 = (int)(idx & 7), chl = (int)((idx >> 3) & 31);
@@ -424,12 +428,24 @@ static void launch_ftc_t(dim3 grid, int smem, const CUtensorMap& tmx, const CUte
 #undef MHCL_FTC
 }
 
-// dx and the G partials [f_splits][nC][Kp] in one pass; packs W' first.  False (nothing launched) when no
-// tensor map could be made.
+// First launch of a backward whose tail is tail_ftc_k: packs W' and clears db / dalpha (null: left alone) in one
+// kernel.  False (nothing launched) when that tail is not available for the plan.
+bool launch_tail_ftc_prep(const mhclite_ctx* c, int N, const TailPlan& p, const float* W, const float* gain, void* Wf,
+                          float* zero_db, float* zero_dalpha, cudaStream_t s) {
+    if (c->n > 4 || !p.ftc || !tensor_maps_available()) return false;
+    c->launches += 1;
+    const int64_t total = (int64_t)c->n * c->C * p.Kp;
+    pack_wf_k<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(c->n, c->C, N, p.Kp, W, gain, (__nv_bfloat16*)Wf, zero_db,
+                                                              zero_dalpha);
+    return true;
+}
+
+// dx and the G partials [f_splits][nC][Kp] in one pass; packs W' first unless launch_tail_ftc_prep has done so.
+// False (nothing launched) when no tensor map could be made.
 bool launch_tail_ftc(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, const void* x, const void* g,
                      const void* du, const void* ehi, const void* elo, const float* kappa, const float* H_res,
-                     const float* H_pre, const float* W, const float* gain, void* Wf, void* dx, int acc_dx,
-                     float* Gpart, int* status, cudaStream_t s) {
+                     const float* H_pre, const float* W, const float* gain, void* Wf, bool wf_packed, void* dx,
+                     int acc_dx, float* Gpart, int* status, cudaStream_t s) {
     const int n = c->n, C = c->C, nC = n * C;
     if (n > 4 || !p.ftc) return false;
     const int mode = g ? 1 : (acc_dx ? 2 : 0);
@@ -455,9 +471,13 @@ bool launch_tail_ftc(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, 
     }
     a.ehi = (const __nv_bfloat16*)ehi; a.elo = (const __nv_bfloat16*)elo; a.Wf = (const __nv_bfloat16*)Wf;
     a.kappa = kappa; a.H_res = H_res; a.H_pre = H_pre; a.Gpart = Gpart; a.status = status;
-    c->launches += 2;
-    const int64_t total = (int64_t)nC * p.Kp;
-    pack_wf_k<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(n, C, N, p.Kp, W, gain, (__nv_bfloat16*)Wf);
+    c->launches += 1;
+    if (!wf_packed) {
+        c->launches += 1;
+        const int64_t total = (int64_t)nC * p.Kp;
+        pack_wf_k<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(n, C, N, p.Kp, W, gain, (__nv_bfloat16*)Wf, nullptr,
+                                                                  nullptr);
+    }
     KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_MMA, s);
     dim3 grid(p.f_slices, p.f_splits);
     switch (n) {

@@ -319,16 +319,15 @@ __global__ void __launch_bounds__(256) tail_finish_k(int nC, int N, int Kp, int 
     const float gm = __ldg(gain + m);
     float dg = 0.f;
     for (int c = lane; c < N; c += 32) {
-        float g0 = 0.f, g1 = 0.f, g2 = 0.f, g3 = 0.f;            // independent partial sums: the loads overlap
-        int s = 0;
-        for (; s + 4 <= splits; s += 4) {
-            g0 += Gpart[((int64_t)(s + 0) * nC + m) * Kp + c];
-            g1 += Gpart[((int64_t)(s + 1) * nC + m) * Kp + c];
-            g2 += Gpart[((int64_t)(s + 2) * nC + m) * Kp + c];
-            g3 += Gpart[((int64_t)(s + 3) * nC + m) * Kp + c];
+        float gv = 0.f;
+        for (int s0 = 0; s0 < splits; s0 += 16) {                 // sixteen loads in flight, then a fixed-order sum
+            float v[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k)
+                v[k] = (s0 + k < splits) ? __ldg(Gpart + ((int64_t)(s0 + k) * nC + m) * Kp + c) : 0.f;
+#pragma unroll
+            for (int k = 0; k < 16; k += 4) gv += (v[k] + v[k + 1]) + (v[k + 2] + v[k + 3]);
         }
-        for (; s < splits; ++s) g0 += Gpart[((int64_t)s * nC + m) * Kp + c];
-        const float gv = (g0 + g1) + (g2 + g3);
         const int64_t i = (int64_t)m * N + c;
         dW[i] = ACC ? dW[i] + gm * gv : gm * gv;
         dg = fmaf(__ldg(W + i), gv, dg);
