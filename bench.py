@@ -219,22 +219,43 @@ def run_ours(args, wl, rank, world):
         step()
     barrier()
 
+    # One step's launches (all issued by the library through the C ABI) captured once in a CUDA graph and
+    # replayed: the nine kernels of a step are short enough for launch gaps to show.  Falls back to plain
+    # launches when the capture is refused.
+    launches_per_step = ctx.kernel_launches()
+    step()
+    launches_per_step = ctx.kernel_launches() - launches_per_step
+    run_step, launch_mode = step, "stream"
+    if not args.no_graph:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            graph.replay()
+            torch.cuda.synchronize()
+            run_step, launch_mode = graph.replay, "cuda_graph"
+        except Exception as exc:                  # noqa: BLE001 - any capture failure means plain launches
+            print(f"bench.py: CUDA graph capture refused ({exc}); timing plain launches", file=sys.stderr)
+            torch.cuda.synchronize()
+    for _ in range(3):
+        run_step()
+    barrier()
+
     # ---- timed region: K steps, device time, max over ranks ------------------------------------
     sampler = ClockSampler(local) if rank == 0 else None
-    launches0 = ctx.kernel_launches()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
     for _ in range(args.steps):
-        step()
+        run_step()
     e1.record()
     barrier()
     ms = e0.elapsed_time(e1)
-    launches = ctx.kernel_launches() - launches0
+    launches = launches_per_step * args.steps
     # keep the GPU busy a little longer so that the sampler sees the loaded clocks even for short runs
     t_end = time.time() + 0.6
     while rank == 0 and time.time() < t_end:
-        step()
+        run_step()
     torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
     ms = D.max_over_ranks(ms, world, dev)
@@ -347,7 +368,7 @@ def run_ours(args, wl, rank, world):
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, f32 accumulate",
             "data": "synthetic",
-            "config": {"workload": wl.name, "n": n, "C": C, "T_per_gpu": T, "passes": "fwd+bwd" if wl.backward else "fwd", "calls": "fused" if fused else "unfused",
+            "config": {"workload": wl.name, "n": n, "C": C, "T_per_gpu": T, "passes": "fwd+bwd" if wl.backward else "fwd", "calls": "fused" if fused else "unfused", "launch": launch_mode,
                        "note": wl.note, "l2": "inputs larger than L2 (working set %.0f MB)" % (total_bytes / 1e6)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
             "cpu_baseline": cpu_baseline, "sk20_comparison": sk20,
@@ -369,6 +390,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sk", action="store_true", help="skip the SK-20 comparison path")
     ap.add_argument("--unfused", action="store_true", help="time the un-fused call sequence (six entry points)")
+    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph of one step")
     args = ap.parse_args()
 
     from paper_2601_05732_b200 import synth
