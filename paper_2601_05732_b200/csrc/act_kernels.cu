@@ -953,11 +953,9 @@ void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const v
     const int C8 = c->C / 8;
     const float inv = 1.f / (float)(c->n * c->C);
     // n <= 4: one warp per token streams for dH_pre and then does the activation backward with a lane per column
-    int64_t blocks = (T * 32 + 255) / 256;
-    if (blocks > (int64_t)c->sm_count * 8) blocks = (int64_t)c->sm_count * 8;
-    if (blocks < 1) blocks = 1;
+    const int blocks = balanced_warp_blocks(T, (int64_t)c->sm_count * 4);      // four blocks per SM fit
     (void)dH_pre_ws;
-#define MHCL_TP_T(N_) lite_tailpre_w_k<N_><<<(int)blocks, 256, 0, s>>>( \
+#define MHCL_TP_T(N_) lite_tailpre_w_k<N_><<<blocks, 256, 0, s>>>( \
         T, C8, inv, (const uint4*)x, (const uint4*)du, a, p, rstd, alpha, H_pre, H_post, dH_res, dH_post, eo, kappa, \
         db, dalpha)
     switch (c->n) {

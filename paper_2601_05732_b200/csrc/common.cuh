@@ -48,6 +48,16 @@ __host__ __device__ inline int64_t e_tiled_index(int Kp, int64_t t, int c) {
     return ((t >> 7) * (Kp >> 3) + (c >> 3)) * 1024 + (t & 127) * 8 + (c & 7);
 }
 
+// Grid of a warp-per-token kernel (8 warps per block) whose warps stride over the tokens: at most cap_blocks
+// blocks, and no more warps than give every warp the same number of tokens (a warp with one token less than
+// its neighbours only idles at the end).
+inline int balanced_warp_blocks(int64_t T, int64_t cap_blocks) {
+    if (T < 1) return 1;
+    const int64_t per_warp = (T + cap_blocks * 8 - 1) / (cap_blocks * 8);
+    const int64_t warps = (T + per_warp - 1) / per_warp;
+    return (int)((warps + 7) / 8);
+}
+
 // Number of projection columns. kind 0: n!+2n (mHC-lite); kind 1: n*n+2n (SK path).
 inline int n_res_cols(int n, int kind) { return kind == 0 ? ipow_fact(n) : n * n; }
 inline int n_cols(int n, int kind) { return n_res_cols(n, kind) + 2 * n; }
