@@ -6,9 +6,10 @@
 //   G[m,c]     = sum_t x[t,m] e[t,c]                              (dW = gain (.) G, dgain = sum_c W G)
 //
 // A CTA owns a slice of 64 channels of all n streams and walks over a range of 128-token tiles.
-//   * x, g and du arrive by TMA (128-byte swizzle) per 32-token quadrant into four slots, one per lane
-//     quadrant of the tensor memory; the tiled e buffers (hi, lo) of a tile arrive as two bulk copies; the
-//     CTA's rows of W' stay in shared memory.
+//   * x, g and du arrive by TMA (128-byte swizzle) per 32-token quadrant into five slots: one per lane
+//     quadrant of the tensor memory plus one that goes round, so that the load of a quadrant's next tile is
+//     under way while the quadrant still works on its current one (load number l goes to slot l mod 5).  The
+//     tiled e buffers (hi, lo) of a tile arrive as two bulk copies; the CTA's rows of W' stay in shared memory.
 //   * One thread issues tcgen05.mma: dxhat of a tile half (M = 128 tokens, N = n x 32 channels, K = Kp) into a
 //     ring of tensor-memory buffers, and per arrived quadrant G += x^T e (M = 128 rows of the slice, N = Kp,
 //     K = 32 tokens, x as the MN-major operand straight from its slot, e as hi | lo side by side in N) into
@@ -33,9 +34,11 @@ constexpr int kFBox = 32 * 128;                 // one TMA box: 32 tokens x 64 c
 constexpr int kFEpiWarps = 8;
 constexpr int kFThreads = 96 + 32 * kFEpiWarps; // operand producer, MMA issuer, data producer, epilogue
 constexpr int kFMaxRing = 3;
+constexpr int kFSlots = 5;                      // data slots: one per lane quadrant plus one that goes round
 
 struct FCtl {
-    uint64_t w_full, e_full[2], e_empty[2], d_full[4], d_empty[4], g_done[4], q_done[4], acc_full[kFMaxRing],
+    uint64_t w_full, e_full[2], e_empty[2], elo_full, elo_empty, d_full[4][2], g_done[4][2], q_done[4],
+        s_free[kFSlots], acc_full[kFMaxRing],
         acc_empty[kFMaxRing], g_final;
     uint32_t tmem_base;
     int abort[3];
@@ -87,8 +90,8 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
     const int e_bytes = a.Kp * kFTok * 2;                      // one of hi / lo of a tile; a multiple of 4096
     const int w_bytes = a.Kp * N_ * kFCs * 2;
     unsigned char* slots = smem;
-    unsigned char* e_s = slots + 4 * kSlot;                    // [2 buffers][hi | lo]
-    unsigned char* w_s = e_s + 4 * e_bytes;
+    unsigned char* e_s = slots + kFSlots * kSlot;              // e_hi of even tiles | e_hi of odd tiles | e_lo
+    unsigned char* w_s = e_s + 3 * e_bytes;
     FCtl* ctl = reinterpret_cast<FCtl*>(w_s + ((w_bytes + 1023) & ~1023));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int c0 = blockIdx.x * kFCs;
@@ -102,9 +105,11 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
     if (tid == 0) {
         mbar_init(smem_u32(&ctl->w_full), 1);
         for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->e_full[s]), 1); mbar_init(smem_u32(&ctl->e_empty[s]), 1); }
+        mbar_init(smem_u32(&ctl->elo_full), 1); mbar_init(smem_u32(&ctl->elo_empty), 1);
+        for (int s = 0; s < kFSlots; ++s) mbar_init(smem_u32(&ctl->s_free[s]), 1);
         for (int s = 0; s < 4; ++s) {
-            mbar_init(smem_u32(&ctl->d_full[s]), 1); mbar_init(smem_u32(&ctl->d_empty[s]), 1);
-            mbar_init(smem_u32(&ctl->g_done[s]), 1); mbar_init(smem_u32(&ctl->q_done[s]), 2);
+            for (int b2 = 0; b2 < 2; ++b2) { mbar_init(smem_u32(&ctl->d_full[s][b2]), 1); mbar_init(smem_u32(&ctl->g_done[s][b2]), 1); }
+            mbar_init(smem_u32(&ctl->q_done[s]), 2);
         }
         for (int s = 0; s < kFMaxRing; ++s) { mbar_init(smem_u32(&ctl->acc_full[s]), 1); mbar_init(smem_u32(&ctl->acc_empty[s]), kFEpiWarps); }
         mbar_init(smem_u32(&ctl->g_final), 1);
@@ -130,12 +135,14 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
             bulk_load(smem_u32(w_s), a.Wf + (int64_t)blockIdx.x * (w_bytes / 2), w_bytes, smem_u32(&ctl->w_full));
             for (int ti = 0; ti < nt; ++ti) {
                 const int buf = ti & 1;
+                // e_hi (dxhat and G) is double-buffered, e_lo (G only) is not: shared memory goes to the data slots
                 if (!mbar_wait(smem_u32(&ctl->e_empty[buf]), ((ti >> 1) & 1) ^ 1, abort, 1, ti)) break;
-                const uint32_t full = smem_u32(&ctl->e_full[buf]);
-                mbar_expect_tx(full, 2 * e_bytes);
                 const int64_t off = (int64_t)tile_of(ti) * a.Kp * kFTok;             // elements
-                bulk_load(smem_u32(e_s + buf * 2 * e_bytes), a.ehi + off, e_bytes, full);
-                bulk_load(smem_u32(e_s + buf * 2 * e_bytes + e_bytes), a.elo + off, e_bytes, full);
+                mbar_expect_tx(smem_u32(&ctl->e_full[buf]), e_bytes);
+                bulk_load(smem_u32(e_s + buf * e_bytes), a.ehi + off, e_bytes, smem_u32(&ctl->e_full[buf]));
+                if (!mbar_wait(smem_u32(&ctl->elo_empty), (ti & 1) ^ 1, abort, 12, ti)) break;
+                mbar_expect_tx(smem_u32(&ctl->elo_full), e_bytes);
+                bulk_load(smem_u32(e_s + 2 * e_bytes), a.elo + off, e_bytes, smem_u32(&ctl->elo_full));
             }
         }
     } else if (warp == 2) {
@@ -150,16 +157,19 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
             bool ok = true;
             for (int ti = 0; ti < nt && ok; ++ti) {
                 for (int q = 0; q < 4 && ok; ++q) {
-                    if (lane == 0) ok = mbar_wait(smem_u32(&ctl->d_empty[q]), (ti & 1) ^ 1, abort, 2, ti * 4 + q);
+                    // load number li goes to slot li % kFSlots: the slot that quadrant q - 1 hands back, so that the
+                    // load of a quadrant's next tile is on its way while the quadrant still works on this one
+                    const int li = ti * 4 + q, sl = li % kFSlots;
+                    if (lane == 0) ok = mbar_wait(smem_u32(&ctl->s_free[sl]), ((li / kFSlots) & 1) ^ 1, abort, 2, li);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
-                    const uint32_t full = smem_u32(&ctl->d_full[q]);
+                    const uint32_t full = smem_u32(&ctl->d_full[q][ti & 1]);
                     if (lane == 0) mbar_expect_tx(full, kSlot);
                     __syncwarp();
                     const int row = tile_of(ti) * kFTok + q * 32;
                     const int next_row = tile_of(ti + 1) * kFTok + q * 32;
                     if (lane < kBoxes) {
-                        tma_load_2d(smem_u32(slots + q * kSlot) + b * kFBox, mp, full, col, row);
+                        tma_load_2d(smem_u32(slots + sl * kSlot) + b * kFBox, mp, full, col, row);
                         // the quadrant's next boxes start their way from HBM to L2 now: a slot is busy for a
                         // whole load + compute + store round, too long to hide the HBM latency with four slots
                         if (ti + 1 < nt) tma_prefetch_2d(mp, col, next_row);
@@ -171,7 +181,7 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
         // ---- MMA issuer ------------------------------------------------------------------------------
         if (lane == 0 && nt > 0) {
             const uint32_t idesc_d = umma_idesc_mn(128, kDW, 0, 0);
-            const uint32_t idesc_g = umma_idesc_mn(128, 2 * a.Kp, 1, 1);
+            const uint32_t idesc_g = umma_idesc_mn(128, a.Kp, 1, 1);
             const int ksteps = a.Kp >> 4;
             const uint32_t w_half = (uint32_t)(a.Kp >> 3) * (kDW * 16);          // bytes of one channel half of W'
             bool ok = mbar_wait(smem_u32(&ctl->w_full), 0, abort, 3, 0);
@@ -180,7 +190,8 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                 const int buf = ti & 1;
                 ok = mbar_wait(smem_u32(&ctl->e_full[buf]), (ti >> 1) & 1, abort, 4, ti);
                 if (!ok) break;
-                const uint32_t eh = smem_u32(e_s + buf * 2 * e_bytes);        // e_lo follows e_hi
+                const uint32_t eh = smem_u32(e_s + buf * e_bytes), el = smem_u32(e_s + 2 * e_bytes);
+                bool lo_ready = false;
                 for (int half = 0; half < 2 && ok; ++half) {
                     const int u = 2 * ti + half, rr = u % a.ring;
                     ok = mbar_wait(smem_u32(&ctl->acc_empty[rr]), ((u / a.ring) & 1) ^ 1, abort, 5, u);
@@ -205,28 +216,36 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                         break;
                     }
                     for (int q = 0; q < 4; ++q) {
-                        if (!(pending & (1u << q)) || !mbar_try_wait(smem_u32(&ctl->d_full[q]), ti & 1)) continue;
+                        if (!(pending & (1u << q)) || !mbar_try_wait(smem_u32(&ctl->d_full[q][ti & 1]), (ti >> 1) & 1)) continue;
+                        if (!lo_ready) {
+                            ok = mbar_wait(smem_u32(&ctl->elo_full), ti & 1, abort, 13, ti);
+                            if (!ok) break;
+                            lo_ready = true;
+                        }
                         pending &= ~(1u << q);
                         tc_fence_after();
-                        const uint32_t xs = smem_u32(slots + q * kSlot);
+                        const uint32_t xs = smem_u32(slots + ((ti * 4 + q) % kFSlots) * kSlot);
 #pragma unroll
                         for (int ks = 0; ks < 2; ++ks) {
-                            // B: columns of e_hi then of e_lo = N (8-column groups 2 KB apart), tokens = K (8-token
-                            // groups 128 B apart)
-                            const uint64_t bd = smem_desc(eh + (uint32_t)(q * 32 + ks * 16) * 16, 128, 2048, 0);
+                            // B: columns of e_hi, of e_lo = N (8-column groups 2 KB apart), tokens = K (8-token groups
+                            // 128 B apart); the two products go to the two halves of the accumulator's columns
+                            const uint32_t eo = (uint32_t)(q * 32 + ks * 16) * 16;
+                            const uint64_t bh = smem_desc(eh + eo, 128, 2048, 0), bl = smem_desc(el + eo, 128, 2048, 0);
 #pragma unroll
                             for (int ac = 0; ac < kNA; ++ac) {
                                 // A: 128 rows = the 64 channels of two streams (boxes 4 KB apart), 8-token groups 1 KB apart
                                 const uint64_t ad = smem_desc(xs + ac * 2 * kFBox + ks * 2048, kFBox, 1024, 2);
-                                tc_mma(tmem_g + ac * 2 * a.Kp, ad, bd, idesc_g, g_started ? 1u : 0u);
+                                tc_mma(tmem_g + ac * 2 * a.Kp, ad, bh, idesc_g, g_started ? 1u : 0u);
+                                tc_mma(tmem_g + ac * 2 * a.Kp + a.Kp, ad, bl, idesc_g, g_started ? 1u : 0u);
                             }
                             g_started = true;
                         }
-                        tc_commit(smem_u32(&ctl->g_done[q]));
+                        tc_commit(smem_u32(&ctl->g_done[q][ti & 1]));
                     }
                 }
                 if (!ok) break;
                 tc_commit(smem_u32(&ctl->e_empty[buf]));
+                tc_commit(smem_u32(&ctl->elo_empty));
             }
             if (ok) tc_commit(smem_u32(&ctl->g_final));
         }
@@ -234,7 +253,6 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
         // ---- epilogue: thread = token; the two warps of a lane quadrant take 16 channels of each half ----
         const int quad = warp & 3;
         const int hw = (warp - 3) >> 2;
-        unsigned char* slot = slots + quad * kSlot;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         float kap = 0.f, hp[N_], hr[N_][N_];
         bool ok = true;
@@ -251,9 +269,10 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
 #pragma unroll
                     for (int j = 0; j < N_; ++j) hr[i][j] = live ? __ldg(a.H_res + t * N_ * N_ + i * N_ + j) : 0.f;
             }
-            ok = mbar_wait(smem_u32(&ctl->d_full[quad]), ti & 1, abort, 7, ti);
+            unsigned char* slot = slots + ((ti * 4 + quad) % kFSlots) * kSlot;
+            ok = mbar_wait(smem_u32(&ctl->d_full[quad][ti & 1]), (ti >> 1) & 1, abort, 7, ti);
             // MODE 0 writes dx over x itself: the G MMAs must have read the boxes
-            if (MODE == 0 && ok) ok = mbar_wait(smem_u32(&ctl->g_done[quad]), ti & 1, abort, 8, ti);
+            if (MODE == 0 && ok) ok = mbar_wait(smem_u32(&ctl->g_done[quad][ti & 1]), (ti >> 1) & 1, abort, 8, ti);
             for (int half = 0; half < 2; ++half) {
                 const int u = 2 * ti + half, rr = u % a.ring;
                 if (ok) ok = mbar_wait(smem_u32(&ctl->acc_full[rr]), (u / a.ring) & 1, abort, 9, u);
@@ -322,9 +341,9 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 }
                 // the slot goes back once the G MMAs have read its x boxes as well (long done by now)
-                if (MODE != 0 && lane == 0 && oks) oks = mbar_wait(smem_u32(&ctl->g_done[quad]), ti & 1, abort, 8, ti);
+                if (MODE != 0 && lane == 0 && oks) oks = mbar_wait(smem_u32(&ctl->g_done[quad][ti & 1]), (ti >> 1) & 1, abort, 8, ti);
                 oks = __all_sync(0xffffffffu, oks);
-                if (oks && lane == 0) mbar_arrive(smem_u32(&ctl->d_empty[quad]));
+                if (oks && lane == 0) mbar_arrive(smem_u32(&ctl->s_free[(ti * 4 + quad) % kFSlots]));
             }
             __syncwarp();
         }
@@ -395,7 +414,7 @@ __global__ void __launch_bounds__(256) pack_wf_k(int n, int C, int N, int Kp, co
 static int ftc_smem_bytes(int n, int Kp, int mode) {
     const int boxes = mode == 1 ? 2 * n + 1 : (mode == 2 ? 2 * n : n);
     const int w_bytes = Kp * n * kFCs * 2;
-    return 4 * boxes * kFBox + 4 * (Kp * kFTok * 2) + ((w_bytes + 1023) & ~1023) + (int)sizeof(FCtl) + 1024;
+    return kFSlots * boxes * kFBox + 3 * (Kp * kFTok * 2) + ((w_bytes + 1023) & ~1023) + (int)sizeof(FCtl) + 1024;
 }
 
 // Fills the plan's fields of this kernel: usable when the slices are whole (C a multiple of 64), the G
