@@ -233,8 +233,11 @@ MHCLITE_API size_t mhclite_step_host_bytes(int n, int C, int64_t T);
  * activations in HOST memory and the sublayer's results supplied: copies x, y, g = dL/dx_next and
  * du = dL/du host->device into `staging`, runs pre_fwd_fused, postres_fwd, postres_bwd and
  * tail_bwd_fused, and copies u, x_next, dy, dx device->host.  Parameters and their gradients stay on
- * the device.  Host buffers should be page-locked for the copies to be asynchronous; results are valid
- * once `stream` has been synchronised.  `staging` is caller-owned device scratch (256-byte aligned) of
+ * the device.  The tokens are processed in up to eight chunks so that the copies in, the kernels and the
+ * copies out of successive chunks overlap (two copy streams owned by the context, made on the first call
+ * and tied to `stream` by events: the call stays ordered on `stream`); the parameter gradients of the chunks
+ * add up.  Host buffers should be page-locked for the copies to be asynchronous; results are valid once
+ * `stream` has been synchronised.  `staging` is caller-owned device scratch (256-byte aligned) of
  * at least mhclite_step_host_bytes; the context's workspace must be attached as well. */
 MHCLITE_API int mhclite_step_host(mhclite_ctx* ctx, int64_t T,
                       const mhclite_bf16* x_host, const mhclite_bf16* y_host,

@@ -11,6 +11,7 @@
 namespace mhcl {
 
 constexpr int kMaxN = 5;          // residual streams supported: 2..5
+#define MHCLITE_STEP_CHUNKS 8      // token chunks that mhclite_step_host keeps in flight
 constexpr int kMaxFact = 120;     // 5!
 constexpr int kWarp = 32;
 
@@ -28,6 +29,9 @@ struct mhclite_ctx {
     bool timing;                  // record CUDA events around the main kernels (mhclite_set_kernel_timing)
     cudaEvent_t ev[MHCLITE_KERNEL_COUNT][2];
     mutable bool ev_recorded[MHCLITE_KERNEL_COUNT];   // the pair has bracketed at least one launch
+    // mhclite_step_host: copy-in and copy-out streams and the events that chain its token chunks (made on first use)
+    cudaStream_t copy_in, copy_out;
+    cudaEvent_t ev_fork, ev_join, ev_in[MHCLITE_STEP_CHUNKS], ev_cmp[MHCLITE_STEP_CHUNKS];
     char err[256];
 };
 

@@ -198,6 +198,8 @@ int mhclite_create(mhclite_ctx** out, int n, int C, int device) {
     ctx->n = n; ctx->C = C; ctx->device = device; ctx->nfact = ipow_fact(n);
     ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->err[0] = 0; ctx->launches = 0; ctx->timing = false; ctx->status_word = nullptr;
     for (int k = 0; k < MHCLITE_KERNEL_COUNT; ++k) { ctx->ev[k][0] = ctx->ev[k][1] = nullptr; ctx->ev_recorded[k] = false; }
+    ctx->copy_in = ctx->copy_out = nullptr; ctx->ev_fork = ctx->ev_join = nullptr;
+    for (int k = 0; k < MHCLITE_STEP_CHUNKS; ++k) ctx->ev_in[k] = ctx->ev_cmp[k] = nullptr;
     {
         DeviceGuard g(device);
         cudaError_t e = g.err;
@@ -214,6 +216,14 @@ int mhclite_destroy(mhclite_ctx* ctx) {
     for (int k = 0; k < MHCLITE_KERNEL_COUNT; ++k)
         for (int e = 0; e < 2; ++e)
             if (ctx->ev[k][e]) cudaEventDestroy(ctx->ev[k][e]);
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    for (int k = 0; k < MHCLITE_STEP_CHUNKS; ++k) {
+        if (ctx->ev_in[k]) cudaEventDestroy(ctx->ev_in[k]);
+        if (ctx->ev_cmp[k]) cudaEventDestroy(ctx->ev_cmp[k]);
+    }
     delete ctx;
     return MHCLITE_OK;
 }
@@ -556,27 +566,62 @@ int mhclite_step_host(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x_host, c
         return fail(ctx, MHCLITE_ERR_WORKSPACE, "staging of %zu bytes needed, %zu given", s.bytes, staging_bytes);
     MHCL_DEVICE(ctx);
     cudaStream_t st = (cudaStream_t)stream;
-    const size_t big = (size_t)T * ctx->n * ctx->C * sizeof(mhclite_bf16), small = (size_t)T * ctx->C * sizeof(mhclite_bf16);
     int rc;
-#define MHCL_COPY(dst, src, bytes, kind) \
-    if ((rc = check_cuda(ctx, cudaMemcpyAsync(dst, src, bytes, kind, st), "cudaMemcpyAsync " #dst))) return rc
-    MHCL_COPY(s.x, x_host, big, cudaMemcpyHostToDevice);
-    if ((rc = mhclite_pre_fwd_fused(ctx, T, s.x, W, b, alpha, gain, eps, s.H_res, s.H_pre, s.H_post, s.a, s.p, s.rstd,
-                                    s.u, stream))) return rc;
-    MHCL_COPY(u_host, s.u, small, cudaMemcpyDeviceToHost);
-    MHCL_COPY(s.y, y_host, small, cudaMemcpyHostToDevice);
-    if ((rc = mhclite_postres_fwd(ctx, T, s.x, s.y, s.H_res, s.H_post, s.x_next, stream))) return rc;
-    MHCL_COPY(x_next_host, s.x_next, big, cudaMemcpyDeviceToHost);
-    MHCL_COPY(s.g, g_host, big, cudaMemcpyHostToDevice);
-    if ((rc = mhclite_postres_bwd(ctx, T, s.x, s.y, s.H_res, s.H_post, s.g, s.dy, s.dH_res, s.dH_post, nullptr, 0,
-                                  stream))) return rc;
-    MHCL_COPY(dy_host, s.dy, small, cudaMemcpyDeviceToHost);
-    MHCL_COPY(s.du, du_host, small, cudaMemcpyHostToDevice);
-    if ((rc = mhclite_tail_bwd_fused(ctx, T, s.x, W, alpha, gain, eps, s.a, s.p, s.rstd, s.H_res, s.H_pre, s.H_post,
-                                     s.g, s.du, s.dH_res, s.dH_post, s.dx, dW, db, dalpha, dgain, accumulate_params,
-                                     stream))) return rc;
-    MHCL_COPY(dx_host, s.dx, big, cudaMemcpyDeviceToHost);
-#undef MHCL_COPY
+    // copy streams and events of the context, made on the first call
+    if (!ctx->copy_in) {
+        if ((rc = check_cuda(ctx, cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking), "copy-in stream"))) return rc;
+        if ((rc = check_cuda(ctx, cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking), "copy-out stream"))) return rc;
+        cudaEvent_t* evs[2] = {&ctx->ev_fork, &ctx->ev_join};
+        for (cudaEvent_t* e : evs)
+            if ((rc = check_cuda(ctx, cudaEventCreateWithFlags(e, cudaEventDisableTiming), "cudaEventCreate"))) return rc;
+        for (int k = 0; k < MHCLITE_STEP_CHUNKS; ++k) {
+            if ((rc = check_cuda(ctx, cudaEventCreateWithFlags(&ctx->ev_in[k], cudaEventDisableTiming), "cudaEventCreate"))) return rc;
+            if ((rc = check_cuda(ctx, cudaEventCreateWithFlags(&ctx->ev_cmp[k], cudaEventDisableTiming), "cudaEventCreate"))) return rc;
+        }
+    }
+    // Tokens are independent: the step runs in up to MHCLITE_STEP_CHUNKS chunks of tokens, so that the
+    // host->device copies of chunk c + 1 (copy-in stream), the kernels of chunk c (the caller's stream) and
+    // the device->host copies of chunk c - 1 (copy-out stream) overlap; PCIe carries both directions at once.
+    // The parameter gradients of the chunks add up (accumulate from the second chunk on).
+    int64_t chunk = round_up64((T + MHCLITE_STEP_CHUNKS - 1) / MHCLITE_STEP_CHUNKS, 128);
+    if (chunk < 256) chunk = 256;
+    const int nchunks = (int)((T + chunk - 1) / chunk);
+    const int n = ctx->n, C = ctx->C, nf = ctx->nfact, N = n_cols(n, 0);
+#define MHCL_CUDA(call, what) if ((rc = check_cuda(ctx, call, what))) return rc
+    MHCL_CUDA(cudaEventRecord(ctx->ev_fork, st), "event record");
+    MHCL_CUDA(cudaStreamWaitEvent(ctx->copy_in, ctx->ev_fork, 0), "stream wait");
+    MHCL_CUDA(cudaStreamWaitEvent(ctx->copy_out, ctx->ev_fork, 0), "stream wait");
+    for (int c = 0; c < nchunks; ++c) {
+        const int64_t t0 = (int64_t)c * chunk, Tc = (t0 + chunk <= T) ? chunk : T - t0;
+        const size_t big = (size_t)Tc * n * C * sizeof(mhclite_bf16), small = (size_t)Tc * C * sizeof(mhclite_bf16);
+        const int64_t ob = t0 * n * C, os = t0 * C;            // element offsets of [T][n][C] and [T][C] tensors
+        MHCL_CUDA(cudaMemcpyAsync(s.x + ob, x_host + ob, big, cudaMemcpyHostToDevice, ctx->copy_in), "copy x");
+        MHCL_CUDA(cudaMemcpyAsync(s.y + os, y_host + os, small, cudaMemcpyHostToDevice, ctx->copy_in), "copy y");
+        MHCL_CUDA(cudaMemcpyAsync(s.g + ob, g_host + ob, big, cudaMemcpyHostToDevice, ctx->copy_in), "copy g");
+        MHCL_CUDA(cudaMemcpyAsync(s.du + os, du_host + os, small, cudaMemcpyHostToDevice, ctx->copy_in), "copy du");
+        MHCL_CUDA(cudaEventRecord(ctx->ev_in[c], ctx->copy_in), "event record");
+        MHCL_CUDA(cudaStreamWaitEvent(st, ctx->ev_in[c], 0), "stream wait");
+        float *H_res = s.H_res + t0 * n * n, *H_pre = s.H_pre + t0 * n, *H_post = s.H_post + t0 * n, *av = s.a + t0 * nf,
+              *pv = s.p + t0 * N, *rs = s.rstd + t0, *dH_res = s.dH_res + t0 * n * n, *dH_post = s.dH_post + t0 * n;
+        if ((rc = mhclite_pre_fwd_fused(ctx, Tc, s.x + ob, W, b, alpha, gain, eps, H_res, H_pre, H_post, av, pv, rs, s.u + os,
+                                        stream))) return rc;
+        if ((rc = mhclite_postres_fwd(ctx, Tc, s.x + ob, s.y + os, H_res, H_post, s.x_next + ob, stream))) return rc;
+        if ((rc = mhclite_postres_bwd(ctx, Tc, s.x + ob, s.y + os, H_res, H_post, s.g + ob, s.dy + os, dH_res, dH_post, nullptr,
+                                      0, stream))) return rc;
+        if ((rc = mhclite_tail_bwd_fused(ctx, Tc, s.x + ob, W, alpha, gain, eps, av, pv, rs, H_res, H_pre, H_post, s.g + ob,
+                                         s.du + os, dH_res, dH_post, s.dx + ob, dW, db, dalpha, dgain,
+                                         (c > 0 || accumulate_params) ? 1 : 0, stream))) return rc;
+        MHCL_CUDA(cudaEventRecord(ctx->ev_cmp[c], st), "event record");
+        MHCL_CUDA(cudaStreamWaitEvent(ctx->copy_out, ctx->ev_cmp[c], 0), "stream wait");
+        MHCL_CUDA(cudaMemcpyAsync(u_host + os, s.u + os, small, cudaMemcpyDeviceToHost, ctx->copy_out), "copy u");
+        MHCL_CUDA(cudaMemcpyAsync(x_next_host + ob, s.x_next + ob, big, cudaMemcpyDeviceToHost, ctx->copy_out), "copy x_next");
+        MHCL_CUDA(cudaMemcpyAsync(dy_host + os, s.dy + os, small, cudaMemcpyDeviceToHost, ctx->copy_out), "copy dy");
+        MHCL_CUDA(cudaMemcpyAsync(dx_host + ob, s.dx + ob, big, cudaMemcpyDeviceToHost, ctx->copy_out), "copy dx");
+    }
+    // join: everything, the last copies included, is ordered before later work on the caller's stream
+    MHCL_CUDA(cudaEventRecord(ctx->ev_join, ctx->copy_out), "event record");
+    MHCL_CUDA(cudaStreamWaitEvent(st, ctx->ev_join, 0), "stream wait");
+#undef MHCL_CUDA
     return MHCLITE_OK;
 }
 

@@ -219,3 +219,33 @@ def test_kernel_timing_of_a_kernel_off_the_path_is_an_argument_error():
     assert G.ctx.kernel_time_ms(0) > 0.0
     G.forward(True); torch.cuda.synchronize()
     compare_forward(G, oracle_fwd(inp))
+
+
+@pytest.mark.parametrize("n,C,T", [(4, 128, 700), (3, 72, 130)])
+def test_step_from_host_buffers(n, C, T):
+    # the whole step through mhclite_step_host: pinned host activations in, host activations out, in chunks of
+    # tokens whose copies and kernels overlap (700 tokens = three chunks, the last one ragged)
+    inp = synth.make_layer_inputs(n, C, T, seed=40 + n, bias_std=0.1, gain_std=0.1)
+    G = GpuLayer(inp)
+    B, P = G.B, G.P
+    pin = lambda t: t.cpu().pin_memory()
+    hx, hy, hg, hdu = pin(G.x), pin(G.y), pin(G.g), pin(G.du)
+    hu, hxn, hdy, hdx = (torch.zeros_like(t, device="cpu").pin_memory() for t in (B.u, B.x_next, B.dy, B.dx))
+    run = lambda acc: G.ctx.step_host(hx, hy, hg, hdu, P.W, P.b, P.alpha, P.gain, 1e-6, hu, hxn, hdy, hdx,
+                                      B.dW, B.db, B.dalpha, B.dgain, acc)
+    run(False)
+    torch.cuda.synchronize()
+    fw, bw = oracle_fwd(inp), oracle_bwd(inp)
+    f64 = lambda t: t.float().numpy().astype(np.float64)
+    check_bf16("u", f64(hu), fw["u"])
+    check_bf16("x_next", f64(hxn), fw["x_next"])
+    check_bf16("dy", f64(hdy), bw["dy"])
+    check_bf16("dx", f64(hdx), bw["dx"], extra=dxhat_allowance(inp, bw["dz"]))
+    for name, got in (("dW", B.dW), ("db", B.db), ("dalpha", B.dalpha), ("dgain", B.dgain)):
+        check_f32(name, host(got), bw[name], 1e-3)
+    run(True)                                       # accumulate_params adds a second copy of the gradients
+    torch.cuda.synchronize()
+    for name, got in (("dW", B.dW), ("db", B.db), ("dalpha", B.dalpha), ("dgain", B.dgain)):
+        check_f32(name + " x2", host(got), 2 * bw[name], 1e-3)
+    check_bf16("dx again", f64(hdx), bw["dx"], extra=dxhat_allowance(inp, bw["dz"]))
+    G.ctx.device_status()
