@@ -224,6 +224,17 @@ MHCLITE_API int mhc_sk20_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhcli
 MHCLITE_API int mhclite_ds_gap(mhclite_ctx* ctx, int64_t T, const float* H_res, float* l1_err, float* colsum_dev,
                    void* stream);
 
+/* Product of the residual mappings over depth (paper Section 3.1: prod_l H_res_l must stay doubly stochastic
+ * for the signal to keep its norm across layers).  Per token: P[t] <- H_res[t] P[t], later layers multiplying
+ * on the left as x_{l+1} = H_l x_l composes; with first != 0, P[t] <- H_res[t].  P is [T][n][n] fp32, updated
+ * in place, and must not alias H_res.  Its gap is read with mhclite_ds_gap(P). */
+MHCLITE_API int mhclite_depth_product(mhclite_ctx* ctx, int64_t T, const float* H_res, float* P, int first,
+                                      void* stream);
+
+/* Relative range of paper Eq. (3), per token: nu[t] = (smallest positive entry) / (largest entry) of the
+ * n x n matrix X[t] (0 when no entry is positive); 1/nu bounds the Sinkhorn-Knopp iteration count. */
+MHCLITE_API int mhclite_relative_range(mhclite_ctx* ctx, int64_t T, const float* X, float* nu, void* stream);
+
 /* ---- whole step from host buffers -------------------------------------------------------------- */
 
 /* Bytes of device staging mhclite_step_host needs for T tokens. */

@@ -56,6 +56,8 @@ SIGNATURES = {
     "mhc_sk20_tail_bwd_fused": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _i, _p, _p, _p, _p, _p, _p, _p, _p, _p,
                                      _p, _p, _p, _p, _p, _i, _p]),
     "mhclite_ds_gap": (_i, [_p, _i64, _p, _p, _p, _p]),
+    "mhclite_depth_product": (_i, [_p, _i64, _p, _p, _i, _p]),
+    "mhclite_relative_range": (_i, [_p, _i64, _p, _p, _p]),
     "mhclite_step_host_bytes": (_sz, [_i, _i, _i64]),
     "mhclite_step_host": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p, _i,
                                _p, _sz, _p]),
@@ -306,6 +308,17 @@ class MhcLite:
             u_host.data_ptr(), x_next_host.data_ptr(), dy_host.data_ptr(), dx_host.data_ptr(),
             self._ptr(dW, f), self._ptr(db, f), self._ptr(dalpha, f), self._ptr(dgain, f), int(accumulate_params),
             base, need, self._stream()), "mhclite_step_host")
+
+    def depth_product(self, H_res, P, first=False):
+        """P[t] <- H_res[t] P[t] in place (P[t] <- H_res[t] when first)."""
+        f = self._torch.float32
+        self._check(self.lib.mhclite_depth_product(self._h, H_res.shape[0], self._ptr(H_res, f), self._ptr(P, f),
+                                                   int(first), self._stream()), "mhclite_depth_product")
+
+    def relative_range(self, X, nu):
+        f = self._torch.float32
+        self._check(self.lib.mhclite_relative_range(self._h, X.shape[0], self._ptr(X, f), self._ptr(nu, f),
+                                                    self._stream()), "mhclite_relative_range")
 
     def ds_gap(self, H_res, l1_err=None, colsum_dev=None):
         f = self._torch.float32

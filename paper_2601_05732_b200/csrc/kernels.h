@@ -16,6 +16,8 @@ void launch_premix_bwd(const mhclite_ctx* c, int64_t T, const void* x, const flo
 void launch_tail_mix(const mhclite_ctx* c, int64_t T, const void* x, const void* g, const void* du, const float* H_res,
                      const float* H_pre, float* dH_pre, void* dx, cudaStream_t s);
 void launch_ds_gap(const mhclite_ctx* c, int64_t T, const float* H_res, float* l1, float* cdev, cudaStream_t s);
+void launch_depth_product(const mhclite_ctx* c, int64_t T, const float* H_res, float* P, int first, cudaStream_t s);
+void launch_relative_range(const mhclite_ctx* c, int64_t T, const float* X, float* nu, cudaStream_t s);
 
 // proj_kernels.cu : RMSNorm statistics + the skinny projection and its gradient
 // proj_mma.cu: W' = diag(gain) W packed as bf16 hi/lo MMA fragments; qpart[s][t][c] = partial x W' of K slice s,

@@ -519,6 +519,27 @@ int mhclite_ds_gap(mhclite_ctx* ctx, int64_t T, const float* H_res, float* l1_er
     return MHCLITE_OK;
 }
 
+int mhclite_depth_product(mhclite_ctx* ctx, int64_t T, const float* H_res, float* P, int first, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, P);
+    if (H_res == P) return fail(ctx, MHCLITE_ERR_BAD_ARG, "H_res and P must not alias");
+    MHCL_DEVICE(ctx);
+    launch_depth_product(ctx, T, H_res, P, first, (cudaStream_t)stream);
+    MHCL_LAUNCH_CHECK(ctx, "depth_product");
+    return MHCLITE_OK;
+}
+
+int mhclite_relative_range(mhclite_ctx* ctx, int64_t T, const float* X, float* nu, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, X); MHCL_PTR(ctx, nu);
+    MHCL_DEVICE(ctx);
+    launch_relative_range(ctx, T, X, nu, (cudaStream_t)stream);
+    MHCL_LAUNCH_CHECK(ctx, "relative_range");
+    return MHCLITE_OK;
+}
+
 // ---- whole step from host buffers ----------------------------------------------------------------
 namespace {
 struct StepStaging {

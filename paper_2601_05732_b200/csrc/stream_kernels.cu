@@ -285,6 +285,38 @@ __global__ void ds_gap_k(int64_t T, int n, const float* __restrict__ H, float* l
     if (cdev) cdev[t] = cmax;
 }
 
+// Product of the residual mappings over depth, one thread per token: P <- H P (later layers multiply on the
+// left, as x_{l+1} = H_l x_l composes); first layer: P <- H.
+__global__ void depth_product_k(int64_t T, int n, const float* __restrict__ H, float* P, int first) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    const float* h = H + t * n * n;
+    float* p = P + t * n * n;
+    float out[kMaxN * kMaxN];
+    for (int i = 0; i < n; ++i)
+        for (int k = 0; k < n; ++k) {
+            float acc = 0.f;
+            if (first) acc = h[i * n + k];
+            else for (int j = 0; j < n; ++j) acc = fmaf(h[i * n + j], p[j * n + k], acc);
+            out[i * n + k] = acc;
+        }
+    for (int e = 0; e < n * n; ++e) p[e] = out[e];
+}
+
+// Eq. (3): nu = smallest positive entry / largest entry of each n x n matrix (0 when no entry is positive).
+__global__ void relative_range_k(int64_t T, int n, const float* __restrict__ X, float* __restrict__ nu) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    const float* x = X + t * n * n;
+    float lo = 3.4e38f, hi = -3.4e38f;
+    for (int e = 0; e < n * n; ++e) {
+        const float v = x[e];
+        hi = fmaxf(hi, v);
+        if (v > 0.f) lo = fminf(lo, v);
+    }
+    nu[t] = (hi > 0.f) ? lo / hi : 0.f;
+}
+
 // ---- launchers -----------------------------------------------------------------------------------
 static int grid_for(int64_t items, int sm_count, int per_sm) {
     int64_t blocks = (items + kThreads - 1) / kThreads;
@@ -348,6 +380,16 @@ void launch_ds_gap(const mhclite_ctx* c, int64_t T, const float* H_res, float* l
     c->launches += 1;
     const int grid = (int)((T + 127) / 128);
     ds_gap_k<<<grid, 128, 0, s>>>(T, c->n, H_res, l1, cdev);
+}
+
+void launch_depth_product(const mhclite_ctx* c, int64_t T, const float* H_res, float* P, int first, cudaStream_t s) {
+    c->launches += 1;
+    depth_product_k<<<(unsigned)((T + 127) / 128), 128, 0, s>>>(T, c->n, H_res, P, first);
+}
+
+void launch_relative_range(const mhclite_ctx* c, int64_t T, const float* X, float* nu, cudaStream_t s) {
+    c->launches += 1;
+    relative_range_k<<<(unsigned)((T + 127) / 128), 128, 0, s>>>(T, c->n, X, nu);
 }
 
 }  // namespace mhcl

@@ -249,3 +249,31 @@ def test_step_from_host_buffers(n, C, T):
         check_f32(name + " x2", host(got), 2 * bw[name], 1e-3)
     check_bf16("dx again", f64(hdx), bw["dx"], extra=dxhat_allowance(inp, bw["dz"]))
     G.ctx.device_status()
+
+
+@pytest.mark.parametrize("n", [2, 3, 4, 5])
+def test_depth_product_and_relative_range(n):
+    # Section 3.1 diagnostics in the library's kernels: prod_l H_l per token (later layers on the left) and
+    # Eq. (3)'s nu, against the oracle on random doubly stochastic and random positive matrices
+    T, depth = 300, 6
+    rng = np.random.default_rng(60 + n)
+    nf = math.factorial(n)
+    Hs = [O.hres_from_weights(rng.dirichlet(np.ones(nf) * 0.3, size=T), n).astype(np.float32) for _ in range(depth)]
+    ctx = GpuLayer(synth.make_layer_inputs(n, 8, 4, seed=1)).ctx
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(DEV)
+    P = torch.empty(T, n, n, device=DEV)
+    for l, H in enumerate(Hs):
+        ctx.depth_product(dev(H), P, first=(l == 0))
+    torch.cuda.synchronize()
+    ref = O.depth_product([H.astype(np.float64) for H in Hs])
+    assert np.abs(host(P) - ref).max() < 1e-6
+    l1 = torch.empty(T, device=DEV); ctx.ds_gap(P, l1, None); torch.cuda.synchronize()
+    assert float(l1.max()) < depth * 4e-6                      # products of doubly stochastic matrices stay so
+    X = rng.uniform(0.0, 1.0, size=(T, n, n)).astype(np.float32)
+    X[rng.uniform(size=X.shape) < 0.2] = 0.0                   # zeros are skipped by Eq. (3)
+    X[0] = 0.0                                                 # degenerate: no positive entry
+    nu = torch.empty(T, device=DEV); ctx.relative_range(dev(X), nu); torch.cuda.synchronize()
+    ok = X.reshape(T, -1).max(axis=1) > 0
+    ref_nu = O.relative_range(X[ok].astype(np.float64))
+    np.testing.assert_allclose(host(nu)[ok], ref_nu, rtol=1e-6)
+    assert float(nu[0]) == 0.0
