@@ -34,7 +34,8 @@ void launch_proj_bwd_dw(const mhclite_ctx* c, int64_t T, int N, int Npad, const 
                         const float* gain, const float* e, float* G, float* dW, float* dgain, int acc,
                         cudaStream_t s);
 
-// proj_tc.cu : the same projection on tcgen05 / TMA / tensor memory (N <= 128 columns)
+// proj_tc.cu : the same projection on tcgen05 / TMA / tensor memory (up to 256 columns); tail_tc.cu : the
+// backward of wide projections (n = 5) on tcgen05
 bool tensor_maps_available();
 bool launch_tail_g_tc(const mhclite_ctx* c, int64_t T, const TailPlan& p, const void* x, const void* ehi,
                       const void* elo, float* Gpart, int* status, cudaStream_t s);

@@ -103,7 +103,8 @@ static int need_workspace(mhclite_ctx* ctx, int64_t T, int kind, Workspace* w) {
 }
 
 // RMSNorm statistics + projection partials of every entry point's forward: tcgen05 / TMA kernel when the
-// projection fits one UMMA tile (N <= 128 columns), the mma.sync kernel otherwise.
+// padded projection has at most 256 columns (hi and lo halves of W' side by side while they fit one instruction,
+// as two instructions into one accumulator beyond that), the mma.sync kernel otherwise.
 static int proj_forward(mhclite_ctx* ctx, int64_t T, int N, const Workspace& w, const ProjPlan& pp, const mhclite_bf16* x,
                         const float* W, const float* gain, cudaStream_t s) {
     if (proj_tc_supported(ctx->n, ctx->C, N)) {

@@ -171,7 +171,7 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                     if (lane < kBoxes) {
                         tma_load_2d(smem_u32(slots + sl * kSlot) + b * kFBox, mp, full, col, row);
                         // the quadrant's next boxes start their way from HBM to L2 now: a slot is busy for a
-                        // whole load + compute + store round, too long to hide the HBM latency with four slots
+                        // whole load + compute + store round, too long to hide the HBM latency with so few slots
                         if (ti + 1 < nt) tma_prefetch_2d(mp, col, next_row);
                     }
                 }
