@@ -51,17 +51,19 @@ struct TcSmem {                       // control block placed after the stage ri
 
 __global__ void __launch_bounds__(192, 1)
 proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw, int64_t T, int nchunks,
-              int chunks_per_split, int nq, int two_pass, int n_out, int stages, int tmem_cols,
+              int chunks_per_split, int nq, int two_pass, int mt, int n_out, int stages, int tmem_cols,
               float* __restrict__ qpart, float* __restrict__ ssq, int* __restrict__ status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     // the ring must start on a 1024-byte boundary (swizzle atoms)
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int w_bytes = 2 * nq * 128;                       // hi rows then lo rows
     const int umma_n = two_pass ? nq : 2 * nq;
-    const int stage_bytes = kTcXBytes + w_bytes;
+    const int x_bytes = mt * kTcXBytes;                     // mt token tiles of 128 share one W' stage
+    const int acc_cols = (umma_n + 31) & ~31;               // tensor-memory columns between the tiles' accumulators
+    const int stage_bytes = x_bytes + w_bytes;
     TcSmem* ctl = reinterpret_cast<TcSmem*>(smem + stages * stage_bytes);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t t0 = (int64_t)blockIdx.x * kTcTok;
+    const int64_t t0 = (int64_t)blockIdx.x * kTcTok * mt;
     const int split = blockIdx.y;
     const int c_begin = split * chunks_per_split;
     const int c_end = (c_begin + chunks_per_split < nchunks) ? c_begin + chunks_per_split : nchunks;
@@ -93,9 +95,9 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
                 mbar_expect_tx(full, stage_bytes);
                 const uint32_t dst = smem_u32(smem + s * stage_bytes);
                 const int k = (c_begin + i) * kTcK;
-                tma_load_2d(dst, &tmx, full, k, (int)t0);
-                tma_load_2d(dst + kTcXBytes, &tmw, full, k, 0);
-                if (two_pass) tma_load_2d(dst + kTcXBytes + nq * 128, &tmw, full, k, nq);   // box = Nq rows
+                for (int m = 0; m < mt; ++m) tma_load_2d(dst + m * kTcXBytes, &tmx, full, k, (int)t0 + m * kTcTok);
+                tma_load_2d(dst + x_bytes, &tmw, full, k, 0);
+                if (two_pass) tma_load_2d(dst + x_bytes + nq * 128, &tmw, full, k, nq);     // box = Nq rows
             }
         }
     } else if (warp == 1) {
@@ -108,12 +110,14 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t xa = smem_u32(smem + s * stage_bytes);
-                const uint64_t ad = smem_desc_k128(xa), bd = smem_desc_k128(xa + kTcXBytes);
-                const uint64_t bl = smem_desc_k128(xa + kTcXBytes + nq * 128);
+                const uint64_t bd = smem_desc_k128(xa + x_bytes), bl = smem_desc_k128(xa + x_bytes + nq * 128);
+                for (int m = 0; m < mt; ++m) {
+                    const uint64_t ad = smem_desc_k128(xa + m * kTcXBytes);
 #pragma unroll
-                for (int kk = 0; kk < kTcK / 16; ++kk) {    // 32 bytes further along the swizzled row per k-step
-                    tc_mma(tmem, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), idesc, (i > 0 || kk > 0) ? 1u : 0u);
-                    if (two_pass) tc_mma(tmem, ad + (uint64_t)(kk * 2), bl + (uint64_t)(kk * 2), idesc, 1u);
+                    for (int kk = 0; kk < kTcK / 16; ++kk) {    // 32 bytes further along the swizzled row per k-step
+                        tc_mma(tmem + m * acc_cols, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                        if (two_pass) tc_mma(tmem + m * acc_cols, ad + (uint64_t)(kk * 2), bl + (uint64_t)(kk * 2), idesc, 1u);
+                    }
                 }
                 tc_commit(smem_u32(&ctl->empty[s]));        // frees the stage when these MMAs have read it
             }
@@ -122,19 +126,24 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
     } else {
         const int quad = warp & 3;
         const int row = quad * 32 + lane;                   // this thread's token within the tile
-        float sq = 0.f;
+        float sqs[2] = {0.f, 0.f};                          // mt <= 2
         bool ok = true;
         for (int i = 0; i < nloc && ok; ++i) {
             const int s = i % stages;
             ok = mbar_wait(smem_u32(&ctl->full[s]), (i / stages) & 1, abort);
             if (!ok) break;
-            const unsigned char* xr = smem + s * stage_bytes + row * 128;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                float f[8];
-                unpack8(*reinterpret_cast<const uint4*>(xr + ((c ^ (row & 7)) << 4)), f);
+            for (int m = 0; m < 2; ++m) {
+                if (m < mt) {
+                    const unsigned char* xr = smem + s * stage_bytes + m * kTcXBytes + row * 128;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) sq = fmaf(f[e], f[e], sq);
+                    for (int c = 0; c < 8; ++c) {
+                        float f[8];
+                        unpack8(*reinterpret_cast<const uint4*>(xr + ((c ^ (row & 7)) << 4)), f);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) sqs[m] = fmaf(f[e], f[e], sqs[m]);
+                    }
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->empty[s]));
@@ -144,9 +153,13 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
         if (ok) {
             tc_fence_after();
             // hi columns [0, nq), lo columns [nq, 2 nq) (already added when the two halves share the accumulator)
-            const int64_t t = t0 + row;
+#pragma unroll
+            for (int m = 0; m < 2; ++m) {
+            if (m >= mt) break;
+            const int64_t t = t0 + m * kTcTok + row;
+            const float sq = sqs[m];
             float* qrow = qpart + ((int64_t)split * T + t) * n_out;
-            const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
+            const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16) + m * acc_cols;
             for (int c0 = 0; c0 < nq; c0 += 16) {
                 float hi[16], lo[16];
                 tc_ld16(lane_base + c0, hi);
@@ -165,6 +178,7 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
                 }
             }
             if (t < T) ssq[(int64_t)split * T + t] = sq;
+            }
         }
     }
     tc_fence_before();
@@ -268,19 +282,22 @@ bool launch_proj_fwd_tc(const mhclite_ctx* c, int64_t T, int N, const ProjPlan& 
     CUtensorMap tmx, tmw;
     if (!make_map(&tmx, x, (uint64_t)nC, (uint64_t)T, (uint64_t)nC, kTcTok)) return false;
     if (!make_map(&tmw, Wt, (uint64_t)Kpad, (uint64_t)(2 * nq), (uint64_t)Kpad, (uint32_t)umma_n)) return false;
-    const int stage_bytes = kTcXBytes + 2 * nq * 128;
+    // wide projections (two instructions per k-step) stream more bytes of W' than of x per 128 tokens: two token
+    // tiles then share each W' stage
+    const int mt = (two_pass && T > kTcTok) ? 2 : 1;
+    const int stage_bytes = mt * kTcXBytes + 2 * nq * 128;
     int stages = 100 * 1024 / stage_bytes;                   // two CTAs per SM when the stages are small enough
     if (stages > 6) stages = 6;
-    if (stages < 3) stages = (200 * 1024 / stage_bytes < 4) ? 200 * 1024 / stage_bytes : 4;
+    if (stages < 3) stages = (220 * 1024 / stage_bytes < 4) ? 220 * 1024 / stage_bytes : 4;   // one CTA per SM
     if (stages > 8) stages = 8;
     const int smem = stages * stage_bytes + (int)sizeof(TcSmem) + 1024;
     int tmem_cols = 32;
-    while (tmem_cols < umma_n) tmem_cols *= 2;
+    while (tmem_cols < (mt - 1) * ((umma_n + 31) & ~31) + umma_n) tmem_cols *= 2;
     c->launches += 1;
     KernelTimer timer_(c, MHCLITE_KERNEL_PROJ_FWD, s);
     cudaFuncSetAttribute(proj_fwd_tc_k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    dim3 grid((unsigned)((T + kTcTok - 1) / kTcTok), p.ksplit);
-    proj_fwd_tc_k<<<grid, 192, smem, s>>>(tmx, tmw, T, p.nchunks, p.chunks_per_split, nq, two_pass, p.Npad, stages,
+    dim3 grid((unsigned)((T + kTcTok * mt - 1) / (kTcTok * mt)), p.ksplit);
+    proj_fwd_tc_k<<<grid, 192, smem, s>>>(tmx, tmw, T, p.nchunks, p.chunks_per_split, nq, two_pass, mt, p.Npad, stages,
                                           tmem_cols, qpart, ssq, status);
     return true;
 }
