@@ -320,13 +320,13 @@ __global__ void __launch_bounds__(256) tail_finish_k(int nC, int N, int Kp, int 
     float dg = 0.f;
     for (int c = lane; c < N; c += 32) {
         float gv = 0.f;
-        for (int s0 = 0; s0 < splits; s0 += 16) {                 // sixteen loads in flight, then a fixed-order sum
-            float v[16];
+        for (int s0 = 0; s0 < splits; s0 += 8) {                  // eight loads in flight, then a fixed-order sum
+            float v[8];
 #pragma unroll
-            for (int k = 0; k < 16; ++k)
+            for (int k = 0; k < 8; ++k)
                 v[k] = (s0 + k < splits) ? __ldg(Gpart + ((int64_t)(s0 + k) * nC + m) * Kp + c) : 0.f;
 #pragma unroll
-            for (int k = 0; k < 16; k += 4) gv += (v[k] + v[k + 1]) + (v[k + 2] + v[k + 3]);
+            for (int k = 0; k < 8; k += 4) gv += (v[k] + v[k + 1]) + (v[k + 2] + v[k + 3]);
         }
         const int64_t i = (int64_t)m * N + c;
         dW[i] = ACC ? dW[i] + gm * gv : gm * gv;
