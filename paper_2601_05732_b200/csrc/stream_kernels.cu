@@ -38,7 +38,7 @@ __global__ void __launch_bounds__(kThreads) premix_fwd_k(int64_t T, int C8, cons
 // x_next[t,i,c] = sum_j H_res[t,i,j] x[t,j,c] + H_post[t,i] y[t,c]                          (Eq. (1))
 // ------------------------------------------------------------------------------------------------
 template <int N_>
-__global__ void __launch_bounds__(kThreads, 3) postres_fwd_k(int64_t T, int C8, const uint4* __restrict__ x,
+__global__ void __launch_bounds__(kThreads, (N_ <= 4 ? 3 : 2)) postres_fwd_k(int64_t T, int C8, const uint4* __restrict__ x,
                                                           const uint4* __restrict__ y, const float* __restrict__ H_res,
                                                           const float* __restrict__ H_post, uint4* __restrict__ x_next) {
     const int64_t total = T * C8;
