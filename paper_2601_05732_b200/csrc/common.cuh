@@ -167,6 +167,35 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
     v.x = pack2(f[0], f[1]); v.y = pack2(f[2], f[3]); v.z = pack2(f[4], f[5]); v.w = pack2(f[6], f[7]);
     return v;
 }
+// Two fp32 in one 64-bit register and the packed fused multiply-add of sm_100 (two FMAs per instruction).
+__device__ __forceinline__ uint64_t pack2f(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2f(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// 8 bf16 (one 16-byte vector) -> 4 packed pairs of floats
+__device__ __forceinline__ void unpack8x2(const uint4& v, uint64_t* f) {
+    f[0] = pack2f(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
+    f[1] = pack2f(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+    f[2] = pack2f(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xFFFF0000u));
+    f[3] = pack2f(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xFFFF0000u));
+}
+__device__ __forceinline__ uint4 pack8x2(const uint64_t* f) {
+    float a[8];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) unpack2f(f[k], a[2 * k], a[2 * k + 1]);
+    uint4 v;
+    v.x = pack2(a[0], a[1]); v.y = pack2(a[2], a[3]); v.z = pack2(a[4], a[5]); v.w = pack2(a[6], a[7]);
+    return v;
+}
 // streaming 16-byte accesses: activations are touched once per kernel
 __device__ __forceinline__ uint4 ld_stream(const void* p) {
     uint4 v;

@@ -254,20 +254,27 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
         const int quad = warp & 3;
         const int hw = (warp - 3) >> 2;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        float kap = 0.f, hp[N_], hr[N_][N_];
+        // the token's coefficients, each twice in a 64-bit register for the packed FMAs (fma.rn.f32x2)
+        uint64_t nkap2 = 0, hp2[N_], hr2[N_][N_];
         bool ok = true;
         for (int ti = 0; ti < nt; ++ti) {
             const int64_t row0 = (int64_t)tile_of(ti) * kFTok + quad * 32;
             const int64_t t = row0 + lane;
             const bool live = t < a.T;
-            kap = live ? __ldg(a.kappa + t) : 0.f;
+            {
+                const float kap = live ? -__ldg(a.kappa + t) : 0.f;
+                nkap2 = pack2f(kap, kap);
+            }
             if (MODE == 1) {
 #pragma unroll
-                for (int j = 0; j < N_; ++j) hp[j] = live ? __ldg(a.H_pre + t * N_ + j) : 0.f;
+                for (int j = 0; j < N_; ++j) { const float h = live ? __ldg(a.H_pre + t * N_ + j) : 0.f; hp2[j] = pack2f(h, h); }
 #pragma unroll
                 for (int i = 0; i < N_; ++i)
 #pragma unroll
-                    for (int j = 0; j < N_; ++j) hr[i][j] = live ? __ldg(a.H_res + t * N_ * N_ + i * N_ + j) : 0.f;
+                    for (int j = 0; j < N_; ++j) {
+                        const float h = live ? __ldg(a.H_res + t * N_ * N_ + i * N_ + j) : 0.f;
+                        hr2[i][j] = pack2f(h, h);
+                    }
             }
             unsigned char* slot = slots + ((ti * 4 + quad) % kFSlots) * kSlot;
             ok = mbar_wait(smem_u32(&ctl->d_full[quad][ti & 1]), (ti >> 1) & 1, abort, 7, ti);
@@ -288,37 +295,38 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                     uint32_t acc[N_][8];
 #pragma unroll
                     for (int j = 0; j < N_; ++j) ftc_ld8(tbase + j * 32 + pcl * 8, acc[j]);
-                    float gf[MODE == 1 ? N_ : 1][8], df[8];
+                    uint64_t gf[MODE == 1 ? N_ : 1][4], df[4];
                     if (MODE == 1) {
 #pragma unroll
-                        for (int i = 0; i < N_; ++i) unpack8(*reinterpret_cast<const uint4*>(slot + (N_ + i) * kFBox + po), gf[i]);
-                        unpack8(*reinterpret_cast<const uint4*>(slot + 2 * N_ * kFBox + po), df);
+                        for (int i = 0; i < N_; ++i) unpack8x2(*reinterpret_cast<const uint4*>(slot + (N_ + i) * kFBox + po), gf[i]);
+                        unpack8x2(*reinterpret_cast<const uint4*>(slot + 2 * N_ * kFBox + po), df);
                     }
                     ftc_ld_wait();
 #pragma unroll
                     for (int j = 0; j < N_; ++j) ftc_settle(acc[j]);
 #pragma unroll
                     for (int j = 0; j < N_; ++j) {
-                        float xf[8], o[8];
-                        unpack8(*reinterpret_cast<const uint4*>(slot + j * kFBox + po), xf);
+                        uint64_t xf[4], o[4];
+                        unpack8x2(*reinterpret_cast<const uint4*>(slot + j * kFBox + po), xf);
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) o[e] = fmaf(-xf[e], kap, __uint_as_float(acc[j][e]));
+                        for (int k = 0; k < 4; ++k)
+                            o[k] = fma2(xf[k], nkap2, pack2f(__uint_as_float(acc[j][2 * k]), __uint_as_float(acc[j][2 * k + 1])));
                         if (MODE == 1) {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) o[e] = fmaf(hp[j], df[e], o[e]);
+                            for (int k = 0; k < 4; ++k) o[k] = fma2(hp2[j], df[k], o[k]);
 #pragma unroll
                             for (int i = 0; i < N_; ++i)
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) o[e] = fmaf(hr[i][j], gf[i][e], o[e]);
+                                for (int k = 0; k < 4; ++k) o[k] = fma2(hr2[i][j], gf[i][k], o[k]);
                         }
                         if (MODE == 2) {
-                            float old[8];
-                            unpack8(*reinterpret_cast<const uint4*>(slot + (N_ + j) * kFBox + po), old);
+                            uint64_t old[4];
+                            unpack8x2(*reinterpret_cast<const uint4*>(slot + (N_ + j) * kFBox + po), old);
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) o[e] += old[e];
+                            for (int k = 0; k < 4; ++k) o[k] = fma2(old[k], pack2f(1.f, 1.f), o[k]);
                         }
                         // dx takes the place of g (of the old dx; of x itself in MODE 0) in the slot
-                        *reinterpret_cast<uint4*>(slot + (kOut + j) * kFBox + po) = pack8(o);
+                        *reinterpret_cast<uint4*>(slot + (kOut + j) * kFBox + po) = pack8x2(o);
                     }
                 }
                 tc_fence_before();
