@@ -18,7 +18,7 @@ CASES = [  # (n, C, T): ragged token tails (T not a multiple of 32/64/128) and r
     (4, 256, 333), (4, 264, 130), (2, 8, 77), (3, 72, 200), (5, 136, 161), (4, 1024, 257), (3, 1536, 65),
     (5, 320, 700),
     # fused tcgen05 tail (C a multiple of 64): n = 2, and several 128-token tiles per CTA with a ragged last tile
-    (2, 128, 300), (4, 2048, 1100),
+    (2, 128, 300), (4, 2048, 1100), (3, 1536, 2000),
 ]
 
 
