@@ -17,6 +17,9 @@ What is computed, with the passage that defines it:
 * Eq. (5)   H_res = sum_k a_k P_k over all n! permutations     -> hres_from_weights
             (Section 3.2 also states it as a product of a with a constant
             0/1 matrix of shape n! x n^2                        -> hres_from_weights_matmul)
+* Section 5 ("larger n"): the same convex combination over a caller-given SUBSET of K
+            permutation matrices (still exactly doubly stochastic)  -> check_perm_rows, hres_from_table,
+            and the `table` argument of coeffs_fwd / coeffs_bwd / layer_fwd / layer_bwd
 * Eq. (2)   mHC: H_res = SK(exp(mat(.))), 20 iterations        -> sk_iterate, sk_coeffs_fwd
 * Section 3.1 footnote / Eq. (3): l1-error and relative range  -> l1_error, relative_range
 * the backward of all of the above is the exact gradient (the paper relies on
@@ -38,7 +41,10 @@ Readings of the paper taken here (each is a choice where the text is silent):
 Pins (tests/test_oracle_*.py): permutation table vs brute force; exact double
 stochasticity; one-hot and uniform weights; the two routes to H_res; products
 over depth; the printed 3x3 SK example; closed forms of RMSNorm / softmax /
-sigmoid; n = 2 closed form; central finite differences for every gradient.
+sigmoid; n = 2 closed form; central finite differences for every gradient;
+the stand-in sublayer and the layer stack by hand cases, hand-chained layers and
+finite differences; the subset variant by exact row / column sums for any subset,
+by the full table reproducing Eq. (5), and by finite differences.
 Parity unpinned: the value of eps (a free argument) and the normalisation of the
 test tolerances, which are choices and not derivable from the paper.
 """
@@ -78,6 +84,38 @@ def hres_from_weights(a: np.ndarray, n: int) -> np.ndarray:
     for k in range(sig.shape[0]):
         for i in range(n):
             H[:, i, sig[k, i]] += a[:, k]
+    return H
+
+
+def check_perm_rows(table, n: int) -> np.ndarray:
+    """Validates a caller-given table of K permutations of (0..n-1) (Section 5: a subset of the n!
+    permutation matrices).  Every row must be a bijection and no row may appear twice; returns the
+    table as int64 [K, n], raises ValueError otherwise."""
+    tab = np.asarray(table)
+    if tab.ndim != 2 or tab.shape[1] != n or tab.shape[0] < 1:
+        raise ValueError("permutation table must have shape [K >= 1, n]")
+    tab = tab.astype(np.int64)
+    seen = set()
+    for k in range(tab.shape[0]):
+        row = tuple(int(v) for v in tab[k])
+        if sorted(row) != list(range(n)):
+            raise ValueError(f"row {k} of the permutation table is not a bijection of 0..{n - 1}: {row}")
+        if row in seen:
+            raise ValueError(f"row {k} of the permutation table repeats an earlier row: {row}")
+        seen.add(row)
+    return tab
+
+
+def hres_from_table(a: np.ndarray, table) -> np.ndarray:
+    """Eq. (5) restricted to the K permutations of `table` (Section 5): H_res[t] = sum_k a[t,k] P_k
+    with P_k[i, table[k,i]] = 1.  a [T, K] -> [T, n, n]."""
+    tab = np.asarray(table).astype(np.int64)
+    K, n = tab.shape
+    a = np.asarray(a, dtype=F64)
+    H = np.zeros((a.shape[0], n, n), dtype=F64)
+    for k in range(K):
+        for i in range(n):
+            H[:, i, tab[k, i]] += a[:, k]
     return H
 
 
@@ -144,18 +182,23 @@ def _softmax(z):
     return e / np.sum(e, axis=-1, keepdims=True)
 
 
-def coeffs_fwd(x, W, b, alpha, gain, eps: float = 1e-6) -> dict:
+def coeffs_fwd(x, W, b, alpha, gain, eps: float = 1e-6, table=None) -> dict:
     """Eq. (4) and (5): the dynamic mappings of mHC-lite for every token.
 
     x [T,n,C]; W [nC, n!+2n]; b [n!+2n]; alpha (res, pre, post); gain [nC].
-    Returns H_res [T,n,n], H_pre [T,n], H_post [T,n], a [T,n!], z, p, rstd.
+    With `table` [K, n] (Section 5: a subset of the permutations) the residual group has K
+    columns instead of n! and the convex combination runs over the table's rows.
+    Returns H_res [T,n,n], H_pre [T,n], H_post [T,n], a [T,n! or K], z, p, rstd.
     """
     n = np.asarray(x).shape[1]
-    n_res = math.factorial(n)
+    if table is not None:
+        table = check_perm_rows(table, n)
+    n_res = math.factorial(n) if table is None else table.shape[0]
     xh, xn, rstd, p, z = _logits(x, W, b, alpha, gain, eps, n_res)
     gr, gp, go = _groups(n, n_res)
     a = _softmax(z[:, gr])
-    return dict(H_res=hres_from_weights(a, n), H_pre=_sigmoid(z[:, gp]),
+    H_res = hres_from_weights(a, n) if table is None else hres_from_table(a, table)
+    return dict(H_res=H_res, H_pre=_sigmoid(z[:, gp]),
                 H_post=2.0 * _sigmoid(z[:, go]), a=a, z=z, p=p, rstd=rstd)
 
 
@@ -209,16 +252,25 @@ def _proj_bwd(xh, xn, rstd, p, W, alpha, gain, dz, n, n_res):
     return dict(dx=dxh.reshape(T, n, nC // n), dW=dW, db=db, dalpha=dalpha, dgain=dgain, dz=dz)
 
 
-def coeffs_bwd(x, W, b, alpha, gain, eps, dH_res, dH_pre, dH_post) -> dict:
+def coeffs_bwd(x, W, b, alpha, gain, eps, dH_res, dH_pre, dH_post, table=None) -> dict:
     """Gradient of coeffs_fwd: from (dH_res, dH_pre, dH_post) to dx, dW, db, dalpha, dgain."""
     x = np.asarray(x, dtype=F64)
     n = x.shape[1]
-    n_res = math.factorial(n)
+    if table is not None:
+        table = check_perm_rows(table, n)
+    n_res = math.factorial(n) if table is None else table.shape[0]
     xh, xn, rstd, p, z = _logits(x, W, b, alpha, gain, eps, n_res)
     gr, gp, go = _groups(n, n_res)
     a = _softmax(z[:, gr]); H_pre = _sigmoid(z[:, gp]); H_post = 2.0 * _sigmoid(z[:, go])
     # Eq. (5): dL/da_k = sum_i dH_res[i, sigma_k(i)]
-    da = np.einsum("tij,kij->tk", np.asarray(dH_res, dtype=F64), perm_matrices(n))
+    dH_res = np.asarray(dH_res, dtype=F64)
+    if table is None:
+        da = np.einsum("tij,kij->tk", dH_res, perm_matrices(n))
+    else:
+        da = np.zeros((x.shape[0], n_res), dtype=F64)
+        for k in range(n_res):
+            for i in range(n):
+                da[:, k] += dH_res[:, i, table[k, i]]
     dz = np.empty_like(z)
     dz[:, gr] = a * (da - np.sum(a * da, axis=1, keepdims=True))
     dz[:, gp] = np.asarray(dH_pre, dtype=F64) * H_pre * (1.0 - H_pre)
@@ -226,21 +278,21 @@ def coeffs_bwd(x, W, b, alpha, gain, eps, dH_res, dH_pre, dH_post) -> dict:
     return _proj_bwd(xh, xn, rstd, p, W, alpha, gain, dz, n, n_res)
 
 
-def layer_fwd(x, y, W, b, alpha, gain, eps: float = 1e-6, kind: str = "lite", iters: int = 20) -> dict:
+def layer_fwd(x, y, W, b, alpha, gain, eps: float = 1e-6, kind: str = "lite", iters: int = 20, table=None) -> dict:
     """One Hyper-Connections layer with the sublayer output y given (Eq. (1))."""
-    co = coeffs_fwd(x, W, b, alpha, gain, eps) if kind == "lite" else sk_coeffs_fwd(x, W, b, alpha, gain, eps, iters)
+    co = coeffs_fwd(x, W, b, alpha, gain, eps, table) if kind == "lite" else sk_coeffs_fwd(x, W, b, alpha, gain, eps, iters)
     co["u"] = premix_fwd(x, co["H_pre"])
     co["x_next"] = postres_fwd(x, y, co["H_res"], co["H_post"])
     return co
 
 
-def layer_bwd(x, y, W, b, alpha, gain, eps, g, du, kind: str = "lite", iters: int = 20) -> dict:
+def layer_bwd(x, y, W, b, alpha, gain, eps, g, du, kind: str = "lite", iters: int = 20, table=None) -> dict:
     """Backward of layer_fwd for L(x_next, u) with g = dL/dx_next, du = dL/du; y is an input."""
-    co = coeffs_fwd(x, W, b, alpha, gain, eps) if kind == "lite" else sk_coeffs_fwd(x, W, b, alpha, gain, eps, iters)
+    co = coeffs_fwd(x, W, b, alpha, gain, eps, table) if kind == "lite" else sk_coeffs_fwd(x, W, b, alpha, gain, eps, iters)
     b1 = postres_bwd(x, y, co["H_res"], co["H_post"], g)
     b2 = premix_bwd(x, co["H_pre"], du)
     if kind == "lite":
-        b3 = coeffs_bwd(x, W, b, alpha, gain, eps, b1["dH_res"], b2["dH_pre"], b1["dH_post"])
+        b3 = coeffs_bwd(x, W, b, alpha, gain, eps, b1["dH_res"], b2["dH_pre"], b1["dH_post"], table)
     else:
         b3 = sk_coeffs_bwd(x, W, b, alpha, gain, eps, b1["dH_res"], b2["dH_pre"], b1["dH_post"], iters)
     return dict(dx=b1["dx"] + b2["dx"] + b3["dx"], dy=b1["dy"], dW=b3["dW"], db=b3["db"],
@@ -321,11 +373,14 @@ def l1_error(X) -> np.ndarray:
 
 
 def relative_range(X) -> np.ndarray:
-    """Eq. (3): nu = (smallest positive entry) / (largest entry), per matrix."""
+    """Eq. (3): nu = (smallest positive entry) / (largest entry), per matrix; zero entries are
+    skipped, and a matrix without any positive entry has nu = 0."""
     X = np.asarray(X, dtype=F64)
     flat = X.reshape(X.shape[:-2] + (-1,))
     pos = np.where(flat > 0, flat, np.inf)
-    return pos.min(axis=-1) / flat.max(axis=-1)
+    lo, hi = pos.min(axis=-1), flat.max(axis=-1)
+    with np.errstate(invalid="ignore", divide="ignore"):
+        return np.where(hi > 0, lo / np.where(hi > 0, hi, 1.0), 0.0)
 
 
 def column_sums(X) -> np.ndarray:

@@ -320,3 +320,222 @@ def test_round_bf16():
     assert abs(out[7] - 3.14159) <= 2 ** -7 * 2
     for o in out:
         assert (np.float32(o).view(np.uint32) & 0xFFFF) == 0
+
+
+# ------------------------------------------------------------------ Eq. (3): zero entries and the degenerate matrix
+def test_relative_range_skips_zeros():
+    # smallest POSITIVE entry over the largest: the zero of [[0,2],[4,8]] is skipped -> 2/8
+    assert O.relative_range(np.array([[[0.0, 2.0], [4.0, 8.0]]]))[0] == 0.25
+    # a negative entry is not "positive" either
+    assert O.relative_range(np.array([[[-1.0, 2.0], [4.0, 8.0]]]))[0] == 0.25
+    # no positive entry at all: nu = 0 (1/nu unbounded)
+    assert O.relative_range(np.zeros((1, 3, 3)))[0] == 0.0
+    # batch of two, mixed
+    out = O.relative_range(np.array([[[1.0, 0.0], [0.0, 4.0]], [[0.0, 0.0], [0.0, 0.0]]]))
+    assert out.tolist() == [0.25, 0.0]
+
+
+# ------------------------------------------------------------------ stand-in sublayer and the layer stack (24-layer workload)
+def test_standin_sublayer_hand_case_and_gradient():
+    # y = u / sqrt(mean(u^2) + eps): u = (3, 4), eps = 0 -> mean square 12.5
+    y = O.standin_sublayer_fwd(np.array([[3.0, 4.0]]), 0.0)
+    assert np.abs(y[0] - np.array([3.0, 4.0]) / math.sqrt(12.5)).max() < 1e-16
+    # eps enters under the root: u = (1,-1,1,-1), eps = 3 -> 1/sqrt(4)
+    y = O.standin_sublayer_fwd(np.array([[1.0, -1.0, 1.0, -1.0]]), 3.0)
+    assert np.abs(y[0] - np.array([0.5, -0.5, 0.5, -0.5])).max() < 1e-16
+    # gradient by central finite differences of the forward
+    r = np.random.default_rng(5)
+    u = r.standard_normal((3, 6)); dy = r.standard_normal((3, 6)); eps = 1e-3
+    an = O.standin_sublayer_bwd(u, dy, eps)
+    h = 1e-6
+    for ix in np.ndindex(u.shape):
+        up = u.copy(); up[ix] += h
+        um = u.copy(); um[ix] -= h
+        fd = ((O.standin_sublayer_fwd(up, eps) - O.standin_sublayer_fwd(um, eps)) * dy).sum() / (2 * h)
+        assert abs(fd - an[ix]) <= 2e-7 * np.abs(an).max(), (ix, fd, an[ix])
+    # eps = 0: y does not depend on the scale of u, so <u, du> = 0 for every token
+    du0 = O.standin_sublayer_bwd(u, dy, 0.0)
+    assert np.abs((u * du0).sum(axis=1)).max() < 1e-13
+
+
+def _stack_params(Ld, n, C, seed):
+    r = np.random.default_rng(seed)
+    N = math.factorial(n) + 2 * n
+    return [(r.standard_normal((n * C, N)) * 0.3, r.standard_normal(N) * 0.5, np.array([0.7, 1.1, 0.9]),
+             1.0 + 0.2 * r.standard_normal(n * C)) for _ in range(Ld)]
+
+
+def _stack_loss(x0, params, R, eps):
+    x = x0
+    for (W, b, al, ga) in params:
+        co = O.coeffs_fwd(x, W, b, al, ga, eps)
+        y = O.standin_sublayer_fwd(O.premix_fwd(x, co["H_pre"]), eps)
+        x = O.postres_fwd(x, y, co["H_res"], co["H_post"])
+    return float((x * R).sum())
+
+
+def test_stack_equals_hand_chained_layers_and_finite_differences():
+    T, n, C, Ld, eps = 2, 3, 4, 3, 1e-3
+    r = np.random.default_rng(21)
+    params = _stack_params(Ld, n, C, 22)
+    x0 = r.standard_normal((T, n, C)); R = r.standard_normal((T, n, C))
+    st = O.stack_fwd_bwd(x0, params, R, eps, bf16_storage=False)
+    # forward: layer by layer with the single-layer functions
+    xs, us, ys = [x0], [], []
+    for (W, b, al, ga) in params:
+        co = O.coeffs_fwd(xs[-1], W, b, al, ga, eps)
+        us.append(O.premix_fwd(xs[-1], co["H_pre"]))
+        ys.append(O.standin_sublayer_fwd(us[-1], eps))
+        fw = O.layer_fwd(xs[-1], ys[-1], W, b, al, ga, eps)
+        assert np.abs(fw["u"] - us[-1]).max() == 0
+        xs.append(fw["x_next"])
+    for l in range(Ld + 1):
+        assert np.abs(st["xs"][l] - xs[l]).max() < 1e-14
+    # backward: layer l gets the gradient that layer l + 1 returned, and du = standin_bwd(u_l, dy_l)
+    g = R
+    for l in reversed(range(Ld)):
+        W, b, al, ga = params[l]
+        dy = O.postres_bwd(xs[l], ys[l], st["H_res"][l], O.coeffs_fwd(xs[l], W, b, al, ga, eps)["H_post"], g)["dy"]
+        du = O.standin_sublayer_bwd(us[l], dy, eps)
+        bw = O.layer_bwd(xs[l], ys[l], W, b, al, ga, eps, g, du)
+        for k in ("dW", "db", "dalpha", "dgain"):
+            assert np.abs(st["grads"][l][k] - bw[k]).max() < 1e-12, (l, k)
+        g = bw["dx"]
+    assert np.abs(st["dx0"] - g).max() < 1e-12
+    # finite differences of the stacked forward: dx0, and one entry of dW, db, dalpha, dgain per layer
+    h = 1e-6
+    scale = np.abs(st["dx0"]).max()
+    for ix in [(0, 0, 0), (1, 2, 3), (0, 1, 2), (1, 0, 1)]:
+        xp = x0.copy(); xp[ix] += h
+        xm = x0.copy(); xm[ix] -= h
+        fd = (_stack_loss(xp, params, R, eps) - _stack_loss(xm, params, R, eps)) / (2 * h)
+        assert abs(fd - st["dx0"][ix]) <= 2e-7 * scale + 1e-9, (ix, fd, st["dx0"][ix])
+    names = ("dW", "db", "dalpha", "dgain")
+    for l in range(Ld):
+        for pi, ix in enumerate([(5, 2), (7,), (1,), (9,)]):
+            def loss_with(delta):
+                ps = [list(p) for p in params]
+                arr = np.array(ps[l][pi], dtype=float, copy=True); arr[ix] += delta
+                ps[l][pi] = arr
+                return _stack_loss(x0, [tuple(p) for p in ps], R, eps)
+            fd = (loss_with(h) - loss_with(-h)) / (2 * h)
+            an = st["grads"][l][names[pi]][ix]
+            assert abs(fd - an) <= 2e-7 * np.abs(st["grads"][l][names[pi]]).max() + 1e-9, (l, names[pi], fd, an)
+
+
+def test_stack_bf16_storage_lies_on_the_bf16_grid():
+    T, n, C, Ld, eps = 3, 4, 8, 2, 1e-6
+    r = np.random.default_rng(23)
+    params = _stack_params(Ld, n, C, 24)
+    x0 = O.round_bf16(r.standard_normal((T, n, C))); R = O.round_bf16(r.standard_normal((T, n, C)))
+    st = O.stack_fwd_bwd(x0, params, R, eps, bf16_storage=True)
+    on_grid = lambda a: ((np.asarray(a, dtype=np.float32).view(np.uint32) & 0xFFFF) == 0).all() and \
+        (np.asarray(a, dtype=np.float32).astype(np.float64) == a).all()
+    for l in range(Ld + 1):
+        assert on_grid(st["xs"][l]), l
+    assert on_grid(st["dx0"])
+    # and it stays within bf16 rounding of the unrounded stack
+    ex = O.stack_fwd_bwd(x0, params, R, eps, bf16_storage=False)
+    assert np.abs(st["xs"][Ld] - ex["xs"][Ld]).max() <= 2.0 ** -6 * np.abs(ex["xs"][Ld]).max()
+    assert np.abs(st["xs"][Ld] - ex["xs"][Ld]).max() > 0
+
+
+# ------------------------------------------------------------------ Section 5: a subset of the permutations
+@pytest.mark.parametrize("n,K", [(3, 2), (4, 7), (5, 8), (5, 64), (6, 24)])
+def test_any_subset_of_permutations_is_exactly_doubly_stochastic(n, K):
+    r = np.random.default_rng(n * 100 + K)
+    full = np.array(list(itertools.permutations(range(n))))
+    tab = full[r.choice(len(full), K, replace=False)]
+    T, C = 16, 4
+    N = K + 2 * n
+    x = r.standard_normal((T, n, C)); W = r.standard_normal((n * C, N)); b = r.standard_normal(N)
+    co = O.coeffs_fwd(x, W, b, [2.0, 1.0, 1.0], np.ones(n * C), 1e-6, table=tab)
+    H = co["H_res"]
+    assert co["a"].shape == (T, K) and H.shape == (T, n, n)
+    assert (H >= 0).all()
+    assert np.abs(H.sum(axis=1) - 1).max() < 1e-14 and np.abs(H.sum(axis=2) - 1).max() < 1e-14
+    # entries outside the support of the sampled permutations are exactly zero
+    support = np.zeros((n, n), dtype=bool)
+    for row in tab:
+        support[np.arange(n), row] = True
+    assert (H[:, ~support] == 0).all()
+    # brute-force Eq. (5) over the subset for one token
+    ref = np.zeros((n, n))
+    for k, row in enumerate(tab):
+        P = np.zeros((n, n)); P[np.arange(n), row] = 1
+        ref += co["a"][0, k] * P
+    assert np.abs(H[0] - ref).max() < 1e-15
+
+
+@pytest.mark.parametrize("n", [3, 4])
+def test_full_table_as_subset_reproduces_eq5(n):
+    L = _rand_layer(5, n, 8, seed=60 + n)
+    tab = O.perm_table(n)
+    a = O.layer_fwd(L["x"], L["y"], L["W"], L["b"], L["alpha"], L["gain"], 1e-6)
+    b = O.layer_fwd(L["x"], L["y"], L["W"], L["b"], L["alpha"], L["gain"], 1e-6, table=tab)
+    for k in ("H_res", "H_pre", "H_post", "a", "u", "x_next"):
+        assert np.abs(a[k] - b[k]).max() < 1e-15, k
+    ga = O.layer_bwd(L["x"], L["y"], L["W"], L["b"], L["alpha"], L["gain"], 1e-6, L["g"], L["du"])
+    gb = O.layer_bwd(L["x"], L["y"], L["W"], L["b"], L["alpha"], L["gain"], 1e-6, L["g"], L["du"], table=tab)
+    for k in ("dx", "dW", "db", "dalpha", "dgain"):
+        assert np.abs(ga[k] - gb[k]).max() < 1e-13, k
+    # a permuted table permutes the residual columns: row order is the caller's
+    perm = np.random.default_rng(3).permutation(len(tab))
+    N = len(tab) + 2 * n
+    cols = np.concatenate([perm, np.arange(len(tab), N)])
+    c = O.coeffs_fwd(L["x"], L["W"][:, cols], L["b"][cols], L["alpha"], L["gain"], 1e-6, table=tab[perm])
+    assert np.abs(c["H_res"] - a["H_res"]).max() < 1e-14
+
+
+def test_subset_one_hot_and_rejections():
+    n, C, T = 5, 4, 2
+    tab = np.array([[0, 1, 2, 3, 4], [4, 3, 2, 1, 0], [1, 0, 3, 2, 4]])
+    N = 3 + 2 * n
+    x = np.random.default_rng(1).standard_normal((T, n, C))
+    for k in range(3):
+        b = np.zeros(N); b[:3] = -800.0; b[k] = 0.0
+        co = O.coeffs_fwd(x, np.zeros((n * C, N)), b, [1, 1, 1], np.ones(n * C), 1e-6, table=tab)
+        expect = np.zeros((n, n)); expect[np.arange(n), tab[k]] = 1.0
+        assert (co["H_res"] == expect).all()
+    with pytest.raises(ValueError):
+        O.check_perm_rows([[0, 1, 1]], 3)                       # not a bijection
+    with pytest.raises(ValueError):
+        O.check_perm_rows([[0, 1, 2], [0, 1, 2]], 3)            # repeated row
+    with pytest.raises(ValueError):
+        O.check_perm_rows([[0, 1, 3]], 3)                       # out of range
+    with pytest.raises(ValueError):
+        O.check_perm_rows([[0, 1]], 3)                          # wrong width
+    assert O.check_perm_rows([[2, 0, 1]], 3).tolist() == [[2, 0, 1]]
+
+
+@pytest.mark.parametrize("n,K", [(4, 5), (5, 8), (6, 6)])
+def test_subset_backward_finite_differences(n, K):
+    T, C = 2, 4
+    r = np.random.default_rng(70 + n)
+    full = np.array(list(itertools.permutations(range(n))))
+    tab = full[r.choice(len(full), K, replace=False)]
+    N = K + 2 * n
+    L = dict(x=r.standard_normal((T, n, C)), y=r.standard_normal((T, C)), W=r.standard_normal((n * C, N)) * 0.3,
+             b=r.standard_normal(N) * 0.5, alpha=np.array([0.7, 1.1, 0.9]), gain=1.0 + 0.2 * r.standard_normal(n * C))
+    R1, R2 = r.standard_normal((T, n, C)), r.standard_normal((T, C))
+
+    def loss(**over):
+        p = {**L, **over}
+        o = O.layer_fwd(p["x"], p["y"], p["W"], p["b"], p["alpha"], p["gain"], 1e-6, table=tab)
+        return float((o["x_next"] * R1).sum() + (o["u"] * R2).sum())
+
+    gr = O.layer_bwd(L["x"], L["y"], L["W"], L["b"], L["alpha"], L["gain"], 1e-6, R1, R2, table=tab)
+    assert np.abs(gr["dz"][:, :K].sum(axis=1)).max() < 1e-12
+    h = 1e-5
+    for key, gname in dict(x="dx", y="dy", W="dW", b="db", alpha="dalpha", gain="dgain").items():
+        base = np.asarray(L[key], dtype=float)
+        an = np.asarray(gr[gname]).reshape(base.shape)
+        idx = list(np.ndindex(base.shape))
+        if len(idx) > 20:
+            idx = [idx[i] for i in r.choice(len(idx), 20, replace=False)]
+        scale = np.abs(an).max() + 1e-30
+        for ix in idx:
+            pp = base.copy(); pp[ix] += h
+            pm = base.copy(); pm[ix] -= h
+            fd = (loss(**{key: pp}) - loss(**{key: pm})) / (2 * h)
+            assert abs(fd - an[ix]) <= 2e-7 * scale + 1e-9, (key, ix, fd, an[ix])
