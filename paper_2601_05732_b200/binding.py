@@ -271,7 +271,7 @@ class MhcLite:
             self._ptr(dH_post, f), self._ptr(dx, h), self._ptr(dW, f), self._ptr(db, f), self._ptr(dalpha, f),
             self._ptr(dgain, f), int(accumulate_params), self._stream()), "mhc_sk20_tail_bwd_fused")
 
-    KERNELS = ("proj_fwd", "act_premix", "postres_fwd", "postres_bwd", "tail_pre", "tail_mma")
+    KERNELS = ("proj_fwd", "act_premix", "postres_fwd", "postres_bwd", "tail_pre", "tail_dx")
 
     def set_kernel_timing(self, on: bool):
         self._check(self.lib.mhclite_set_kernel_timing(self._h, int(on)), "mhclite_set_kernel_timing")

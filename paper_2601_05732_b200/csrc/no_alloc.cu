@@ -13,7 +13,7 @@
 
 namespace mhcl {
 
-constexpr size_t kStaticScratchBytes = 4u << 20;        // 4 MiB: e.g. n = 4, C = 1024, T <= 8192 tokens
+constexpr size_t kStaticScratchBytes = 4u << 20;        // 4 MiB: e.g. n = 4, C = 1024 up to about 27 000 tokens
 
 // The scratch itself.  In host code this name is only a handle for the runtime's symbol look-up,
 // never a device address: kernels get the pointer obtained by cudaGetSymbolAddress below.

@@ -505,7 +505,7 @@ bool launch_tail_ftc(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, 
         pack_wf_k<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(n, C, N, p.Kp, W, gain, (__nv_bfloat16*)Wf, nullptr,
                                                                   nullptr);
     }
-    KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_MMA, s);
+    KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_DX, s);
     dim3 grid(p.f_slices, p.f_splits);
     switch (n) {
         case 2: launch_ftc_t<2>(grid, smem, tmx, tmg, tmdu, tmdx, a, mode, s); break;

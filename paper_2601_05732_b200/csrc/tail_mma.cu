@@ -404,7 +404,7 @@ void launch_tail_mma(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, 
         default: launch_tail_t<N_, 3>(p, a, fused, acc_dx != 0, s); break;        \
     }
     {
-        KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_MMA, s);
+        KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_DX, s);
         MHCL_DISPATCH_N(c->n, MHCL_TAIL_KS(N_));
     }
 #undef MHCL_TAIL_KS

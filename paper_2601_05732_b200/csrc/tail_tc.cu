@@ -530,7 +530,7 @@ bool launch_tail_dx_tc(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p
     c->launches += 2;
     const int64_t total = (int64_t)n * a.ncb * p.Kp * kDCh;
     pack_wb_k<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(n, C, N, p.Kp, a.ncb, W, gain, (__nv_bfloat16*)Wb);
-    KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_MMA, s);
+    KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_DX, s);
     MHCL_DISPATCH_N(n, (launch_dx_t<N_>(grid, smem, tmx, tmg, tmdu, a, fused, acc_dx != 0, s)));
     return true;
 }

@@ -91,3 +91,31 @@ def tail_bwd(ctx: MhcLite, P: LayerParams, B: LayerBuffers, x, g, du, eps=1e-6, 
         ctx.premix_bwd(x, B.H_pre, du, B.dH_pre, B.dx, True)
         ctx.coeffs_bwd(x, P.W, P.alpha, P.gain, eps, B.a_saved, B.p_saved, B.rstd, B.H_pre, B.H_post,
                        B.dH_res, B.dH_pre, B.dH_post, B.dx, True, B.dW, B.db, B.dalpha, B.dgain, accumulate_params)
+
+
+def stack_fwd(ctx: MhcLite, Ps, Bs, x0, sublayer, eps=1e-6):
+    """Forward through len(Ps) layers (the paper's models are 6, 12 or 24 of them back to back): layer l reads the
+    x_next of layer l - 1.  `sublayer(l, u)` is the caller's f and returns y [T,C] bf16.  Each layer's input, y
+    and outputs stay in its LayerBuffers for the backward.  Returns the last layer's x_next."""
+    x = x0
+    for l, (P, B) in enumerate(zip(Ps, Bs)):
+        B.x_in = x
+        pre_fwd(ctx, P, B, x, eps, True)
+        B.y = sublayer(l, B.u)
+        post_fwd(ctx, B, x, B.y)
+        x = B.x_next
+    return x
+
+
+def stack_bwd(ctx: MhcLite, Ps, Bs, g_top, sublayer_bwd, eps=1e-6):
+    """Backward through the stack: `sublayer_bwd(l, u, dy)` is the caller's backward of f and returns du [T,C] bf16.
+    Returns dL/dx_0; each layer's parameter gradients are in its LayerBuffers."""
+    g = g_top
+    for l in reversed(range(len(Ps))):
+        P, B = Ps[l], Bs[l]
+        B.g_in = g
+        post_bwd(ctx, B, B.x_in, B.y, g, True)
+        B.du = sublayer_bwd(l, B.u, B.dy)
+        tail_bwd(ctx, P, B, B.x_in, g, B.du, eps, True)
+        g = B.dx
+    return g

@@ -27,3 +27,20 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+def pytest_sessionfinish(session, exitstatus):
+    """Writes the raw error figures that the parity helpers collected (one JSON object per comparison) to
+    gpurun_out/parity_errors.jsonl at the repository root; tests/parity_report.py turns them into a table."""
+    try:
+        import json
+        import parity_utils
+    except Exception:
+        return
+    if not parity_utils.RECORDS:
+        return
+    out = os.path.join(ROOT, "gpurun_out")
+    os.makedirs(out, exist_ok=True)
+    with open(os.path.join(out, "parity_errors.jsonl"), "w") as f:
+        for r in parity_utils.RECORDS:
+            f.write(json.dumps(r) + "\n")

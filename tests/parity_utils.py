@@ -27,14 +27,38 @@ def rms(a):
     return float(np.sqrt(np.mean(a * a))) if a.size else 0.0
 
 
+RECORDS = []     # raw error figures of every comparison made in this session (written out by conftest.py)
+
+
+def _record(name, kind, got, ref, tol, tol_plain):
+    """Raw figures of one comparison: max relative error over the elements with |ref| >= rms/16, max
+    absolute error over rms, and the worst error as a fraction of the tolerance, with and without the
+    per-element allowance (`extra`) -- so that neither the floor term nor an allowance can hide anything."""
+    import os
+    err = np.abs(got - ref)
+    r = rms(ref)
+    big = np.abs(ref) >= r / 16 if r > 0 else np.zeros(ref.shape, dtype=bool)
+    rec = dict(test=os.environ.get("PYTEST_CURRENT_TEST", "").split(" ")[0], tensor=name, kind=kind, size=int(ref.size),
+               rms=r, max_abs_err=float(err.max()) if err.size else 0.0,
+               max_abs_err_over_rms=float(err.max() / r) if (err.size and r > 0) else 0.0,
+               max_rel_err_big=float((err[big] / np.abs(ref[big])).max()) if big.any() else 0.0,
+               worst_over_tol=float((err / tol).max()) if err.size else 0.0,
+               worst_over_tol_no_extra=float((err / tol_plain).max()) if err.size else 0.0)
+    RECORDS.append(rec)
+    return rec
+
+
 def check_bf16(name, got, ref, rel=2e-2, floor=1e-3, extra=0.0):
     """`extra` (per element) allows for a tensor that was stored in bf16 on the way: one rounding of
     an intermediate v moves the result by up to 2^-8 |v|, whatever the size of the final value."""
     got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (name, got.shape, ref.shape)
-    tol = rel * np.abs(ref) + floor * rms(ref) + extra
+    plain = rel * np.abs(ref) + floor * rms(ref) + 1e-300
+    tol = plain + extra
+    rec = _record(name, "bf16", got, ref, tol, plain)
     bad = np.abs(got - ref) > tol
     assert not bad.any(), f"{name}: {bad.sum()} of {bad.size} elements off; worst {np.abs(got - ref).max():.3e} (rms {rms(ref):.3e})"
+    return rec
 
 
 def check_f32(name, got, ref, rel=1e-5):
@@ -42,7 +66,9 @@ def check_f32(name, got, ref, rel=1e-5):
     assert got.shape == ref.shape, (name, got.shape, ref.shape)
     tol = rel * np.maximum(np.abs(ref), rms(ref)) + 1e-30
     err = np.abs(got - ref)
+    rec = _record(name, "f32@%g" % rel, got, ref, tol, tol)
     assert (err <= tol).all(), f"{name}: worst err/tol {np.max(err / tol):.2f}, max abs err {err.max():.3e}, rms {rms(ref):.3e}"
+    return rec
 
 
 def host(t):

@@ -42,9 +42,10 @@ def _oracle_param_grads(inp, kind, chunk=4096):
     return acc
 
 
-def _run_and_check(wl, kind="lite", param_grads=True, T=None):
+def _run_and_check(wl, kind="lite", param_grads=True, T=None, inp=None):
     T = T or wl.T
-    inp = synth.make_layer_inputs(wl.n, wl.C, T, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std, kind=kind)
+    if inp is None:
+        inp = synth.make_layer_inputs(wl.n, wl.C, T, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std, kind=kind)
     G = GpuLayer(inp, kind=kind)
     G.forward(True)
     if wl.backward:
@@ -56,7 +57,7 @@ def _run_and_check(wl, kind="lite", param_grads=True, T=None):
     if kind == "lite":
         assert float((Hr.sum(1) - 1).abs().max()) < 1e-6 and float((Hr.sum(2) - 1).abs().max()) < 1e-6
     for t in (B.u, B.x_next, B.H_pre, B.H_post, B.p_saved, B.rstd) + ((B.dx, B.dy, B.dW, B.dgain) if wl.backward else ()):
-        assert bool(torch.isfinite(t.float()).all())
+        assert bool(torch.isfinite(t).all())
     # sampled tokens, element by element
     idx = np.sort(np.random.default_rng(wl.seed).choice(T, NS, replace=False))
     sub = _subset(inp, idx)
@@ -102,9 +103,8 @@ def test_cfg4a_n3():
 
 
 def test_cfg4b_n5():
-    _run_and_check(synth.WORKLOADS["cfg4b"], param_grads=False)
-    # the parameter gradients of n = 5 on a quarter of the tokens (the oracle's n*C x 130 products are slow)
-    _run_and_check(synth.WORKLOADS["cfg4b"], T=8192)
+    # full size, parameter gradients included (the oracle runs over the 32768 tokens in chunks)
+    _run_and_check(synth.WORKLOADS["cfg4b"])
 
 
 @pytest.mark.parametrize("T", [4096, 32768])
@@ -118,6 +118,31 @@ def test_cfg5_lite_and_sk(T):
     torch.cuda.synchronize()
     assert float(l1.max()) < 4e-6
     assert float(l2.max()) < 1e-4          # near-uniform logits: SK converges; the stress case is in test_gpu_parity
+
+
+@pytest.mark.parametrize("T", [65536, 131072])
+def test_cfg5_upper_half_of_the_sweep(T):
+    # the largest points of the token sweep (x alone is 4.3 GB at T = 131072, 2^31 elements): all-token
+    # properties and sampled tokens against the oracle, both paths on the same tokens
+    wl = synth.WORKLOADS["cfg5"]
+    inp = synth.make_layer_inputs(wl.n, wl.C, T, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std)
+    GL = _run_and_check(wl, "lite", param_grads=False, T=T, inp=inp)
+    l1 = torch.empty(T, device=DEV)
+    GL.ctx.ds_gap(GL.B.H_res, l1, None); torch.cuda.synchronize()
+    assert float(l1.max()) < 4e-6
+    GL.ctx.device_status()
+    # the last token's outputs are where a 32-bit element offset would wrap
+    assert bool((GL.B.dx[-1].float().abs().sum() > 0)) and bool((GL.B.x_next[-1].float().abs().sum() > 0))
+    del GL
+    torch.cuda.empty_cache()
+    sk = synth.make_layer_params(wl.n, wl.C, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std, kind="sk")
+    inp_sk = dict(inp, W=sk["W"], b=sk["b"], alpha=sk["alpha"], gain=sk["gain"], N=sk["N"], kind="sk")
+    GS = _run_and_check(wl, "sk", param_grads=False, T=T, inp=inp_sk)
+    GS.ctx.ds_gap(GS.B.H_res, l1, None); torch.cuda.synchronize()
+    assert float(l1.max()) < 1e-4
+    GS.ctx.device_status()
+    del GS
+    torch.cuda.empty_cache()
 
 
 def test_cfg3_stack_of_24_layers():
@@ -140,19 +165,13 @@ def test_cfg3_stack_of_24_layers():
         r = torch.rsqrt(uf.pow(2).mean(-1, keepdim=True) + eps)
         return (r * d - uf * r.pow(3) * (uf * d).sum(-1, keepdim=True) / C).to(torch.bfloat16)
 
-    xs, ys = [L.to_device_bf16(x0, DEV)], []
-    for l in range(Ld):
-        L.pre_fwd(ctx, P[l], Bs[l], xs[l], eps, True)
-        ys.append(standin(Bs[l].u))
-        L.post_fwd(ctx, Bs[l], xs[l], ys[l])
-        xs.append(Bs[l].x_next)
-    gs, dus = {Ld: L.to_device_bf16(gtop, DEV)}, {}
-    for l in reversed(range(Ld)):
-        L.post_bwd(ctx, Bs[l], xs[l], ys[l], gs[l + 1], True)
-        dus[l] = standin_bwd(Bs[l].u, Bs[l].dy)
-        L.tail_bwd(ctx, P[l], Bs[l], xs[l], gs[l + 1], dus[l], eps, True)
-        gs[l] = Bs[l].dx
+    L.stack_fwd(ctx, P, Bs, L.to_device_bf16(x0, DEV), lambda l, u: standin(u), eps)
+    L.stack_bwd(ctx, P, Bs, L.to_device_bf16(gtop, DEV), lambda l, u, dy: standin_bwd(u, dy), eps)
     torch.cuda.synchronize()
+    xs = [B.x_in for B in Bs] + [Bs[-1].x_next]
+    ys = [B.y for B in Bs]
+    gs = {l + 1: Bs[l].g_in for l in range(Ld)}; gs[0] = Bs[0].dx
+    dus = {l: Bs[l].du for l in range(Ld)}
 
     # cumulative product of H_res over depth stays doubly stochastic, for every token
     prod = torch.empty_like(Bs[0].H_res)
@@ -180,6 +199,19 @@ def test_cfg3_stack_of_24_layers():
         check_bf16(f"dy[{l}]", pick(Bs[l].dy), bw["dy"])
         check_bf16(f"dx[{l}]", pick(Bs[l].dx), bw["dx"],
                    extra=dxhat_allowance_f(xl, p["W"], p["alpha"], p["gain"], bw["dz"], eps))
+    # parameter gradients of the first and the last layer over ALL tokens (the oracle is fed the tensors the
+    # GPU layer was fed, in chunks)
+    for l in (0, Ld - 1):
+        p = {k: params[l][k].astype(np.float64) for k in ("W", "b", "alpha", "gain")}
+        acc = None
+        for a in range(0, T, 4096):
+            sl = slice(a, min(T, a + 4096))
+            r = O.layer_bwd(host(xs[l][sl]), host(ys[l][sl]), p["W"], p["b"], p["alpha"], p["gain"], eps,
+                            host(gs[l + 1][sl]), host(dus[l][sl]))
+            part = {k: r[k] for k in ("dW", "db", "dalpha", "dgain")}
+            acc = part if acc is None else {k: acc[k] + part[k] for k in acc}
+        for k in ("dW", "db", "dalpha", "dgain"):
+            check_f32(f"{k}[{l}]", host(getattr(Bs[l], k)), acc[k], 1e-3)
     ref_prod = O.depth_product(oracle_H)
     assert np.abs(pick(prod) - ref_prod).max() < 1e-5
     # end to end: the oracle's own stack (bf16 storage between layers) on the sampled tokens

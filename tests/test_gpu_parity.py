@@ -40,7 +40,7 @@ def test_permutation_table_on_device_bit_exact(n):
     assert (got == O.perm_table(n)).all()
 
 
-@pytest.mark.parametrize("n", [2, 3, 4])
+@pytest.mark.parametrize("n", [2, 3, 4, 5])
 def test_one_hot_weight_selects_each_permutation(n):
     # W = 0, b_res = 0 at k and -200 elsewhere: a = e_k and H_res = P_k exactly (fp32 exp underflows to 0)
     C, T = 64, 5
@@ -188,6 +188,33 @@ def test_sk_gap_vs_lite_on_ill_conditioned_logits():
     assert float(l1.max()) < 4e-6 and float(cd.max()) < 1e-6
 
 
+def test_sk_gap_with_the_papers_initialisation_bias():
+    # Section 4, "Initialization": b_res = -8 off the diagonal, 0 on it (mHC); -8 / 0 at the identity (mHC-lite).
+    # With W != 0 at alpha = 1 the logits spread around that pattern; the SK path's gap must match the oracle's,
+    # mHC-lite has none.
+    n, C, T = 4, 256, 4096
+    sk = synth.make_layer_inputs(n, C, T, seed=6, kind="sk", alpha=[1.0, 1.0, 1.0], w_std=0.1)
+    sk["b"][:] = synth.paper_init_bias(n, "sk")
+    G = GpuLayer(sk, kind="sk"); G.forward()
+    ref = oracle_fwd(sk, kind="sk")
+    compare_forward(G, ref, coeff_rel=1e-4)
+    l1 = torch.empty(T, device=DEV); cd = torch.empty(T, device=DEV)
+    G.ctx.ds_gap(G.B.H_res, l1, cd); torch.cuda.synchronize()
+    gap_ref = O.l1_error(ref["H_res"])
+    assert np.abs(host(l1) - gap_ref).max() <= 1e-2 * gap_ref.max() + 4e-6
+    assert np.abs(host(cd) - np.abs(O.column_sums(ref["H_res"]) - 1).max(axis=1)).max() <= 1e-2 * gap_ref.max() + 4e-6
+    nu = torch.empty(T, device=DEV)
+    M0 = torch.from_numpy(np.ascontiguousarray(ref["M0"], dtype=np.float32)).to(DEV)
+    G.ctx.relative_range(M0, nu); torch.cuda.synchronize()
+    np.testing.assert_allclose(host(nu), O.relative_range(ref["M0"].astype(np.float32).astype(np.float64)), rtol=1e-6)
+    lite = synth.make_layer_inputs(n, C, T, seed=6, alpha=[1.0, 1.0, 1.0], w_std=0.1)
+    lite["b"][:] = synth.paper_init_bias(n)
+    GL = GpuLayer(lite); GL.forward()
+    compare_forward(GL, oracle_fwd(lite), coeff_rel=2e-4)
+    GL.ctx.ds_gap(GL.B.H_res, l1, cd); torch.cuda.synchronize()
+    assert float(l1.max()) < 4e-6 and float(cd.max()) < 1e-6
+
+
 def test_kernel_timing_and_device_status():
     # the library's own per-kernel events and its device status word (bounded waits record a status there)
     n, C, T = 4, 256, 2048
@@ -212,7 +239,7 @@ def test_kernel_timing_of_a_kernel_off_the_path_is_an_argument_error():
     G.ctx.set_kernel_timing(True)
     G.forward(True)
     torch.cuda.synchronize()
-    tail = G.ctx.KERNELS.index("tail_mma")
+    tail = G.ctx.KERNELS.index("tail_dx")
     with pytest.raises(MhcLiteError) as ei:
         G.ctx.kernel_time_ms(tail)
     assert ei.value.status == -1

@@ -37,8 +37,8 @@ def _upstream(G, seed):
             f(synth.normal(seed, 52, (T, n), 8.0)))
 
 
-def test_static_scratch_matches_workspace_entry_point_twice():
-    n, C, T = 4, 256, 700
+@pytest.mark.parametrize("n,C,T", [(4, 256, 700), (3, 72, 130), (5, 40, 70)])
+def test_static_scratch_matches_workspace_entry_point_twice(n, C, T):
     assert _scratch_need(n, C, T) <= load().mhclite_static_scratch_bytes()
     outs = []
     for call, seed in enumerate((61, 62)):           # two calls in a row, different data
@@ -58,21 +58,31 @@ def test_static_scratch_matches_workspace_entry_point_twice():
         dx = torch.full_like(B.dx, float("nan")); dW = torch.full_like(B.dW, float("nan"))
         db = torch.full_like(B.db, float("nan")); dal = torch.full((4,), float("nan"), device=DEV)[:3]
         dg = torch.full_like(B.dgain, float("nan"))
-        bare.coeffs_bwd_static(G.x, P.W, P.alpha, P.gain, 1e-6, B.a_saved, B.p_saved, B.rstd, B.H_pre, B.H_post,
-                               dHr, dHp, dHo, dx, False, dW, db, dal, dg, False)
+        args = (G.x, P.W, P.alpha, P.gain, 1e-6, B.a_saved, B.p_saved, B.rstd, B.H_pre, B.H_post, dHr, dHp, dHo)
+        bare.coeffs_bwd_static(*args, dx, False, dW, db, dal, dg, False)
         torch.cuda.synchronize()
         assert bare._ws is None
-        # the workspace entry point rounds the operands of sum_c e W' to bf16 (tensor cores), this one
-        # keeps them in fp32: allow for that rounding exactly as the parity tests do
+        # against the workspace entry point: that one rounds the operands of sum_c e W' to bf16 (tensor
+        # cores), this one keeps them in fp32; allow for that rounding exactly as the parity tests do
         o = oracle_inputs(inp)
-        dz = O.coeffs_bwd(o["x"], o["W"], o["b"], o["alpha"], o["gain"], 1e-6, host(dHr), host(dHp), host(dHo))["dz"]
-        check_bf16(f"dx (call {call})", host(dx), ref["dx"], extra=dxhat_allowance(inp, dz))
-        check_f32(f"dW (call {call})", host(dW), ref["dW"], 1e-3)
-        check_f32(f"db (call {call})", host(db), ref["db"], 1e-3)
-        check_f32(f"dalpha (call {call})", host(dal), ref["dalpha"], 1e-3)
-        check_f32(f"dgain (call {call})", host(dg), ref["dgain"], 1e-3)
+        orc = O.coeffs_bwd(o["x"], o["W"], o["b"], o["alpha"], o["gain"], 1e-6, host(dHr), host(dHp), host(dHo))
+        check_bf16(f"dx vs workspace call (call {call})", host(dx), ref["dx"], extra=dxhat_allowance(inp, orc["dz"]))
+        check_f32(f"dW vs workspace call (call {call})", host(dW), ref["dW"], 1e-3)
+        check_f32(f"db vs workspace call (call {call})", host(db), ref["db"], 1e-3)
+        check_f32(f"dalpha vs workspace call (call {call})", host(dal), ref["dalpha"], 1e-3)
+        check_f32(f"dgain vs workspace call (call {call})", host(dg), ref["dgain"], 1e-3)
+        # and against the oracle's gradient of the mappings itself (no allowance: fp32 operands here)
+        check_bf16(f"dx vs oracle (call {call})", host(dx), orc["dx"])
+        for k, got in (("dW", dW), ("db", db), ("dalpha", dal), ("dgain", dg)):
+            check_f32(f"{k} vs oracle (call {call})", host(got), orc[k], 1e-3)
         assert np.abs(ref["dW"]).max() > 0 and np.isfinite(host(dx)).all()
-        outs.append(host(dW))
+        # both accumulate flags: a second call adds the same gradients on top
+        bare.coeffs_bwd_static(*args, dx, True, dW, db, dal, dg, True)
+        torch.cuda.synchronize()
+        check_bf16(f"dx x2 (call {call})", host(dx), 2 * orc["dx"], rel=3e-2)
+        for k, got in (("dW", dW), ("db", db), ("dalpha", dal), ("dgain", dg)):
+            check_f32(f"{k} x2 (call {call})", host(got), 2 * orc[k], 1e-3)
+        outs.append(ref["dW"])
     assert np.abs(outs[0] - outs[1]).max() > 0        # the two calls really computed different things
 
 
