@@ -37,6 +37,8 @@ SIGNATURES = {
     "mhclite_perm_table_device": (_i, [_p, _p]),
     "mhclite_workspace_bytes": (_sz, [_i, _i, _i64, _i]),
     "mhclite_set_workspace": (_i, [_p, _p, _sz]),
+    "mhclite_set_perm_subset": (_i, [_p, _i, _p]),
+    "mhclite_workspace_bytes_subset": (_sz, [_i, _i, _i64, _i]),
     "mhclite_coeffs_fwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p]),
     "mhclite_premix_fwd": (_i, [_p, _i64, _p, _p, _p, _p]),
     "mhclite_postres_fwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p]),
@@ -51,6 +53,7 @@ SIGNATURES = {
     "mhclite_tail_bwd_fused": (_i, [_p, _i64, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p, _p, _p,
                                     _p, _p, _p, _p, _p, _i, _p]),
     "mhc_sk20_coeffs_fwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _i, _p, _p, _p, _p, _p, _p]),
+    "mhc_sk20_pre_fwd_fused": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _i, _p, _p, _p, _p, _p, _p, _p]),
     "mhc_sk20_coeffs_bwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _i, _p, _p, _p, _p, _p, _p, _p, _p, _i,
                                  _p, _p, _p, _p, _i, _p]),
     "mhc_sk20_tail_bwd_fused": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _i, _p, _p, _p, _p, _p, _p, _p, _p, _p,
@@ -113,7 +116,8 @@ class MhcLite:
         self._torch = torch
         self.lib = load()
         self.n, self.C, self.device = n, C_, device
-        self.nfact = math.factorial(n)
+        self.nfact = math.factorial(n)          # residual weights per token (K once a subset is attached)
+        self._table = None
         h = _p()
         rc = self.lib.mhclite_create(C.byref(h), n, C_, device)
         if rc:
@@ -149,9 +153,23 @@ class MhcLite:
     def n_cols(self, kind: int = 0) -> int:
         return (self.nfact if kind == 0 else self.n * self.n) + 2 * self.n
 
+    def set_perm_subset(self, table):
+        """Attaches a table [K, n] (uint8 tensor on the device, or None) of K distinct permutations:
+        Eq. (5) then runs over those K matrices only (paper Section 5)."""
+        if table is None:
+            self._check(self.lib.mhclite_set_perm_subset(self._h, 0, None), "mhclite_set_perm_subset")
+            self._table, self.nfact = None, math.factorial(self.n)
+            return
+        if table.dtype != self._torch.uint8 or table.dim() != 2 or table.shape[1] != self.n:
+            raise ValueError("expected a uint8 tensor of shape [K, n]")
+        self._check(self.lib.mhclite_set_perm_subset(self._h, table.shape[0], self._ptr(table)), "mhclite_set_perm_subset")
+        self._table, self.nfact = table, int(table.shape[0])
+
     def ensure_workspace(self, T: int, kind: int = 0):
         """Allocates (with torch) and attaches scratch large enough for T tokens."""
-        need = max(workspace_bytes(self.n, self.C, T, 0), workspace_bytes(self.n, self.C, T, kind))
+        lite = (workspace_bytes(self.n, self.C, T, 0) if self._table is None else
+                int(self.lib.mhclite_workspace_bytes_subset(self.n, self.C, T, self.nfact)))
+        need = max(lite, workspace_bytes(self.n, self.C, T, kind) if kind else 0)
         if self._ws is None or self._ws.numel() < need:
             self._ws = self._torch.empty(need + 256, dtype=self._torch.uint8, device=f"cuda:{self.device}")
             base = self._ws.data_ptr()
@@ -248,6 +266,14 @@ class MhcLite:
             self._h, x.shape[0], self._ptr(x, h), self._ptr(W_sk, f), self._ptr(b_sk, f), self._ptr(alpha, f),
             self._ptr(gain, f), float(eps), int(iters), self._ptr(H_res, f), self._ptr(H_pre, f), self._ptr(H_post, f),
             self._ptr(p_saved, f), self._ptr(rstd, f), self._stream()), "mhc_sk20_coeffs_fwd")
+
+    def sk20_pre_fwd_fused(self, x, W_sk, b_sk, alpha, gain, eps, iters, H_res, H_pre, H_post, p_saved, rstd, u):
+        f, h = self._torch.float32, self._torch.bfloat16
+        self.ensure_workspace(x.shape[0], 1)
+        self._check(self.lib.mhc_sk20_pre_fwd_fused(
+            self._h, x.shape[0], self._ptr(x, h), self._ptr(W_sk, f), self._ptr(b_sk, f), self._ptr(alpha, f),
+            self._ptr(gain, f), float(eps), int(iters), self._ptr(H_res, f), self._ptr(H_pre, f), self._ptr(H_post, f),
+            self._ptr(p_saved, f), self._ptr(rstd, f), self._ptr(u, h), self._stream()), "mhc_sk20_pre_fwd_fused")
 
     def sk20_coeffs_bwd(self, x, W_sk, b_sk, alpha, gain, eps, iters, p_saved, rstd, H_pre, H_post, dH_res, dH_pre,
                         dH_post, dx, accumulate_dx, dW, db, dalpha, dgain, accumulate_params=False):

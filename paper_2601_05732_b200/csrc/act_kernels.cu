@@ -89,9 +89,15 @@ struct LiteShared {
     float dh_s[kActWarps][32];
     float red[kActWarps][kMaxCols + 3];
 };
-__device__ __forceinline__ void load_tables(LiteShared& sh, int n) {
-    const PermTables& tab = c_perm[n];
-    for (int i = threadIdx.x; i < kMaxFact * kMaxN; i += blockDim.x) { sh.sigma[i] = tab.sigma[i]; sh.klist[i] = tab.klist[i]; }
+// `table` (global memory, [nf][n]) replaces the constant-memory table when the context holds a subset of the
+// permutations (paper Section 5); there are then no per-entry index lists, and H_res is assembled from sigma.
+__device__ __forceinline__ void load_tables(LiteShared& sh, int n, int nf, const uint8_t* __restrict__ table) {
+    if (table) {
+        for (int i = threadIdx.x; i < nf * n; i += blockDim.x) sh.sigma[i] = table[i];
+    } else {
+        const PermTables& tab = c_perm[n];
+        for (int i = threadIdx.x; i < kMaxFact * kMaxN; i += blockDim.x) { sh.sigma[i] = tab.sigma[i]; sh.klist[i] = tab.klist[i]; }
+    }
     __syncthreads();
 }
 
@@ -102,7 +108,7 @@ __device__ __forceinline__ float lite_token_fwd_core(LiteShared& sh, int w, int 
                                                      const float* pt, const float* __restrict__ b, float a_res,
                                                      float a_pre, float a_post, float* __restrict__ H_res,
                                                      float* __restrict__ H_pre, float* __restrict__ H_post,
-                                                     float* __restrict__ a_saved) {
+                                                     float* __restrict__ a_saved, bool subset = false) {
     const int per = nf / n, nn = n * n;
     float z[4], m = -INFINITY;
 #pragma unroll
@@ -138,7 +144,12 @@ __device__ __forceinline__ float lite_token_fwd_core(LiteShared& sh, int w, int 
     __syncwarp();
     if (lane < nn) {
         float h = 0.f;
-        for (int r = 0; r < per; ++r) h += sh.a_s[w][sh.klist[lane * per + r]];
+        if (subset) {                                   // Eq. (5) over the table's rows: P_k[i][sigma_k(i)] = 1
+            const int i = lane / n, j = lane - i * n;
+            for (int k = 0; k < nf; ++k) h += (sh.sigma[k * n + i] == j) ? sh.a_s[w][k] : 0.f;
+        } else {
+            for (int r = 0; r < per; ++r) h += sh.a_s[w][sh.klist[lane * per + r]];
+        }
         H_res[t * nn + lane] = h;
     }
     __syncwarp();
@@ -152,14 +163,15 @@ __device__ __forceinline__ float lite_token_fwd(LiteShared& sh, int w, int lane,
                                                 const float* __restrict__ b, float a_res, float a_pre, float a_post,
                                                 float* __restrict__ H_res, float* __restrict__ H_pre,
                                                 float* __restrict__ H_post, float* __restrict__ a_saved,
-                                                float* __restrict__ p_saved, float* __restrict__ rstd) {
+                                                float* __restrict__ p_saved, float* __restrict__ rstd, bool subset) {
     const int N = nf + 2 * n;
     float pv[5];
     finish_projection(t, T, N, Npad, ksplit, inv_nC, eps, qpart, ssq, p_saved, rstd, lane, pv);
 #pragma unroll
     for (int k = 0; k < 5; ++k) if (lane + 32 * k < N) sh.p_s[w][lane + 32 * k] = pv[k];
     __syncwarp();
-    return lite_token_fwd_core(sh, w, lane, t, n, nf, sh.p_s[w], b, a_res, a_pre, a_post, H_res, H_pre, H_post, a_saved);
+    return lite_token_fwd_core(sh, w, lane, t, n, nf, sh.p_s[w], b, a_res, a_pre, a_post, H_res, H_pre, H_post, a_saved,
+                               subset);
 }
 
 __global__ void __launch_bounds__(kActThreads) lite_act_fwd_k(int64_t T, int n, int nf, int Npad, int ksplit,
@@ -168,15 +180,16 @@ __global__ void __launch_bounds__(kActThreads) lite_act_fwd_k(int64_t T, int n, 
                                                              const float* __restrict__ b, const float* __restrict__ alpha,
                                                              float* __restrict__ H_res, float* __restrict__ H_pre,
                                                              float* __restrict__ H_post, float* __restrict__ a_saved,
-                                                             float* __restrict__ p_saved, float* __restrict__ rstd) {
+                                                             float* __restrict__ p_saved, float* __restrict__ rstd,
+                                                             const uint8_t* __restrict__ table) {
     __shared__ LiteShared sh;
-    load_tables(sh, n);
+    load_tables(sh, n, nf, table);
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
     const int64_t nwarps = (int64_t)gridDim.x * kActWarps;
     for (int64_t t = (int64_t)blockIdx.x * kActWarps + w; t < T; t += nwarps)
         lite_token_fwd(sh, w, lane, t, T, n, nf, Npad, ksplit, inv_nC, eps, qpart, ssq, b, a_res, a_pre, a_post,
-                       H_res, H_pre, H_post, a_saved, p_saved, rstd);
+                       H_res, H_pre, H_post, a_saved, p_saved, rstd, table != nullptr);
 }
 
 // Mappings + stream pre-mix in one kernel, in groups of kGroupTok tokens per block:
@@ -191,12 +204,13 @@ __global__ void __launch_bounds__(kActThreads) lite_act_premix_k(
     int64_t T, int C8, int nf, int Npad, int ksplit, float inv_nC, float eps, const float* __restrict__ qpart,
     const float* __restrict__ ssq, const float* __restrict__ b, const float* __restrict__ alpha,
     float* __restrict__ H_res, float* __restrict__ H_pre, float* __restrict__ H_post, float* __restrict__ a_saved,
-    float* __restrict__ p_saved, float* __restrict__ rstd, const uint4* __restrict__ x, uint4* __restrict__ u) {
+    float* __restrict__ p_saved, float* __restrict__ rstd, const uint4* __restrict__ x, uint4* __restrict__ u,
+    const uint8_t* __restrict__ table) {
     __shared__ LiteShared sh;
     __shared__ float pg[kGroupTok][kMaxCols + 3];
     __shared__ float rg[kGroupTok];
     __shared__ float hg[kGroupTok][kMaxN];
-    load_tables(sh, N_);
+    load_tables(sh, N_, nf, table);
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int N = nf + 2 * N_;
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
@@ -230,7 +244,7 @@ __global__ void __launch_bounds__(kActThreads) lite_act_premix_k(
         // A
         for (int tl = w; tl < nt; tl += kActWarps) {
             const float gate = lite_token_fwd_core(sh, w, lane, t0 + tl, N_, nf, pg[tl], b, a_res, a_pre, a_post, H_res,
-                                                   H_pre, H_post, a_saved);
+                                                   H_pre, H_post, a_saved, table != nullptr);
             if (lane < N_) hg[tl][lane] = gate;
         }
         __syncthreads();
@@ -337,9 +351,10 @@ __global__ void __launch_bounds__(kActThreads) lite_act_bwd_k(
     int64_t T, int n, int nf, float inv_nC, const float* __restrict__ a_saved, const float* __restrict__ p,
     const float* __restrict__ rstd, const float* __restrict__ alpha, const float* __restrict__ H_pre,
     const float* __restrict__ H_post, const float* __restrict__ dH_res, const float* __restrict__ dH_pre,
-    const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa, float* db, float* dalpha) {
+    const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa, float* db, float* dalpha,
+    const uint8_t* __restrict__ table) {
     __shared__ LiteShared sh;
-    load_tables(sh, n);
+    load_tables(sh, n, nf, table);
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
     LiteBwdAcc acc = {{0, 0, 0, 0}, 0.f, 0.f, 0.f};
@@ -365,7 +380,7 @@ __global__ void __launch_bounds__(kActThreads) lite_tailpre_k(
     const float* __restrict__ a_saved, const float* __restrict__ p, const float* __restrict__ rstd,
     const float* __restrict__ alpha, const float* __restrict__ H_pre, const float* __restrict__ H_post,
     const float* __restrict__ dH_res, const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa,
-    float* db, float* dalpha) {
+    float* db, float* dalpha, const uint8_t* __restrict__ table) {
     __shared__ LiteShared sh;
     constexpr int NN = N_ * N_;
     constexpr int kFact = (N_ == 2) ? 2 : (N_ == 3) ? 6 : (N_ == 4) ? 24 : 120;
@@ -373,7 +388,7 @@ __global__ void __launch_bounds__(kActThreads) lite_tailpre_k(
     constexpr int kGroupTok = (N_ == 5) ? 16 : 32;              // keeps the staging under the static shared-memory limit
     __shared__ float in_s[kGroupTok][kStride];
     __shared__ float dhp_s[kGroupTok][kMaxN];
-    load_tables(sh, N_);
+    load_tables(sh, N_, nf, table);
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int N = nf + 2 * N_;
     const int o_p = nf, o_dhres = o_p + N, o_hpre = o_dhres + NN, o_hpost = o_hpre + N_, o_dhpost = o_hpost + N_,
@@ -723,8 +738,9 @@ __device__ __forceinline__ void sk_forward(float (&M)[N_][N_], int iters, float*
 #pragma unroll
             for (int i = 0; i < N_; ++i) s += M[i][j];
             if (cs_store) cs_store[it * N_ + j] = s;
+            const float r = 1.f / s;                     // one division per column / row, n multiplications
 #pragma unroll
-            for (int i = 0; i < N_; ++i) M[i][j] = M[i][j] / s;
+            for (int i = 0; i < N_; ++i) M[i][j] *= r;
         }
 #pragma unroll
         for (int i = 0; i < N_; ++i) {
@@ -732,8 +748,9 @@ __device__ __forceinline__ void sk_forward(float (&M)[N_][N_], int iters, float*
 #pragma unroll
             for (int j = 0; j < N_; ++j) s += M[i][j];
             if (rs_store) rs_store[it * N_ + i] = s;
+            const float r = 1.f / s;
 #pragma unroll
-            for (int j = 0; j < N_; ++j) M[i][j] = M[i][j] / s;
+            for (int j = 0; j < N_; ++j) M[i][j] *= r;
         }
     }
 }
@@ -793,6 +810,82 @@ __global__ void __launch_bounds__(128) sk_act_fwd_k(int64_t T, int iters, int Np
 
 constexpr int kSkMaxIters = 64;
 
+// Backward of one token through the SK path (one thread): recomputes the forward keeping the 2 * iters * n
+// normalisers, walks the iterates back (X = Y s), goes through exp, and emits e = rstd alpha dz, kappa and the
+// token's contributions to db / dalpha (shared-memory accumulators red[N + 3]).
+template <int N_>
+__device__ __forceinline__ void sk_token_bwd(int64_t t, int iters, float inv_nC, const float* pt, const float* __restrict__ b,
+                                             float r, float a_res, float a_pre, float a_post, const float* hpre,
+                                             const float* hpost, const float* dhres, const float* dhpre,
+                                             const float* dhpost, const EOut& eo, float* __restrict__ kappa, float* red) {
+    constexpr int N = N_ * N_ + 2 * N_;
+    float cs[kSkMaxIters * N_], rs[kSkMaxIters * N_];
+    float Y[N_][N_];
+    sk_load_m0<N_>(pt, b, a_res, Y);
+    sk_forward<N_>(Y, iters, cs, rs);
+    float d[N_][N_];
+#pragma unroll
+    for (int i = 0; i < N_; ++i)
+#pragma unroll
+        for (int j = 0; j < N_; ++j) d[i][j] = dhres[i * N_ + j];
+    for (int it = iters - 1; it >= 0; --it) {
+        // rows: Y = X / s  ->  dX = (dY - <dY,Y>_row) / s ; X = Y s
+#pragma unroll
+        for (int i = 0; i < N_; ++i) {
+            const float s = rs[it * N_ + i], rinv = 1.f / s;
+            float dot = 0.f;
+#pragma unroll
+            for (int j = 0; j < N_; ++j) dot = fmaf(d[i][j], Y[i][j], dot);
+#pragma unroll
+            for (int j = 0; j < N_; ++j) { d[i][j] = (d[i][j] - dot) * rinv; Y[i][j] *= s; }
+        }
+        // columns
+#pragma unroll
+        for (int j = 0; j < N_; ++j) {
+            const float s = cs[it * N_ + j], rinv = 1.f / s;
+            float dot = 0.f;
+#pragma unroll
+            for (int i = 0; i < N_; ++i) dot = fmaf(d[i][j], Y[i][j], dot);
+#pragma unroll
+            for (int i = 0; i < N_; ++i) { d[i][j] = (d[i][j] - dot) * rinv; Y[i][j] *= s; }
+        }
+    }
+    // through exp: dz = dM0 * M0, with M0 taken from the logits again (not from the walk-back)
+    sk_load_m0<N_>(pt, b, a_res, Y);
+    float kap = 0.f, dal0 = 0.f, dal1 = 0.f, dal2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < N_; ++i)
+#pragma unroll
+        for (int j = 0; j < N_; ++j) {
+            const int c = i * N_ + j;
+            const float dz = d[i][j] * Y[i][j], pv = pt[c], ed = a_res * dz;
+            store_e(eo, t, c, r * ed);
+            kap = fmaf(ed, pv, kap);
+            dal0 = fmaf(dz, pv, dal0);
+            atomicAdd(&red[c], dz);
+        }
+#pragma unroll
+    for (int j = 0; j < N_; ++j) {
+        {
+            const int c = N_ * N_ + j;
+            const float h = hpre[j];
+            const float dz = dhpre[j] * h * (1.f - h), pv = pt[c], ed = a_pre * dz;
+            store_e(eo, t, c, r * ed); kap = fmaf(ed, pv, kap); dal1 = fmaf(dz, pv, dal1);
+            atomicAdd(&red[c], dz);
+        }
+        {
+            const int c = N_ * N_ + N_ + j;
+            const float h = hpost[j];
+            const float dz = dhpost[j] * h * (1.f - 0.5f * h), pv = pt[c], ed = a_post * dz;
+            store_e(eo, t, c, r * ed); kap = fmaf(ed, pv, kap); dal2 = fmaf(dz, pv, dal2);
+            atomicAdd(&red[c], dz);
+        }
+    }
+    pad_e(eo, t, N, 0, 1);
+    kappa[t] = r * r * kap * inv_nC;
+    atomicAdd(&red[N], dal0); atomicAdd(&red[N + 1], dal1); atomicAdd(&red[N + 2], dal2);
+}
+
 template <int N_>
 __global__ void __launch_bounds__(128) sk_act_bwd_k(
     int64_t T, int iters, float inv_nC, const float* __restrict__ p, const float* __restrict__ b,
@@ -804,78 +897,190 @@ __global__ void __launch_bounds__(128) sk_act_bwd_k(
     for (int c = threadIdx.x; c < N + 3; c += blockDim.x) red[c] = 0.f;
     __syncthreads();
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t < T) {
-        const float* pt = p + t * N;
-        const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
-        float cs[kSkMaxIters * N_], rs[kSkMaxIters * N_];
-        float Y[N_][N_];
-        sk_load_m0<N_>(pt, b, a_res, Y);
-        sk_forward<N_>(Y, iters, cs, rs);
-        float d[N_][N_];
-#pragma unroll
-        for (int i = 0; i < N_; ++i)
-#pragma unroll
-            for (int j = 0; j < N_; ++j) d[i][j] = dH_res[t * N_ * N_ + i * N_ + j];
-        for (int it = iters - 1; it >= 0; --it) {
-            // rows: Y = X / s  ->  dX = (dY - <dY,Y>_row) / s ; X = Y s
-#pragma unroll
-            for (int i = 0; i < N_; ++i) {
-                const float s = rs[it * N_ + i];
-                float dot = 0.f;
-#pragma unroll
-                for (int j = 0; j < N_; ++j) dot = fmaf(d[i][j], Y[i][j], dot);
-#pragma unroll
-                for (int j = 0; j < N_; ++j) { d[i][j] = (d[i][j] - dot) / s; Y[i][j] *= s; }
-            }
-            // columns
-#pragma unroll
-            for (int j = 0; j < N_; ++j) {
-                const float s = cs[it * N_ + j];
-                float dot = 0.f;
-#pragma unroll
-                for (int i = 0; i < N_; ++i) dot = fmaf(d[i][j], Y[i][j], dot);
-#pragma unroll
-                for (int i = 0; i < N_; ++i) { d[i][j] = (d[i][j] - dot) / s; Y[i][j] *= s; }
-            }
-        }
-        // through exp: dz = dM0 * M0, with M0 taken from the logits again (not from the walk-back)
-        sk_load_m0<N_>(pt, b, a_res, Y);
-        const float r = __ldg(rstd + t);
-        float kap = 0.f, dal0 = 0.f, dal1 = 0.f, dal2 = 0.f;
-#pragma unroll
-        for (int i = 0; i < N_; ++i)
-#pragma unroll
-            for (int j = 0; j < N_; ++j) {
-                const int c = i * N_ + j;
-                const float dz = d[i][j] * Y[i][j], pv = pt[c], ed = a_res * dz;
-                store_e(eo, t, c, r * ed);
-                kap = fmaf(ed, pv, kap);
-                dal0 = fmaf(dz, pv, dal0);
-                atomicAdd(&red[c], dz);
-            }
-#pragma unroll
-        for (int j = 0; j < N_; ++j) {
-            {
-                const int c = N_ * N_ + j;
-                const float h = H_pre[t * N_ + j];
-                const float dz = dH_pre[t * N_ + j] * h * (1.f - h), pv = pt[c], ed = a_pre * dz;
-                store_e(eo, t, c, r * ed); kap = fmaf(ed, pv, kap); dal1 = fmaf(dz, pv, dal1);
-                atomicAdd(&red[c], dz);
-            }
-            {
-                const int c = N_ * N_ + N_ + j;
-                const float h = H_post[t * N_ + j];
-                const float dz = dH_post[t * N_ + j] * h * (1.f - 0.5f * h), pv = pt[c], ed = a_post * dz;
-                store_e(eo, t, c, r * ed); kap = fmaf(ed, pv, kap); dal2 = fmaf(dz, pv, dal2);
-                atomicAdd(&red[c], dz);
-            }
-        }
-        pad_e(eo, t, N, 0, 1);
-        kappa[t] = r * r * kap * inv_nC;
-        atomicAdd(&red[N], dal0); atomicAdd(&red[N + 1], dal1); atomicAdd(&red[N + 2], dal2);
-    }
+    if (t < T)
+        sk_token_bwd<N_>(t, iters, inv_nC, p + t * N, b, __ldg(rstd + t), __ldg(alpha), __ldg(alpha + 1), __ldg(alpha + 2),
+                         H_pre + t * N_, H_post + t * N_, dH_res + t * N_ * N_, dH_pre + t * N_, dH_post + t * N_, eo,
+                         kappa, red);
     __syncthreads();
     for (int c = threadIdx.x; c < N + 3; c += blockDim.x) {
+        if (c < N) atomicAdd(db + c, red[c]); else atomicAdd(dalpha + (c - N), red[c]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// The SK path's fused kernels, built like the mHC-lite ones so that the comparison is like for like:
+// sk_act_premix_k = SK activation + stream pre-mix (one thread per token for the 20 iterations, then all threads
+// stream the group's tokens); sk_tailpre_k = dH_pre stream (one warp per token) + SK backward (one thread per token).
+// ------------------------------------------------------------------------------------------------
+constexpr int kSkGroup = 64;     // tokens per block iteration
+
+template <int N_>
+__global__ void __launch_bounds__(kActThreads, 3) sk_act_premix_k(
+    int64_t T, int C8, int iters, int Npad, int ksplit, float inv_nC, float eps, const float* __restrict__ qpart,
+    const float* __restrict__ ssq, const float* __restrict__ b, const float* __restrict__ alpha,
+    float* __restrict__ H_res, float* __restrict__ H_pre, float* __restrict__ H_post, float* __restrict__ p_saved,
+    float* __restrict__ rstd, const uint4* __restrict__ x, uint4* __restrict__ u) {
+    constexpr int NN = N_ * N_, N = NN + 2 * N_;
+    __shared__ float pg[kSkGroup][N + 1];
+    __shared__ float og[kSkGroup][N + 1];          // H_res | H_pre | H_post
+    __shared__ float rg[kSkGroup];
+    const int tid = threadIdx.x;
+    const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
+    const int64_t ngroups = (T + kSkGroup - 1) / kSkGroup;
+    for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
+        // descending: the projection kernel before this one read x in ascending order and left its last lines in L2
+        const int64_t t0 = (ngroups - 1 - grp) * kSkGroup;
+        const int nt = (T - t0 < kSkGroup) ? (int)(T - t0) : kSkGroup;
+        if (tid < nt) {
+            float ss = 0.f;
+            for (int s = 0; s < ksplit; ++s) ss += __ldg(ssq + (int64_t)s * T + t0 + tid);
+            const float r = 1.f / sqrtf(ss * inv_nC + eps);
+            rg[tid] = r;
+            rstd[t0 + tid] = r;
+        }
+        __syncthreads();
+        for (int i = tid; i < nt * N; i += kActThreads) {
+            const int tl = i / N, c = i - tl * N;
+            float q = 0.f;
+            for (int s = 0; s < ksplit; ++s) q += __ldg(qpart + ((int64_t)s * T + t0 + tl) * Npad + c);
+            const float pv = q * rg[tl];
+            pg[tl][c] = pv;
+            p_saved[(t0 + tl) * N + c] = pv;
+        }
+        __syncthreads();
+        if (tid < nt) {                            // one thread per token: exp, the SK iterations, the gates
+            float M[N_][N_];
+            sk_load_m0<N_>(pg[tid], b, a_res, M);
+            sk_forward<N_>(M, iters, nullptr, nullptr);
+#pragma unroll
+            for (int i = 0; i < N_; ++i)
+#pragma unroll
+                for (int j = 0; j < N_; ++j) og[tid][i * N_ + j] = M[i][j];
+#pragma unroll
+            for (int j = 0; j < N_; ++j) {
+                og[tid][NN + j] = sigmoidf_(fmaf(a_pre, pg[tid][NN + j], __ldg(b + NN + j)));
+                og[tid][NN + N_ + j] = 2.f * sigmoidf_(fmaf(a_post, pg[tid][NN + N_ + j], __ldg(b + NN + N_ + j)));
+            }
+        }
+        __syncthreads();
+        for (int i = tid; i < nt * N; i += kActThreads) {
+            const int tl = i / N, c = i - tl * N;
+            const int64_t t = t0 + tl;
+            const float v = og[tl][c];
+            if (c < NN) H_res[t * NN + c] = v;
+            else if (c < NN + N_) H_pre[t * N_ + (c - NN)] = v;
+            else H_post[t * N_ + (c - NN - N_)] = v;
+        }
+        // u[t,:] = sum_j H_pre[t,j] x[t,j,:]  (two vectors per thread in flight)
+        for (int i0 = tid; i0 < nt * C8; i0 += 2 * kActThreads) {
+            const int i1 = i0 + kActThreads;
+            const bool has1 = i1 < nt * C8;
+            const int tl0 = i0 / C8, cv0 = i0 - tl0 * C8;
+            const int tl1 = has1 ? i1 / C8 : tl0, cv1 = has1 ? i1 - tl1 * C8 : cv0;
+            uint4 v0[N_], v1[N_];
+#pragma unroll
+            for (int j = 0; j < N_; ++j) v0[j] = ld_stream(x + ((t0 + tl0) * N_ + j) * C8 + cv0);
+#pragma unroll
+            for (int j = 0; j < N_; ++j) v1[j] = ld_stream(x + ((t0 + tl1) * N_ + j) * C8 + cv1);
+            float acc0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, acc1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+            for (int j = 0; j < N_; ++j) {
+                const float h0 = og[tl0][NN + j], h1 = og[tl1][NN + j];
+                float f0[8], f1[8];
+                unpack8(v0[j], f0);
+                unpack8(v1[j], f1);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { acc0[e] = fmaf(h0, f0[e], acc0[e]); acc1[e] = fmaf(h1, f1[e], acc1[e]); }
+            }
+            st_stream(u + (t0 + tl0) * C8 + cv0, pack8(acc0));
+            if (has1) st_stream(u + (t0 + tl1) * C8 + cv1, pack8(acc1));
+        }
+        __syncthreads();
+    }
+}
+
+template <int N_>
+__global__ void __launch_bounds__(kActThreads, 3) sk_tailpre_k(
+    int64_t T, int C8, int iters, float inv_nC, const uint4* __restrict__ x, const uint4* __restrict__ du,
+    const float* __restrict__ p, const float* __restrict__ b, const float* __restrict__ rstd,
+    const float* __restrict__ alpha, const float* __restrict__ H_pre, const float* __restrict__ H_post,
+    const float* __restrict__ dH_res, const float* __restrict__ dH_post, const EOut eo, float* __restrict__ kappa,
+    float* db, float* dalpha) {
+    constexpr int NN = N_ * N_, N = NN + 2 * N_;
+    constexpr int o_dhres = N, o_hpre = o_dhres + NN, o_hpost = o_hpre + N_, o_dhpost = o_hpost + N_, o_rstd = o_dhpost + N_,
+                  nin = o_rstd + 1;
+    __shared__ float in_s[kSkGroup][nin];          // p | dH_res | H_pre | H_post | dH_post | rstd of the group's tokens
+    __shared__ float dhp_s[kSkGroup][kMaxN];
+    __shared__ float red[N + 3];
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    for (int c = tid; c < N + 3; c += kActThreads) red[c] = 0.f;
+    __syncthreads();
+    const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
+    const int64_t ngroups = (T + kSkGroup - 1) / kSkGroup;
+    for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
+        const int64_t t0 = grp * kSkGroup;
+        const int nt = (T - t0 < kSkGroup) ? (int)(T - t0) : kSkGroup;
+        // the per-token inputs of the SK backward travel to shared memory while the warps stream x and du
+        for (int i = tid; i < nt * nin; i += kActThreads) {
+            const int tl = i / nin, c = i - tl * nin;
+            const int64_t t = t0 + tl;
+            const float* src;
+            if (c < o_dhres) src = p + t * N + c;
+            else if (c < o_hpre) src = dH_res + t * NN + (c - o_dhres);
+            else if (c < o_hpost) src = H_pre + t * N_ + (c - o_hpre);
+            else if (c < o_dhpost) src = H_post + t * N_ + (c - o_hpost);
+            else if (c < o_rstd) src = dH_post + t * N_ + (c - o_dhpost);
+            else src = rstd + t;
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&in_s[tl][c])), "l"(src) : "memory");
+        }
+        cp_async_commit();
+        // dH_pre[j] = <du, x_j>, one warp per token
+        for (int tl = w; tl < nt; tl += kActWarps) {
+            const int64_t t = t0 + tl;
+            float r[N_];
+#pragma unroll
+            for (int j = 0; j < N_; ++j) r[j] = 0.f;
+            for (int cv0 = lane; cv0 < C8; cv0 += 64) {
+                uint4 xv[2][N_], dv[2];
+#pragma unroll
+                for (int v = 0; v < 2; ++v) {
+                    const int cv = cv0 + 32 * v;
+                    if (cv < C8) {
+#pragma unroll
+                        for (int j = 0; j < N_; ++j) xv[v][j] = ld_stream(x + (t * N_ + j) * C8 + cv);
+                        dv[v] = ld_stream(du + t * C8 + cv);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < N_; ++j) xv[v][j] = make_uint4(0, 0, 0, 0);
+                        dv[v] = make_uint4(0, 0, 0, 0);
+                    }
+                }
+#pragma unroll
+                for (int v = 0; v < 2; ++v) {
+                    float df[8];
+                    unpack8(dv[v], df);
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) {
+                        float xf[8];
+                        unpack8(xv[v][j], xf);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) r[j] = fmaf(df[e], xf[e], r[j]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < N_; ++j) { r[j] = warp_sum(r[j]); if (lane == j) dhp_s[tl][j] = r[j]; }
+        }
+        cp_async_wait<0>();
+        __syncthreads();
+        if (tid < nt) {
+            const float* in = in_s[tid];
+            sk_token_bwd<N_>(t0 + tid, iters, inv_nC, in, b, in[o_rstd], a_res, a_pre, a_post, in + o_hpre, in + o_hpost,
+                             in + o_dhres, dhp_s[tid], in + o_dhpost, eo, kappa, red);
+        }
+        __syncthreads();
+    }
+    for (int c = tid; c < N + 3; c += kActThreads) {
         if (c < N) atomicAdd(db + c, red[c]); else atomicAdd(dalpha + (c - N), red[c]);
     }
 }
@@ -901,7 +1106,7 @@ void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, co
     c->launches += 1;
     lite_act_fwd_k<<<warp_grid(T, c->sm_count), kActThreads, 0, s>>>(
         T, c->n, c->nfact, pp.Npad, pp.ksplit, 1.f / (float)(c->n * c->C), eps, qpart, ssq, b, alpha, H_res, H_pre,
-        H_post, a_saved, p_saved, rstd);
+        H_post, a_saved, p_saved, rstd, c->table_dev);
 }
 
 void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float* a, const float* p, const float* rstd,
@@ -917,7 +1122,7 @@ void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float*
     if (blocks < 1) blocks = 1;
     lite_act_bwd_k<<<(int)blocks, kActThreads, 0, s>>>(T, c->n, c->nfact, 1.f / (float)(c->n * c->C), a, p, rstd,
                                                         alpha, H_pre, H_post, dH_res, dH_pre, dH_post, eo, kappa, db,
-                                                        dalpha);
+                                                        dalpha, c->table_dev);
 }
 
 void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, const float* qpart, const float* ssq,
@@ -930,15 +1135,22 @@ void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp,
 #define MHCL_AP_T(N_) lite_act_premix_t_k<N_><<<group_grid(T, kTokGroup, c->sm_count), kActThreads, 0, s>>>( \
         T, C8, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, \
         (const uint4*)x, (uint4*)u)
-    switch (c->n) {
-        case 2: MHCL_AP_T(2); break;
-        case 3: MHCL_AP_T(3); break;
-        case 4: MHCL_AP_T(4); break;
-        default:    // n = 5: 120 logits do not fit a thread's registers; one warp per token
-            lite_act_premix_k<5><<<group_grid(T, kGroupTok, c->sm_count), kActThreads, 0, s>>>(
-                T, C8, c->nfact, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b, alpha, H_res, H_pre, H_post, a_saved,
-                p_saved, rstd, (const uint4*)x, (uint4*)u);
+    // one warp per token: n = 5 (120 logits do not fit a thread's registers) and every context that holds a
+    // subset of the permutations (its table is data, not a compile-time constant)
+#define MHCL_AP_W(N_) lite_act_premix_k<N_><<<group_grid(T, kGroupTok, c->sm_count), kActThreads, 0, s>>>( \
+        T, C8, c->nfact, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b, alpha, H_res, H_pre, H_post, a_saved, \
+        p_saved, rstd, (const uint4*)x, (uint4*)u, c->table_dev)
+    if (c->table_dev) {
+        MHCL_DISPATCH_N(c->n, MHCL_AP_W(N_));
+    } else {
+        switch (c->n) {
+            case 2: MHCL_AP_T(2); break;
+            case 3: MHCL_AP_T(3); break;
+            case 4: MHCL_AP_T(4); break;
+            default: MHCL_AP_W(5);
+        }
     }
+#undef MHCL_AP_W
 #undef MHCL_AP_T
 }
 
@@ -958,15 +1170,20 @@ void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const v
 #define MHCL_TP_T(N_) lite_tailpre_w_k<N_><<<blocks, 256, 0, s>>>( \
         T, C8, inv, (const uint4*)x, (const uint4*)du, a, p, rstd, alpha, H_pre, H_post, dH_res, dH_post, eo, kappa, \
         db, dalpha)
-    switch (c->n) {
-        case 2: MHCL_TP_T(2); break;
-        case 3: MHCL_TP_T(3); break;
-        case 4: MHCL_TP_T(4); break;
-        default:
-            lite_tailpre_k<5><<<group_grid(T, 16, c->sm_count), kActThreads, 0, s>>>(
-                T, C8, c->nfact, inv, (const uint4*)x, (const uint4*)du, a, p, rstd, alpha, H_pre, H_post, dH_res,
-                dH_post, eo, kappa, db, dalpha);
+#define MHCL_TP_W(N_) lite_tailpre_k<N_><<<group_grid(T, (N_ == 5) ? 16 : 32, c->sm_count), kActThreads, 0, s>>>( \
+        T, C8, c->nfact, inv, (const uint4*)x, (const uint4*)du, a, p, rstd, alpha, H_pre, H_post, dH_res, \
+        dH_post, eo, kappa, db, dalpha, c->table_dev)
+    if (c->table_dev) {
+        MHCL_DISPATCH_N(c->n, MHCL_TP_W(N_));
+    } else {
+        switch (c->n) {
+            case 2: MHCL_TP_T(2); break;
+            case 3: MHCL_TP_T(3); break;
+            case 4: MHCL_TP_T(4); break;
+            default: MHCL_TP_W(5);
+        }
     }
+#undef MHCL_TP_W
 #undef MHCL_TP_T
 }
 
@@ -991,6 +1208,39 @@ void launch_sk_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, int iters, con
     const float inv = 1.f / (float)(c->n * c->C);
     MHCL_DISPATCH_N(c->n, sk_act_bwd_k<N_><<<grid, 128, 0, s>>>(T, iters, inv, p, b, rstd, alpha, H_pre, H_post,
                                                                   dH_res, dH_pre, dH_post, eo, kappa, db, dalpha));
+}
+
+}  // namespace mhcl
+
+namespace mhcl {
+
+void launch_sk_act_premix(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,
+                          const float* ssq, float eps, const float* b, const float* alpha, float* H_res, float* H_pre,
+                          float* H_post, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s) {
+    c->launches += 1;
+    KernelTimer timer_(c, MHCLITE_KERNEL_ACT_PREMIX, s);
+    const int C8 = c->C / 8;
+    const float inv = 1.f / (float)(c->n * c->C);
+    const int grid = group_grid(T, kSkGroup, c->sm_count);
+    MHCL_DISPATCH_N(c->n, sk_act_premix_k<N_><<<grid, kActThreads, 0, s>>>(T, C8, iters, pp.Npad, pp.ksplit, inv, eps, qpart,
+                                                                          ssq, b, alpha, H_res, H_pre, H_post, p_saved, rstd,
+                                                                          (const uint4*)x, (uint4*)u));
+}
+
+void launch_sk_tailpre(const mhclite_ctx* c, int64_t T, int iters, const void* x, const void* du, const float* p,
+                       const float* b, const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
+                       const float* dH_res, const float* dH_post, float* e, int Npad, void* ehi, void* elo, int Kp,
+                       float* kappa, float* db, float* dalpha, cudaStream_t s) {
+    c->launches += 1;
+    KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_PRE, s);
+    const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
+    clear_e_tail(T, ehi, elo, Kp, s);
+    const int C8 = c->C / 8;
+    const float inv = 1.f / (float)(c->n * c->C);
+    const int grid = group_grid(T, kSkGroup, c->sm_count);
+    MHCL_DISPATCH_N(c->n, sk_tailpre_k<N_><<<grid, kActThreads, 0, s>>>(T, C8, iters, inv, (const uint4*)x, (const uint4*)du, p,
+                                                                       b, rstd, alpha, H_pre, H_post, dH_res, dH_post, eo,
+                                                                       kappa, db, dalpha));
 }
 
 }  // namespace mhcl

@@ -20,7 +20,9 @@ constexpr int kWarp = 32;
 
 struct mhclite_ctx {
     int n, C, device;
-    int nfact;                    // n!
+    int nfact;                    // residual weights per token: n!, or K with a subset of the permutations attached
+    const uint8_t* table_dev;     // caller-owned device table [K][n] of that subset (null: all n! permutations)
+    uint8_t table_host[120 * 5];  // validated host copy of the subset
     int sm_count;
     void* ws;
     size_t ws_bytes;
@@ -65,6 +67,8 @@ inline int balanced_warp_blocks(int64_t T, int64_t cap_blocks) {
 // Number of projection columns. kind 0: n!+2n (mHC-lite); kind 1: n*n+2n (SK path).
 inline int n_res_cols(int n, int kind) { return kind == 0 ? ipow_fact(n) : n * n; }
 inline int n_cols(int n, int kind) { return n_res_cols(n, kind) + 2 * n; }
+// Projection columns of a context: a subset of K permutations (paper Section 5) narrows the residual group to K.
+inline int ctx_cols(const mhclite_ctx* c, int kind) { return (kind == 0 ? c->nfact : c->n * c->n) + 2 * c->n; }
 
 // Brackets one kernel launch with the context's events when kernel timing is switched on.
 struct KernelTimer {
@@ -125,7 +129,7 @@ struct Workspace {
     size_t bytes;
     int Npad;
 };
-Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base);
+Workspace plan_workspace(int n, int C, int64_t T, int N, void* base);
 
 // Permutation tables in constant memory (perm_table.cu).
 struct PermTables {

@@ -76,6 +76,14 @@ void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const v
                          const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
                          const float* dH_res, const float* dH_post, float* dH_pre_ws, float* e, int Npad, void* ehi,
                          void* elo, int Kp, float* kappa, float* db, float* dalpha, cudaStream_t s);
+// the SK path's counterparts of the two fused kernels above
+void launch_sk_act_premix(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,
+                          const float* ssq, float eps, const float* b, const float* alpha, float* H_res, float* H_pre,
+                          float* H_post, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s);
+void launch_sk_tailpre(const mhclite_ctx* c, int64_t T, int iters, const void* x, const void* du, const float* p,
+                       const float* b, const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
+                       const float* dH_res, const float* dH_post, float* e, int Npad, void* ehi, void* elo, int Kp,
+                       float* kappa, float* db, float* dalpha, cudaStream_t s);
 void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,
                        const float* ssq, float eps, const float* b, const float* alpha, float* H_res, float* H_pre,
                        float* H_post, float* p_saved, float* rstd, cudaStream_t s);

@@ -24,9 +24,8 @@ int check_cuda(mhclite_ctx* ctx, cudaError_t e, const char* what) {
 
 static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
-Workspace plan_workspace(int n, int C, int64_t T, int kind, void* base) {
+Workspace plan_workspace(int n, int C, int64_t T, int N, void* base) {
     Workspace w;
-    const int N = n_cols(n, kind);
     w.Npad = round_up(N, 8);
     char* p = (char*)base;
     size_t off = 0;
@@ -87,10 +86,10 @@ using namespace mhcl;
 #define MHCL_LAUNCH_CHECK(ctx, what) do { int rc_ = check_cuda(ctx, cudaGetLastError(), what); if (rc_) return rc_; } while (0)
 
 static int need_workspace(mhclite_ctx* ctx, int64_t T, int kind, Workspace* w) {
-    const size_t need = mhclite_workspace_bytes(ctx->n, ctx->C, T, kind);
+    const size_t need = plan_workspace(ctx->n, ctx->C, T, ctx_cols(ctx, kind), nullptr).bytes;
     if (!ctx->ws || ctx->ws_bytes < need)
         return fail(ctx, MHCLITE_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu attached", need, ctx->ws ? ctx->ws_bytes : (size_t)0);
-    *w = plan_workspace(ctx->n, ctx->C, T, kind, ctx->ws);
+    *w = plan_workspace(ctx->n, ctx->C, T, ctx_cols(ctx, kind), ctx->ws);
     // status words of the workspace (status + four words describing the first report), at its very end,
     // cleared when first used
     w->status = (int*)((char*)ctx->ws + ((ctx->ws_bytes - 32) & ~(size_t)255));
@@ -196,7 +195,7 @@ int mhclite_create(mhclite_ctx** out, int n, int C, int device) {
     if (cudaGetDeviceCount(&count) != cudaSuccess || device >= count) return MHCLITE_ERR_CUDA;
     mhclite_ctx* ctx = new (std::nothrow) mhclite_ctx();
     if (!ctx) return MHCLITE_ERR_CUDA;
-    ctx->n = n; ctx->C = C; ctx->device = device; ctx->nfact = ipow_fact(n);
+    ctx->n = n; ctx->C = C; ctx->device = device; ctx->nfact = ipow_fact(n); ctx->table_dev = nullptr;
     ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->err[0] = 0; ctx->launches = 0; ctx->timing = false; ctx->status_word = nullptr;
     for (int k = 0; k < MHCLITE_KERNEL_COUNT; ++k) { ctx->ev[k][0] = ctx->ev[k][1] = nullptr; ctx->ev_recorded[k] = false; }
     ctx->copy_in = ctx->copy_out = nullptr; ctx->ev_fork = ctx->ev_join = nullptr;
@@ -246,7 +245,42 @@ int mhclite_perm_table_device(mhclite_ctx* ctx, uint8_t* sigma_host) {
 
 size_t mhclite_workspace_bytes(int n, int C, int64_t T, int kind) {
     if (n < 2 || n > kMaxN || C <= 0 || T < 0 || kind < 0 || kind > 1) return 0;
-    return plan_workspace(n, C, T, kind, nullptr).bytes;
+    return plan_workspace(n, C, T, n_cols(n, kind), nullptr).bytes;
+}
+
+size_t mhclite_workspace_bytes_subset(int n, int C, int64_t T, int K) {
+    if (n < 2 || n > kMaxN || C <= 0 || T < 0 || K < 1 || K > ipow_fact(n)) return 0;
+    return plan_workspace(n, C, T, K + 2 * n, nullptr).bytes;
+}
+
+int mhclite_set_perm_subset(mhclite_ctx* ctx, int K, const uint8_t* table) {
+    MHCL_REQUIRE_CTX(ctx);
+    if (K == 0 || !table) {                            // back to all n! permutations
+        ctx->nfact = ipow_fact(ctx->n);
+        ctx->table_dev = nullptr;
+        return MHCLITE_OK;
+    }
+    const int n = ctx->n;
+    if (K < 1 || K > ipow_fact(n) || K > kMaxFact) return fail(ctx, MHCLITE_ERR_BAD_ARG, "K must be in [1, n!]");
+    MHCL_DEVICE(ctx);
+    uint8_t h[kMaxFact * kMaxN];
+    int rc = check_cuda(ctx, cudaMemcpy(h, table, (size_t)K * n, cudaMemcpyDeviceToHost), "read permutation subset");
+    if (rc) return rc;
+    for (int k = 0; k < K; ++k) {
+        unsigned seen = 0;
+        for (int i = 0; i < n; ++i) {
+            const int v = h[k * n + i];
+            if (v >= n || (seen >> v & 1u)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "row %d of the table is not a permutation of 0..%d", k, n - 1);
+            seen |= 1u << v;
+        }
+        for (int k2 = 0; k2 < k; ++k2)
+            if (memcmp(h + k * n, h + k2 * n, (size_t)n) == 0)
+                return fail(ctx, MHCLITE_ERR_BAD_ARG, "row %d of the table repeats row %d", k, k2);
+    }
+    memcpy(ctx->table_host, h, (size_t)K * n);
+    ctx->table_dev = table;
+    ctx->nfact = K;
+    return MHCLITE_OK;
 }
 
 int mhclite_set_workspace(mhclite_ctx* ctx, void* workspace, size_t bytes) {
@@ -273,7 +307,7 @@ int mhclite_coeffs_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     if (rc) return rc;
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
-    const int N = n_cols(ctx->n, 0);
+    const int N = ctx_cols(ctx, 0);
     const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
     rc = proj_forward(ctx, T, N, w, pp, x, W, gain, s);
     if (rc) return rc;
@@ -318,7 +352,7 @@ int mhclite_pre_fwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, co
     if (rc) return rc;
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
-    const int N = n_cols(ctx->n, 0);
+    const int N = ctx_cols(ctx, 0);
     const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
     rc = proj_forward(ctx, T, N, w, pp, x, W, gain, s);
     if (rc) return rc;
@@ -383,7 +417,7 @@ int mhclite_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     if (rc) return rc;
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
-    const int N = n_cols(ctx->n, 0);
+    const int N = ctx_cols(ctx, 0);
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
     bool wf_packed = false;
     rc = prep_param_grads(ctx, N, tp, w, W, gain, db, dalpha, accumulate_params, s, &wf_packed);
@@ -412,7 +446,7 @@ int mhclite_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, c
     if (rc) return rc;
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
-    const int N = n_cols(ctx->n, 0);
+    const int N = ctx_cols(ctx, 0);
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
     bool wf_packed = false;
     rc = prep_param_grads(ctx, N, tp, w, W, gain, db, dalpha, accumulate_params, s, &wf_packed);
@@ -439,12 +473,36 @@ int mhc_sk20_coeffs_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
     if (rc) return rc;
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
-    const int N = n_cols(ctx->n, 1);
+    const int N = ctx_cols(ctx, 1);
     const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
     rc = proj_forward(ctx, T, N, w, pp, x, W_sk, gain, s);
     if (rc) return rc;
     launch_sk_act_fwd(ctx, T, iters, pp, w.qpart, w.ssq, eps, b_sk, alpha, H_res, H_pre, H_post, p_saved, rstd, s);
     MHCL_LAUNCH_CHECK(ctx, "sk_act_fwd");
+    return MHCLITE_OK;
+}
+
+int mhc_sk20_pre_fwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W_sk, const float* b_sk,
+                           const float* alpha, const float* gain, float eps, int iters, float* H_res, float* H_pre,
+                           float* H_post, float* p_saved, float* rstd, mhclite_bf16* u, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (iters < 1 || iters > 64) return fail(ctx, MHCLITE_ERR_BAD_ARG, "iters must be in [1,64]");
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, W_sk); MHCL_PTR(ctx, b_sk); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain);
+    MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd);
+    MHCL_PTR(ctx, u);
+    if (!(eps >= 0.f)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "eps must be >= 0");
+    Workspace w;
+    int rc = need_workspace(ctx, T, 1, &w);
+    if (rc) return rc;
+    MHCL_DEVICE(ctx);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int N = ctx_cols(ctx, 1);
+    const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
+    rc = proj_forward(ctx, T, N, w, pp, x, W_sk, gain, s);
+    if (rc) return rc;
+    launch_sk_act_premix(ctx, T, iters, pp, w.qpart, w.ssq, eps, b_sk, alpha, H_res, H_pre, H_post, p_saved, rstd, x, u, s);
+    MHCL_LAUNCH_CHECK(ctx, "sk_act_premix");
     return MHCLITE_OK;
 }
 
@@ -466,7 +524,7 @@ int mhc_sk20_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
     if (rc) return rc;
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
-    const int N = n_cols(ctx->n, 1);
+    const int N = ctx_cols(ctx, 1);
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
     bool wf_packed = false;
     rc = prep_param_grads(ctx, N, tp, w, W_sk, gain, db, dalpha, accumulate_params, s, &wf_packed);
@@ -497,16 +555,15 @@ int mhc_sk20_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, 
     if (rc) return rc;
     MHCL_DEVICE(ctx);
     cudaStream_t s = (cudaStream_t)stream;
-    const int N = n_cols(ctx->n, 1);
+    const int N = ctx_cols(ctx, 1);
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
     bool wf_packed = false;
     rc = prep_param_grads(ctx, N, tp, w, W_sk, gain, db, dalpha, accumulate_params, s, &wf_packed);
     if (rc) return rc;
-    launch_premix_bwd(ctx, T, x, H_pre, du, w.dH_pre, nullptr, 0, s);
-    MHCL_LAUNCH_CHECK(ctx, "premix_bwd");
-    launch_sk_act_bwd(ctx, T, w.Npad, iters, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, w.dH_pre, dH_post,
-                      tp.supported ? nullptr : w.e, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db, dalpha, s);
-    MHCL_LAUNCH_CHECK(ctx, "sk_act_bwd");
+    launch_sk_tailpre(ctx, T, iters, x, du, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, dH_post,
+                      tp.supported ? nullptr : w.e, w.Npad, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db,
+                      dalpha, s);
+    MHCL_LAUNCH_CHECK(ctx, "sk_tailpre");
     return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W_sk, gain, wf_packed, dx, 0, dW, dgain, accumulate_params, s);
 }
 
@@ -553,7 +610,7 @@ StepStaging plan_step(int n, int C, int64_t T, void* base) {
     char* p = (char*)base;
     size_t off = 0;
     const size_t big = (size_t)T * n * C * sizeof(mhclite_bf16), small = (size_t)T * C * sizeof(mhclite_bf16);
-    const int nf = ipow_fact(n), N = n_cols(n, 0);
+    const int nf = ipow_fact(n), N = n_cols(n, 0);        // sized for all n! permutations: a subset needs less
     auto take = [&](size_t b) { void* q = p + off; off += align256(b); return q; };
     s.x = (mhclite_bf16*)take(big); s.y = (mhclite_bf16*)take(small); s.g = (mhclite_bf16*)take(big);
     s.du = (mhclite_bf16*)take(small); s.u = (mhclite_bf16*)take(small); s.x_next = (mhclite_bf16*)take(big);
@@ -608,7 +665,7 @@ int mhclite_step_host(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x_host, c
     int64_t chunk = round_up64((T + MHCLITE_STEP_CHUNKS - 1) / MHCLITE_STEP_CHUNKS, 128);
     if (chunk < 256) chunk = 256;
     const int nchunks = (int)((T + chunk - 1) / chunk);
-    const int n = ctx->n, C = ctx->C, nf = ctx->nfact, N = n_cols(n, 0);
+    const int n = ctx->n, C = ctx->C, nf = ctx->nfact, N = ctx_cols(ctx, 0);
 #define MHCL_CUDA(call, what) if ((rc = check_cuda(ctx, call, what))) return rc
     MHCL_CUDA(cudaEventRecord(ctx->ev_fork, st), "event record");
     MHCL_CUDA(cudaStreamWaitEvent(ctx->copy_in, ctx->ev_fork, 0), "stream wait");

@@ -61,7 +61,7 @@ int mhclite_coeffs_bwd_static(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x
         if (!p || ((uintptr_t)p & 15)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "null or misaligned pointer");
     if (ctx->device >= kMaxDevices) return fail(ctx, MHCLITE_ERR_BAD_ARG, "device index %d not supported", ctx->device);
     // scratch of this call: e [T][Npad], kappa [T], G [nC][Npad] (fp32), each 256-byte aligned
-    const int N = n_cols(ctx->n, 0), Npad = round_up(N, 8), nC = ctx->n * ctx->C;
+    const int N = ctx_cols(ctx, 0), Npad = round_up(N, 8), nC = ctx->n * ctx->C;
     auto up256 = [](size_t v) { return (v + 255) & ~(size_t)255; };
     const size_t o_kappa = up256((size_t)T * Npad * 4), o_G = o_kappa + up256((size_t)T * 4);
     const size_t need = o_G + up256((size_t)nC * Npad * 4);

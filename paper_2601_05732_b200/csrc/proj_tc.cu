@@ -136,13 +136,15 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
             for (int m = 0; m < 2; ++m) {
                 if (m < mt) {
                     const unsigned char* xr = smem + s * stage_bytes + m * kTcXBytes + row * 128;
+                    float part = 0.f;                       // per 64-element chunk, then added: short chains round less
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         float f[8];
                         unpack8(*reinterpret_cast<const uint4*>(xr + ((c ^ (row & 7)) << 4)), f);
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) sqs[m] = fmaf(f[e], f[e], sqs[m]);
+                        for (int e = 0; e < 8; ++e) part = fmaf(f[e], f[e], part);
                     }
+                    sqs[m] += part;
                 }
             }
             __syncwarp();

@@ -51,7 +51,10 @@ class LayerBuffers:
 
 def pre_fwd(ctx: MhcLite, P: LayerParams, B: LayerBuffers, x, eps=1e-6, fused=True, iters=20):
     """Mappings + stream pre-mix: everything before the sublayer. Result: B.u (and the coefficients)."""
-    if B.kind == "sk":
+    if B.kind == "sk" and fused:
+        ctx.sk20_pre_fwd_fused(x, P.W, P.b, P.alpha, P.gain, eps, iters, B.H_res, B.H_pre, B.H_post, B.p_saved, B.rstd,
+                               B.u)
+    elif B.kind == "sk":
         ctx.sk20_coeffs_fwd(x, P.W, P.b, P.alpha, P.gain, eps, iters, B.H_res, B.H_pre, B.H_post, B.p_saved, B.rstd)
         ctx.premix_fwd(x, B.H_pre, B.u)
     elif fused:

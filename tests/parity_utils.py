@@ -5,10 +5,11 @@ Tolerances (they follow the arithmetic: bf16 storage rounds to 2^-9 relative, fp
 n*C <= 2^15 terms leaves ~1e-6 relative):
   bf16 tensors : |gpu - ref| <= 2e-2 |ref| + 1e-3 rms(ref)          for every element
   fp32 mappings: |gpu - ref| <= 1e-5 max(|ref|, rms(ref))           (H_res, H_pre, H_post, a, rstd)
-  saved projection p = x' W: 1e-4 max(|ref|, rms(ref)) -- W' enters the tensor cores as a bf16 pair
-                hi + lo (up to 2^-18 relative error per weight) and the tensor cores' fp32 accumulation
-                over n*C/8 steps adds a few 1e-5 of rms(p) at n*C = 7680; alpha scales this down by 100x
-                before it reaches the mappings, which are checked at 1e-5
+  saved projection p = x' W: p_tolerance(nC) max(|ref|, rms(ref)) = 2^-16 + (nC / 16) 2^-24 -- W' enters the
+                tensor cores as a bf16 pair hi + lo (16 mantissa bits: 2^-17 relative per weight) and the
+                tensor cores add each 16-deep k-step to the fp32 accumulator with up to one unit in the last
+                place lost (nC / 16 steps).  Measured: 1.0e-5 at nC = 4096, 3.8e-5 at nC = 7680, 4.9e-5 at
+                nC = 16384.  alpha scales this down by 100x before it reaches the mappings, checked at 1e-5
   fp32 parameter gradients: |gpu - ref| <= 1e-3 max(|ref|, rms(ref)) (the binding tolerance is 2e-2)
 """
 import numpy as np
@@ -20,6 +21,11 @@ from paper_2601_05732_b200.binding import MhcLite
 from paper_2601_05732_b200 import layer as L
 
 DEV = "cuda:0"
+
+
+def p_tolerance(nC):
+    """Relative tolerance of the saved projection for a contraction over nC terms (see the module docstring)."""
+    return 2.0 ** -16 + (nC / 16) * 2.0 ** -24
 
 
 def rms(a):
@@ -78,10 +84,13 @@ def host(t):
 class GpuLayer:
     """Uploads one layer's host inputs and runs the library's call sequence on them."""
 
-    def __init__(self, inp, eps=1e-6, kind="lite", iters=20):
+    def __init__(self, inp, eps=1e-6, kind="lite", iters=20, table=None):
         self.inp, self.eps, self.kind, self.iters = inp, eps, kind, iters
         n, C, T = inp["n"], inp["C"], inp["T"]
         self.ctx = MhcLite(n, C, 0)
+        if table is not None:                       # a subset of the permutations (paper Section 5)
+            self.table = torch.from_numpy(np.ascontiguousarray(table, dtype=np.uint8)).to(DEV)
+            self.ctx.set_perm_subset(self.table)
         self.P = L.LayerParams(inp["W"], inp["b"], inp["alpha"], inp["gain"], DEV)
         self.B = L.LayerBuffers(self.ctx, T, kind)
         self.x = L.to_device_bf16(inp["x"], DEV); self.y = L.to_device_bf16(inp["y"], DEV)
@@ -105,20 +114,21 @@ def oracle_inputs(inp):
                 alpha=inp["alpha"].astype(np.float64), gain=inp["gain"].astype(np.float64))
 
 
-def oracle_fwd(inp, eps=1e-6, kind="lite", iters=20):
+def oracle_fwd(inp, eps=1e-6, kind="lite", iters=20, table=None):
     o = oracle_inputs(inp)
-    return O.layer_fwd(o["x"], o["y"], o["W"], o["b"], o["alpha"], o["gain"], eps, kind=kind, iters=iters)
+    return O.layer_fwd(o["x"], o["y"], o["W"], o["b"], o["alpha"], o["gain"], eps, kind=kind, iters=iters, table=table)
 
 
-def oracle_bwd(inp, eps=1e-6, kind="lite", iters=20):
+def oracle_bwd(inp, eps=1e-6, kind="lite", iters=20, table=None):
     o = oracle_inputs(inp)
-    return O.layer_bwd(o["x"], o["y"], o["W"], o["b"], o["alpha"], o["gain"], eps, o["g"], o["du"], kind=kind, iters=iters)
+    return O.layer_bwd(o["x"], o["y"], o["W"], o["b"], o["alpha"], o["gain"], eps, o["g"], o["du"], kind=kind, iters=iters,
+                       table=table)
 
 
 def compare_forward(G, ref, coeff_rel=1e-5):
     B = G.B
     check_f32("rstd", host(B.rstd), ref["rstd"], coeff_rel)
-    check_f32("p_saved", host(B.p_saved), ref["p"], max(coeff_rel, 1e-4))
+    check_f32("p_saved", host(B.p_saved), ref["p"], max(coeff_rel, p_tolerance(G.ctx.n * G.ctx.C)))
     if G.kind == "lite":
         check_f32("a_saved", host(B.a_saved), ref["a"], coeff_rel)
     check_f32("H_res", host(B.H_res), ref["H_res"], coeff_rel)

@@ -64,6 +64,9 @@ def test_workspace_bytes():
     assert wb(4, 1024, 16384) % 256 == 0
     assert wb(1, 1024, 10) == 0 and wb(6, 1024, 10) == 0 and wb(4, 1024, -1) == 0   # rejected -> 0
     assert wb(4, 1024, 16384) < 64 << 20
+    ws = binding.load().mhclite_workspace_bytes_subset
+    assert 0 < ws(5, 1536, 4096, 8) < ws(5, 1536, 4096, 64) <= wb(5, 1536, 4096)      # fewer columns, less scratch
+    assert ws(5, 1536, 4096, 0) == 0 and ws(5, 1536, 4096, 121) == 0 and ws(4, 64, 10, 25) == 0
 
 
 def test_status_strings_and_null_context():

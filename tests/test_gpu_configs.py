@@ -16,8 +16,7 @@ from oracle import mhclite_oracle as O
 from paper_2601_05732_b200 import synth
 from paper_2601_05732_b200 import layer as L
 from paper_2601_05732_b200.binding import MhcLite
-from parity_utils import (DEV, GpuLayer, check_bf16, check_f32, dxhat_allowance, dxhat_allowance_f, host,
-                          oracle_inputs, rms)
+from parity_utils import DEV, GpuLayer, check_bf16, check_f32, host, oracle_inputs, p_tolerance, rms
 
 pytestmark = pytest.mark.gpu
 NS = 48   # sampled tokens
@@ -66,7 +65,7 @@ def _run_and_check(wl, kind="lite", param_grads=True, T=None, inp=None):
     ti = torch.from_numpy(idx).to(DEV)
     pick = lambda t: host(t.index_select(0, ti))
     check_f32("rstd", pick(B.rstd), fw["rstd"])
-    check_f32("p_saved", pick(B.p_saved), fw["p"], 1e-4)
+    check_f32("p_saved", pick(B.p_saved), fw["p"], p_tolerance(wl.n * wl.C))
     check_f32("H_res", pick(B.H_res), fw["H_res"])
     check_f32("H_pre", pick(B.H_pre), fw["H_pre"])
     check_f32("H_post", pick(B.H_post), fw["H_post"])
@@ -80,7 +79,9 @@ def _run_and_check(wl, kind="lite", param_grads=True, T=None, inp=None):
     check_bf16("dy", pick(B.dy), bw["dy"])
     check_f32("dH_res", pick(B.dH_res), bw["dH_res"], 2e-5)
     check_f32("dH_post", pick(B.dH_post), bw["dH_post"], 2e-5)
-    check_bf16("dx", pick(B.dx), bw["dx"], extra=dxhat_allowance(sub, bw["dz"]))
+    # the plain bf16 tolerance: at the workloads' distributions the bf16 operands of the projection backward's
+    # dx term stay far inside it (no allowance, unlike the stress cases of test_gpu_parity.py)
+    check_bf16("dx", pick(B.dx), bw["dx"])
     if param_grads:
         ref = _oracle_param_grads(inp, kind)
         check_f32("dW", host(B.dW), ref["dW"], 1e-3)
@@ -197,8 +198,7 @@ def test_cfg3_stack_of_24_layers():
         check_bf16(f"x_next[{l}]", pick(Bs[l].x_next), fw["x_next"])
         bw = O.layer_bwd(xl, yl, p["W"], p["b"], p["alpha"], p["gain"], eps, gl, dul)
         check_bf16(f"dy[{l}]", pick(Bs[l].dy), bw["dy"])
-        check_bf16(f"dx[{l}]", pick(Bs[l].dx), bw["dx"],
-                   extra=dxhat_allowance_f(xl, p["W"], p["alpha"], p["gain"], bw["dz"], eps))
+        check_bf16(f"dx[{l}]", pick(Bs[l].dx), bw["dx"])
     # parameter gradients of the first and the last layer over ALL tokens (the oracle is fed the tensors the
     # GPU layer was fed, in chunks)
     for l in (0, Ld - 1):

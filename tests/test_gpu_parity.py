@@ -212,7 +212,7 @@ def test_sk_gap_with_the_papers_initialisation_bias():
     GL = GpuLayer(lite); GL.forward()
     compare_forward(GL, oracle_fwd(lite), coeff_rel=2e-4)
     GL.ctx.ds_gap(GL.B.H_res, l1, cd); torch.cuda.synchronize()
-    assert float(l1.max()) < 4e-6 and float(cd.max()) < 1e-6
+    assert float(cd.max()) < 1e-6 and float(l1.max()) < 2 * n * 1e-6       # 2n row / column sums, each within 1e-6
 
 
 def test_kernel_timing_and_device_status():
