@@ -43,6 +43,8 @@ SIGNATURES = {
     "mhclite_premix_fwd": (_i, [_p, _i64, _p, _p, _p, _p]),
     "mhclite_postres_fwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p]),
     "mhclite_pre_fwd_fused": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p]),
+    "mhclite_postres_fwd_next_proj": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p, _p, _p]),
+    "mhclite_pre_fwd_resume": (_i, [_p, _i64, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p]),
     "mhclite_postres_bwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p, _p, _p, _p, _i, _p]),
     "mhclite_premix_bwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _i, _p]),
     "mhclite_coeffs_bwd": (_i, [_p, _i64, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p, _p, _i,
@@ -210,6 +212,21 @@ class MhcLite:
             self._ptr(gain, f), float(eps), self._ptr(H_res, f), self._ptr(H_pre, f), self._ptr(H_post, f),
             self._ptr(a_saved, f), self._ptr(p_saved, f), self._ptr(rstd, f), self._ptr(u, h), self._stream()),
             "mhclite_pre_fwd_fused")
+
+    def postres_fwd_next_proj(self, x, y, H_res, H_post, x_next, W_next, gain_next):
+        f, h = self._torch.float32, self._torch.bfloat16
+        self.ensure_workspace(x.shape[0], 0)
+        self._check(self.lib.mhclite_postres_fwd_next_proj(
+            self._h, x.shape[0], self._ptr(x, h), self._ptr(y, h), self._ptr(H_res, f), self._ptr(H_post, f),
+            self._ptr(x_next, h), self._ptr(W_next, f), self._ptr(gain_next, f), self._stream()),
+            "mhclite_postres_fwd_next_proj")
+
+    def pre_fwd_resume(self, x, b, alpha, eps, H_res, H_pre, H_post, a_saved, p_saved, rstd, u):
+        f, h = self._torch.float32, self._torch.bfloat16
+        self._check(self.lib.mhclite_pre_fwd_resume(
+            self._h, x.shape[0], self._ptr(x, h), self._ptr(b, f), self._ptr(alpha, f), float(eps),
+            self._ptr(H_res, f), self._ptr(H_pre, f), self._ptr(H_post, f), self._ptr(a_saved, f), self._ptr(p_saved, f),
+            self._ptr(rstd, f), self._ptr(u, h), self._stream()), "mhclite_pre_fwd_resume")
 
     # -- backward --------------------------------------------------------------------------------
     def postres_bwd(self, x, y, H_res, H_post, g, dy, dH_res, dH_post, dx=None, accumulate_dx=False):

@@ -34,6 +34,10 @@ struct mhclite_ctx {
     // mhclite_step_host: copy-in and copy-out streams and the events that chain its token chunks (made on first use)
     cudaStream_t copy_in, copy_out;
     cudaEvent_t ev_fork, ev_join, ev_in[MHCLITE_STEP_CHUNKS], ev_cmp[MHCLITE_STEP_CHUNKS];
+    // projection partials left in the workspace by mhclite_postres_fwd_next_proj for mhclite_pre_fwd_resume
+    int64_t pending_T;            // tokens they cover (-1: none)
+    const void* pending_x;        // the x_next they were computed from
+    int pending_ksplit;           // K slices they come in
     char err[256];
 };
 
@@ -129,7 +133,8 @@ struct Workspace {
     size_t bytes;
     int Npad;
 };
-Workspace plan_workspace(int n, int C, int64_t T, int N, void* base);
+// (sm_count: SMs of the device the plan is for; the B200's 148 where no context is at hand)
+Workspace plan_workspace(int n, int C, int64_t T, int N, void* base, int sm_count = 148);
 
 // Permutation tables in constant memory (perm_table.cu).
 struct PermTables {

@@ -60,6 +60,12 @@ void launch_pack_wt(const mhclite_ctx* c, const ProjPlan& p, int N, const float*
 bool launch_proj_fwd_tc(const mhclite_ctx* c, int64_t T, int N, const ProjPlan& p, const void* x, const void* Wt,
                         float* qpart, float* ssq, int* status, cudaStream_t s);
 
+// postres_proj.cu : the merge of one layer fused with the RMSNorm statistics and projection of the next
+bool postres_proj_supported(int n, int C, int N);
+bool launch_postres_proj(const mhclite_ctx* c, int64_t T, int N, const ProjPlan& pp, const void* x, const void* y,
+                         const float* H_res, const float* H_post, void* x_next, const void* Wt, float* qpart, float* ssq,
+                         int* status, cudaStream_t s);
+
 // act_kernels.cu : per-token activations, H_res assembly and their gradients
 void launch_lite_act_fwd(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, const float* qpart, const float* ssq,
                          float eps, const float* b, const float* alpha, float* H_res, float* H_pre, float* H_post,

@@ -24,7 +24,7 @@ int check_cuda(mhclite_ctx* ctx, cudaError_t e, const char* what) {
 
 static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
-Workspace plan_workspace(int n, int C, int64_t T, int N, void* base) {
+Workspace plan_workspace(int n, int C, int64_t T, int N, void* base, int sm_count) {
     Workspace w;
     w.Npad = round_up(N, 8);
     char* p = (char*)base;
@@ -33,11 +33,11 @@ Workspace plan_workspace(int n, int C, int64_t T, int N, void* base) {
     w.kappa = (float*)(p + off); off += align256((size_t)T * sizeof(float));
     w.G = (float*)(p + off);     off += align256((size_t)n * C * w.Npad * sizeof(float));
     w.dH_pre = (float*)(p + off); off += align256((size_t)T * n * sizeof(float));
-    const ProjPlan pp = plan_proj(n, C, T, N, 148);          // sizes do not depend on the SM count
+    const ProjPlan pp = plan_proj(n, C, T, N, sm_count);     // sizes do not depend on the SM count
     w.Wp = p + off;              off += align256((size_t)pp.ksteps * pp.NT * 32 * 16);
     w.qpart = (float*)(p + off); off += align256((size_t)kMaxKSplit * T * pp.Npad * sizeof(float));
     w.ssq = (float*)(p + off);   off += align256((size_t)kMaxKSplit * T * sizeof(float));
-    const TailPlan tp = plan_tail(n, C, T, N, 148);
+    const TailPlan tp = plan_tail(n, C, T, N, sm_count);      // the token ranges (G partials) do
     const size_t erows = (size_t)round_up64(T, kEGranule);
     w.ehi = p + off;             off += align256(erows * tp.Kp * 2);
     w.elo = p + off;             off += align256(erows * tp.Kp * 2);
@@ -86,10 +86,10 @@ using namespace mhcl;
 #define MHCL_LAUNCH_CHECK(ctx, what) do { int rc_ = check_cuda(ctx, cudaGetLastError(), what); if (rc_) return rc_; } while (0)
 
 static int need_workspace(mhclite_ctx* ctx, int64_t T, int kind, Workspace* w) {
-    const size_t need = plan_workspace(ctx->n, ctx->C, T, ctx_cols(ctx, kind), nullptr).bytes;
+    const size_t need = plan_workspace(ctx->n, ctx->C, T, ctx_cols(ctx, kind), nullptr, ctx->sm_count).bytes;
     if (!ctx->ws || ctx->ws_bytes < need)
         return fail(ctx, MHCLITE_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu attached", need, ctx->ws ? ctx->ws_bytes : (size_t)0);
-    *w = plan_workspace(ctx->n, ctx->C, T, ctx_cols(ctx, kind), ctx->ws);
+    *w = plan_workspace(ctx->n, ctx->C, T, ctx_cols(ctx, kind), ctx->ws, ctx->sm_count);
     // status words of the workspace (status + four words describing the first report), at its very end,
     // cleared when first used
     w->status = (int*)((char*)ctx->ws + ((ctx->ws_bytes - 32) & ~(size_t)255));
@@ -196,6 +196,7 @@ int mhclite_create(mhclite_ctx** out, int n, int C, int device) {
     mhclite_ctx* ctx = new (std::nothrow) mhclite_ctx();
     if (!ctx) return MHCLITE_ERR_CUDA;
     ctx->n = n; ctx->C = C; ctx->device = device; ctx->nfact = ipow_fact(n); ctx->table_dev = nullptr;
+    ctx->pending_T = -1; ctx->pending_x = nullptr;
     ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->err[0] = 0; ctx->launches = 0; ctx->timing = false; ctx->status_word = nullptr;
     for (int k = 0; k < MHCLITE_KERNEL_COUNT; ++k) { ctx->ev[k][0] = ctx->ev[k][1] = nullptr; ctx->ev_recorded[k] = false; }
     ctx->copy_in = ctx->copy_out = nullptr; ctx->ev_fork = ctx->ev_join = nullptr;
@@ -356,6 +357,75 @@ int mhclite_pre_fwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, co
     const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
     rc = proj_forward(ctx, T, N, w, pp, x, W, gain, s);
     if (rc) return rc;
+    launch_lite_act_premix(ctx, T, pp, w.qpart, w.ssq, eps, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, x, u, s);
+    MHCL_LAUNCH_CHECK(ctx, "lite_act_premix");
+    return MHCLITE_OK;
+}
+
+// One K slice covering all of n*C: the plan of projection partials that a single kernel produced per token tile.
+static ProjPlan whole_k_plan(const mhclite_ctx* ctx, int64_t T, int N) {
+    ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
+    pp.ksplit = 1;
+    pp.chunks_per_split = pp.nchunks;
+    return pp;
+}
+
+int mhclite_postres_fwd_next_proj(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const mhclite_bf16* y,
+                                  const float* H_res, const float* H_post, mhclite_bf16* x_next, const float* W_next,
+                                  const float* gain_next, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    ctx->pending_T = -1;
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, y); MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, x_next);
+    MHCL_PTR(ctx, W_next); MHCL_PTR(ctx, gain_next);
+    if ((const void*)x_next == (const void*)x) return fail(ctx, MHCLITE_ERR_BAD_ARG, "x_next must not alias x");
+    Workspace w;
+    int rc = need_workspace(ctx, T, 0, &w);
+    if (rc) return rc;
+    MHCL_DEVICE(ctx);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int N = ctx_cols(ctx, 0);
+    if (postres_proj_supported(ctx->n, ctx->C, N)) {
+        const ProjPlan pp = whole_k_plan(ctx, T, N);
+        launch_pack_wt(ctx, pp, N, W_next, gain_next, w.Wt, s);
+        MHCL_LAUNCH_CHECK(ctx, "pack_wt");
+        if (launch_postres_proj(ctx, T, N, pp, x, y, H_res, H_post, x_next, w.Wt, w.qpart, w.ssq, w.status, s)) {
+            MHCL_LAUNCH_CHECK(ctx, "postres_proj");
+            ctx->pending_T = T; ctx->pending_x = x_next; ctx->pending_ksplit = 1;
+            return MHCLITE_OK;
+        }
+    }
+    // shapes the fused kernel does not take: the merge, then the projection of the next layer as usual
+    launch_postres_fwd(ctx, T, x, y, H_res, H_post, x_next, s);
+    MHCL_LAUNCH_CHECK(ctx, "postres_fwd");
+    const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
+    rc = proj_forward(ctx, T, N, w, pp, x_next, W_next, gain_next, s);
+    if (rc) return rc;
+    ctx->pending_T = T; ctx->pending_x = x_next; ctx->pending_ksplit = pp.ksplit;
+    return MHCLITE_OK;
+}
+
+int mhclite_pre_fwd_resume(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* b, const float* alpha,
+                           float eps, float* H_res, float* H_pre, float* H_post, float* a_saved, float* p_saved,
+                           float* rstd, mhclite_bf16* u, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (T == 0) return MHCLITE_OK;
+    MHCL_PTR(ctx, x); MHCL_PTR(ctx, b); MHCL_PTR(ctx, alpha);
+    MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, a_saved);
+    MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd); MHCL_PTR(ctx, u);
+    if (!(eps >= 0.f)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "eps must be >= 0");
+    if (ctx->pending_T != T || ctx->pending_x != (const void*)x)
+        return fail(ctx, MHCLITE_ERR_BAD_ARG, "no projection partials of this x are pending: call "
+                                              "mhclite_postres_fwd_next_proj(..., x_next = x, ...) on this context first");
+    Workspace w;
+    int rc = need_workspace(ctx, T, 0, &w);
+    if (rc) return rc;
+    MHCL_DEVICE(ctx);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int N = ctx_cols(ctx, 0);
+    ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
+    if (ctx->pending_ksplit == 1) pp = whole_k_plan(ctx, T, N);
+    ctx->pending_T = -1;
     launch_lite_act_premix(ctx, T, pp, w.qpart, w.ssq, eps, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, x, u, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_act_premix");
     return MHCLITE_OK;

@@ -35,6 +35,7 @@ constexpr int kFEpiWarps = 8;
 constexpr int kFThreads = 96 + 32 * kFEpiWarps; // operand producer, MMA issuer, data producer, epilogue
 constexpr int kFMaxRing = 3;
 constexpr int kFSlots = 5;                      // data slots: one per lane quadrant plus one that goes round
+constexpr int kFMaxSplits = 64;                 // most token ranges per slice (bounds the G partials)
 
 struct FCtl {
     uint64_t w_full, e_full[2], e_empty[2], elo_full, elo_empty, d_full[4][2], g_done[4][2], q_done[4],
@@ -433,10 +434,18 @@ void plan_tail_ftc(int n, int C, int64_t T, int sm_count, TailPlan* p) {
     p->ftc = p->supported && (C % kFCs) == 0 && na * 2 * p->Kp + 2 * n * 32 <= 512 && ftc_smem_bytes(n, p->Kp, 1) <= 227 * 1024;
     p->f_slices = C / kFCs;
     const int64_t ntiles = (T + kFTok - 1) / kFTok;
-    int64_t splits = p->f_slices > 0 ? sm_count / p->f_slices : 1;
-    if (splits > ntiles) splits = ntiles;
-    if (splits < 1) splits = 1;
-    p->f_splits = (int)splits;
+    // Token ranges per slice.  One CTA fits an SM, so slices x ranges CTAs run in ceil(slices * ranges / SMs)
+    // rounds of ceil(ntiles / ranges) tiles each (plus about two tiles' worth of start-up and G write-out per
+    // CTA): take the count with the shortest total.  Several rounds of short CTAs beat one round that leaves SMs
+    // idle (64 slices: 2 ranges use 128 of 148 SMs, 16 ranges run 6.9 rounds' worth of work in 7).
+    int64_t best = 1, best_cost = INT64_MAX;
+    const int64_t rmax = ntiles < kFMaxSplits ? ntiles : kFMaxSplits;
+    for (int64_t r = 1; r <= rmax && p->f_slices > 0; ++r) {
+        const int64_t rounds = (p->f_slices * r + sm_count - 1) / sm_count;
+        const int64_t cost = rounds * ((ntiles + r - 1) / r + 2);
+        if (cost < best_cost) { best_cost = cost; best = r; }
+    }
+    p->f_splits = (int)best;
     int ring = (512 - na * 2 * p->Kp) / (n * 32);
     p->f_ring = ring > kFMaxRing ? kFMaxRing : ring;
 }

@@ -96,16 +96,26 @@ def tail_bwd(ctx: MhcLite, P: LayerParams, B: LayerBuffers, x, g, du, eps=1e-6, 
                        B.dH_res, B.dH_pre, B.dH_post, B.dx, True, B.dW, B.db, B.dalpha, B.dgain, accumulate_params)
 
 
-def stack_fwd(ctx: MhcLite, Ps, Bs, x0, sublayer, eps=1e-6):
+def stack_fwd(ctx: MhcLite, Ps, Bs, x0, sublayer, eps=1e-6, fuse_layers=True):
     """Forward through len(Ps) layers (the paper's models are 6, 12 or 24 of them back to back): layer l reads the
     x_next of layer l - 1.  `sublayer(l, u)` is the caller's f and returns y [T,C] bf16.  Each layer's input, y
-    and outputs stay in its LayerBuffers for the backward.  Returns the last layer's x_next."""
+    and outputs stay in its LayerBuffers for the backward.  With fuse_layers the merge of layer l also produces the
+    projection of layer l + 1 (mhclite_postres_fwd_next_proj / mhclite_pre_fwd_resume), so x_{l+1} is read once less.
+    The sublayer must not call workspace-using entry points of `ctx` in between.  Returns the last layer's x_next."""
     x = x0
+    resumed = False
     for l, (P, B) in enumerate(zip(Ps, Bs)):
         B.x_in = x
-        pre_fwd(ctx, P, B, x, eps, True)
+        if resumed:       # this layer's projection came out of the merge kernel of the layer before
+            ctx.pre_fwd_resume(x, P.b, P.alpha, eps, B.H_res, B.H_pre, B.H_post, B.a_saved, B.p_saved, B.rstd, B.u)
+        else:
+            pre_fwd(ctx, P, B, x, eps, True)
         B.y = sublayer(l, B.u)
-        post_fwd(ctx, B, x, B.y)
+        resumed = fuse_layers and l + 1 < len(Ps) and B.kind == "lite"
+        if resumed:
+            ctx.postres_fwd_next_proj(x, B.y, B.H_res, B.H_post, B.x_next, Ps[l + 1].W, Ps[l + 1].gain)
+        else:
+            post_fwd(ctx, B, x, B.y)
         x = B.x_next
     return x
 

@@ -150,8 +150,10 @@ def staged_dx_allowance(ref, fused):
 
 def dxhat_allowance_f(x, W, alpha, gain, dz, eps=1e-6):
     """Allowance for the projection-backward term of dx, sum_c e[t,c] W'[m,c]: the tensor-core kernel
-    rounds both operands to bf16 (as bf16 mixed-precision training does for this matmul), so each
-    product carries up to 2^-8 relative error: |error| <= 2^-8 sum_c |e[t,c]| |W'[m,c]|."""
+    rounds both operands to bf16 (as bf16 mixed-precision training does for this matmul).  bf16 keeps 8
+    significant bits, so rounding to nearest moves an operand by up to 2^-8 of its size and a product of
+    two rounded operands by up to 2^-7: |error| <= 2^-7 sum_c |e[t,c]| |W'[m,c]|.  Only the stress cases
+    (sharp logits, the mappings' gradient in isolation) use it; the five workloads pass without."""
     T, n, C = x.shape
     xh = x.reshape(T, n * C)
     rstd = 1.0 / np.sqrt((xh * xh).mean(axis=1) + eps)
@@ -159,7 +161,7 @@ def dxhat_allowance_f(x, W, alpha, gain, dz, eps=1e-6):
     av = np.concatenate([np.full(n_res, alpha[0]), np.full(n, alpha[1]), np.full(n, alpha[2])])
     e = np.abs(rstd[:, None] * av * dz)
     Wp = np.abs(gain[:, None] * W)
-    return 2.0 ** -8 * (e @ Wp.T).reshape(T, n, C)
+    return 2.0 ** -7 * (e @ Wp.T).reshape(T, n, C)
 
 
 def dxhat_allowance(inp, dz, eps=1e-6):
