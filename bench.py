@@ -376,6 +376,28 @@ def run_ours(args, wl, rank, world):
     acts = pool.views(T, n, C)
     x, y, g, du = acts
 
+    if wl.layers > 1:
+        # a stack of layers as the headline (--workload cfg3): the library calls of all layers, nothing else
+        sampler = ClockSampler(local) if rank == 0 else None
+        r = time_stack_case(mods, timer, ctx, wl, acts, dev, max(2, steps // 4), args.min_ms, not args.no_graph)
+        clocks = sampler.stop() if sampler else None
+        ctx.device_status()
+        if rank == 0:
+            rt = rates(n, C, T, r["ms_per_step"], peak, layers=wl.layers)
+            print(json.dumps({
+                "metric": METRIC, "value": D.job_tokens_per_s(T, world, 1, r["ms_per_step"]), "unit": UNIT, "n_gpus": world,
+                "steps": max(2, steps // 4), "warmup": warm, "ms_per_step": r["ms_per_step"], "repeats": r["repeats"],
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, f32 accumulate",
+                "data": "synthetic",
+                "config": {"workload": wl.name, "n": n, "C": C, "T_per_gpu": T, "layers": wl.layers, "passes": "fwd+bwd",
+                           "launch": r["launch"], "note": wl.note + "; library calls only, y_l and du_l are inputs"},
+                "clocks": clocks, "e2e": None, "gpu_launches": r["launches_per_step"] * max(2, steps // 4) * r["repeats"],
+                "roofline": {"bound": "hbm", "kernel": "whole stack", "achieved": rt["algorithmic_gbs"], "peak": peak,
+                             "peak_kind": peak_kind, "unit": "GB/s", "frac": rt["frac_of_measured_peak"], "traffic": None},
+                "token_layers_per_s": rt["token_layers_per_s"], "cpu_baseline": cpu_baseline}), flush=True)
+        D.shutdown()
+        return
+
     # ---- headline: K steps per repeat, device time, max over ranks -----------------------------
     sampler = ClockSampler(local) if rank == 0 else None
     # (the warm-up steps run inside time_layer_case: three plain, one counted, the capture, three replays)

@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(kActThreads) lite_act_fwd_k(int64_t T, int n, 
 constexpr int kGroupTok = 32;
 
 template <int N_>
-__global__ void __launch_bounds__(kActThreads) lite_act_premix_k(
+__global__ void __launch_bounds__(kActThreads, 4) lite_act_premix_k(
     int64_t T, int C8, int nf, int Npad, int ksplit, float inv_nC, float eps, const float* __restrict__ qpart,
     const float* __restrict__ ssq, const float* __restrict__ b, const float* __restrict__ alpha,
     float* __restrict__ H_res, float* __restrict__ H_pre, float* __restrict__ H_post, float* __restrict__ a_saved,
@@ -375,7 +375,7 @@ __global__ void __launch_bounds__(kActThreads) lite_act_bwd_k(
 //   A: one warp per token: activation backward from shared memory (no global load on the way).
 // (one token's staged inputs, as floats: a | p | dH_res | H_pre | H_post | dH_post | rstd)
 template <int N_>
-__global__ void __launch_bounds__(kActThreads) lite_tailpre_k(
+__global__ void __launch_bounds__(kActThreads, 4) lite_tailpre_k(
     int64_t T, int C8, int nf, float inv_nC, const uint4* __restrict__ x, const uint4* __restrict__ du,
     const float* __restrict__ a_saved, const float* __restrict__ p, const float* __restrict__ rstd,
     const float* __restrict__ alpha, const float* __restrict__ H_pre, const float* __restrict__ H_post,

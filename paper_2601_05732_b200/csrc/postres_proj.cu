@@ -51,6 +51,10 @@ struct PpArgs {
 __device__ __forceinline__ uint64_t pp_desc_k128(uint32_t addr) {     // K-major rows of 128 bytes, 128-byte swizzle
     return smem_desc(addr, 16, 1024, 2);
 }
+// Asks the L2 cache for a box ahead of the TMA load that will bring it to shared memory.
+__device__ __forceinline__ void pp_prefetch(const CUtensorMap* map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
+}
 __device__ __forceinline__ void pp_tma_store(const CUtensorMap* map, uint32_t src, int x, int y) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
@@ -110,9 +114,18 @@ postres_proj_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 if (lane == 0) mbar_expect_tx(full, (uint32_t)((N_ + 1) * a.tm * 128 + N_ * w_tile));
                 __syncwarp();
                 const uint32_t slot = smem_u32(smem + s * stage_bytes);
-                if (lane < N_) tma_load_2d(slot + lane * kPpBox, &tmx, full, lane * a.C + cb * 64, row0);
-                else if (lane == N_) tma_load_2d(slot + N_ * kPpBox, &tmy, full, cb * 64, row0);
-                else if (lane < nb) {
+                // the boxes two stages ahead start their way from HBM to L2 now: with two or three slots, each busy
+                // for a whole load + merge + store round, the loads alone keep too few bytes in flight
+                int pcb = cb + a.stages, prow = row0;
+                if (pcb >= nchunk) { pcb -= nchunk; prow = (tile + (int)gridDim.x) * a.tm; }
+                const bool pf = pcb < nchunk && (int64_t)prow < a.T;
+                if (lane < N_) {
+                    tma_load_2d(slot + lane * kPpBox, &tmx, full, lane * a.C + cb * 64, row0);
+                    if (pf) pp_prefetch(&tmx, lane * a.C + pcb * 64, prow);
+                } else if (lane == N_) {
+                    tma_load_2d(slot + N_ * kPpBox, &tmy, full, cb * 64, row0);
+                    if (pf) pp_prefetch(&tmy, pcb * 64, prow);
+                } else if (lane < nb) {
                     const int i = lane - N_ - 1;
                     tma_load_2d(slot + (N_ + 1) * kPpBox + i * w_tile, &tmw, full, i * a.C + cb * 64, 0);
                 }
