@@ -271,8 +271,13 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
             }
         }
     } else if (warp == 2) {
-        // ---- producer of the epilogue's data: x, g, du per 32-token quadrant, as far ahead as the ring allows
-        if (lane == 0) {
+        // ---- producer of the epilogue's data: x, g, du per 32-token quadrant, as far ahead as the ring allows.
+        //      Lane b issues the copy of box b (issuing a TMA instruction keeps a thread busy for ~100 cycles: eleven in
+        //      a row from one thread would hold back the slots behind it); lane 0 waits for the slot and arms its barrier.
+        {
+            constexpr int kBoxes = FUSED ? 2 * N_ + 1 : N_;
+            const CUtensorMap* mp = lane < N_ ? &tmx : (lane < 2 * N_ ? &tmg : &tmdu);
+            const int colb = lane < N_ ? lane * a.C : (lane < 2 * N_ ? (lane - N_) * a.C : 0);
             bool ok = true;
             for (int li = 0; li < nit && ok; ++li) {
                 const int64_t item = it_begin + li;
@@ -280,18 +285,15 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
                 const int cb = (int)(item - tile * a.ncb);
                 for (int q = 0; q < 4 && ok; ++q) {
                     const int si = li * 4 + q, ds = si % kDDSlots;
-                    ok = mbar_wait(smem_u32(&ctl->d_empty[ds]), ((si / kDDSlots) & 1) ^ 1, abort, 3, si);
+                    if (lane == 0) ok = mbar_wait(smem_u32(&ctl->d_empty[ds]), ((si / kDDSlots) & 1) ^ 1, abort, 3, si);
+                    ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     const uint32_t full = smem_u32(&ctl->d_full[ds]);
-                    mbar_expect_tx(full, kDSlot);
+                    if (lane == 0) mbar_expect_tx(full, kDSlot);
+                    __syncwarp();
                     const uint32_t dst = smem_u32(d_s + ds * kDSlot);
                     const int row = (int)(tile * kDTok + q * 32);
-#pragma unroll
-                    for (int j = 0; j < N_; ++j) {
-                        tma_load_2d(dst + j * kDBox, &tmx, full, j * a.C + cb * kDCh, row);
-                        if (FUSED) tma_load_2d(dst + (N_ + j) * kDBox, &tmg, full, j * a.C + cb * kDCh, row);
-                    }
-                    if (FUSED) tma_load_2d(dst + 2 * N_ * kDBox, &tmdu, full, cb * kDCh, row);
+                    if (lane < kBoxes) tma_load_2d(dst + lane * kDBox, mp, full, colb + cb * kDCh, row);
                 }
             }
         }
