@@ -61,6 +61,8 @@ SIGNATURES = {
     "mhc_sk20_tail_bwd_fused": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _i, _p, _p, _p, _p, _p, _p, _p, _p, _p,
                                      _p, _p, _p, _p, _p, _i, _p]),
     "mhclite_ds_gap": (_i, [_p, _i64, _p, _p, _p, _p]),
+    "mhclite_ds_gap_stats": (_i, [_p, _i64, _p, _p, _p]),
+    "mhclite_log_inv_nu_histogram": (_i, [_p, _i64, _p, _i, _f, _f, _p, _p]),
     "mhclite_depth_product": (_i, [_p, _i64, _p, _p, _i, _p]),
     "mhclite_relative_range": (_i, [_p, _i64, _p, _p, _p]),
     "mhclite_step_host_bytes": (_sz, [_i, _i, _i64]),
@@ -351,6 +353,18 @@ class MhcLite:
             u_host.data_ptr(), x_next_host.data_ptr(), dy_host.data_ptr(), dx_host.data_ptr(),
             self._ptr(dW, f), self._ptr(db, f), self._ptr(dalpha, f), self._ptr(dgain, f), int(accumulate_params),
             base, need, self._stream()), "mhclite_step_host")
+
+    def ds_gap_stats(self, H_res, stats):
+        """stats [4] f32 <- (max l1, sum l1, max column deviation, sum column deviation) over the tokens."""
+        f = self._torch.float32
+        self._check(self.lib.mhclite_ds_gap_stats(self._h, H_res.shape[0], self._ptr(H_res, f), self._ptr(stats, f),
+                                                  self._stream()), "mhclite_ds_gap_stats")
+
+    def log_inv_nu_histogram(self, X, bins, lo, hi, hist):
+        """hist [bins + 1] int64 <- histogram of log10(1/nu) of the matrices X[t]; hist[bins] counts nu == 0."""
+        self._check(self.lib.mhclite_log_inv_nu_histogram(self._h, X.shape[0], self._ptr(X, self._torch.float32), int(bins),
+                                                          float(lo), float(hi), self._ptr(hist, self._torch.int64),
+                                                          self._stream()), "mhclite_log_inv_nu_histogram")
 
     def depth_product(self, H_res, P, first=False):
         """P[t] <- H_res[t] P[t] in place (P[t] <- H_res[t] when first)."""

@@ -16,6 +16,9 @@ void launch_premix_bwd(const mhclite_ctx* c, int64_t T, const void* x, const flo
 void launch_tail_mix(const mhclite_ctx* c, int64_t T, const void* x, const void* g, const void* du, const float* H_res,
                      const float* H_pre, float* dH_pre, void* dx, cudaStream_t s);
 void launch_ds_gap(const mhclite_ctx* c, int64_t T, const float* H_res, float* l1, float* cdev, cudaStream_t s);
+void launch_ds_gap_stats(const mhclite_ctx* c, int64_t T, const float* H_res, float* stats, cudaStream_t s);
+void launch_log_inv_nu_hist(const mhclite_ctx* c, int64_t T, const float* X, int bins, float lo, float hi,
+                            unsigned long long* hist, cudaStream_t s);
 void launch_depth_product(const mhclite_ctx* c, int64_t T, const float* H_res, float* P, int first, cudaStream_t s);
 void launch_relative_range(const mhclite_ctx* c, int64_t T, const float* X, float* nu, cudaStream_t s);
 

@@ -80,6 +80,12 @@ using namespace mhcl;
     do {                                                                                            \
         if ((p) && !aligned16(p)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "pointer not 16-byte aligned: %s", #p); \
     } while (0)
+// An output that aliases an input is refused: the kernels read activations through the read-only path and by TMA.
+#define MHCL_NO_ALIAS(ctx, out, in)                                                                 \
+    do {                                                                                            \
+        if ((const void*)(out) == (const void*)(in))                                                \
+            return fail(ctx, MHCLITE_ERR_BAD_ARG, "%s must not alias %s", #out, #in);               \
+    } while (0)
 #define MHCL_DEVICE(ctx)                                                                            \
     DeviceGuard guard_((ctx)->device);                                                              \
     if (guard_.err != cudaSuccess) return check_cuda(ctx, guard_.err, "cudaSetDevice")
@@ -322,6 +328,7 @@ int mhclite_premix_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
     if (T == 0) return MHCLITE_OK;
     MHCL_PTR(ctx, x); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, u);
+    MHCL_NO_ALIAS(ctx, u, x);
     MHCL_DEVICE(ctx);
     launch_premix_fwd(ctx, T, x, H_pre, u, (cudaStream_t)stream);
     MHCL_LAUNCH_CHECK(ctx, "premix_fwd");
@@ -333,6 +340,7 @@ int mhclite_postres_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
     MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
     if (T == 0) return MHCLITE_OK;
     MHCL_PTR(ctx, x); MHCL_PTR(ctx, y); MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, x_next);
+    MHCL_NO_ALIAS(ctx, x_next, x); MHCL_NO_ALIAS(ctx, x_next, y);
     MHCL_DEVICE(ctx);
     launch_postres_fwd(ctx, T, x, y, H_res, H_post, x_next, (cudaStream_t)stream);
     MHCL_LAUNCH_CHECK(ctx, "postres_fwd");
@@ -347,6 +355,7 @@ int mhclite_pre_fwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, co
     MHCL_PTR(ctx, x); MHCL_PTR(ctx, W); MHCL_PTR(ctx, b); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain);
     MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, a_saved);
     MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd); MHCL_PTR(ctx, u);
+    MHCL_NO_ALIAS(ctx, u, x);
     if (!(eps >= 0.f)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "eps must be >= 0");
     Workspace w;
     int rc = need_workspace(ctx, T, 0, &w);
@@ -439,6 +448,8 @@ int mhclite_postres_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
     if (T == 0) return MHCLITE_OK;
     MHCL_PTR(ctx, x); MHCL_PTR(ctx, y); MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, g);
     MHCL_PTR(ctx, dy); MHCL_PTR(ctx, dH_res); MHCL_PTR(ctx, dH_post); MHCL_OPT_PTR(ctx, dx);
+    MHCL_NO_ALIAS(ctx, dy, y); MHCL_NO_ALIAS(ctx, dy, g); MHCL_NO_ALIAS(ctx, dy, x);
+    if (dx) { MHCL_NO_ALIAS(ctx, dx, x); MHCL_NO_ALIAS(ctx, dx, g); }
     MHCL_DEVICE(ctx);
     launch_postres_bwd(ctx, T, x, y, H_res, H_post, g, dy, dH_res, dH_post, dx, accumulate_dx, (cudaStream_t)stream);
     MHCL_LAUNCH_CHECK(ctx, "postres_bwd");
@@ -450,6 +461,7 @@ int mhclite_premix_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
     if (T == 0) return MHCLITE_OK;
     MHCL_PTR(ctx, x); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, du); MHCL_PTR(ctx, dH_pre); MHCL_OPT_PTR(ctx, dx);
+    if (dx) MHCL_NO_ALIAS(ctx, dx, x);
     MHCL_DEVICE(ctx);
     launch_premix_bwd(ctx, T, x, H_pre, du, dH_pre, dx, accumulate_dx, (cudaStream_t)stream);
     MHCL_LAUNCH_CHECK(ctx, "premix_bwd");
@@ -482,6 +494,7 @@ int mhclite_coeffs_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post); MHCL_PTR(ctx, dH_res);
     MHCL_PTR(ctx, dH_pre); MHCL_PTR(ctx, dH_post); MHCL_PTR(ctx, dx); MHCL_PTR(ctx, dW); MHCL_PTR(ctx, db);
     MHCL_PTR(ctx, dalpha); MHCL_PTR(ctx, dgain);
+    MHCL_NO_ALIAS(ctx, dx, x); MHCL_NO_ALIAS(ctx, dW, W);
     Workspace w;
     int rc = need_workspace(ctx, T, 0, &w);
     if (rc) return rc;
@@ -511,6 +524,7 @@ int mhclite_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, c
     MHCL_PTR(ctx, p_saved); MHCL_PTR(ctx, rstd); MHCL_PTR(ctx, H_res); MHCL_PTR(ctx, H_pre); MHCL_PTR(ctx, H_post);
     MHCL_PTR(ctx, g); MHCL_PTR(ctx, du); MHCL_PTR(ctx, dH_res); MHCL_PTR(ctx, dH_post); MHCL_PTR(ctx, dx);
     MHCL_PTR(ctx, dW); MHCL_PTR(ctx, db); MHCL_PTR(ctx, dalpha); MHCL_PTR(ctx, dgain);
+    MHCL_NO_ALIAS(ctx, dx, x); MHCL_NO_ALIAS(ctx, dx, g); MHCL_NO_ALIAS(ctx, dW, W);
     Workspace w;
     int rc = need_workspace(ctx, T, 0, &w);
     if (rc) return rc;
@@ -644,6 +658,31 @@ int mhclite_ds_gap(mhclite_ctx* ctx, int64_t T, const float* H_res, float* l1_er
     MHCL_DEVICE(ctx);
     launch_ds_gap(ctx, T, H_res, l1_err, colsum_dev, (cudaStream_t)stream);
     MHCL_LAUNCH_CHECK(ctx, "ds_gap");
+    return MHCLITE_OK;
+}
+
+int mhclite_ds_gap_stats(mhclite_ctx* ctx, int64_t T, const float* H_res, float* stats, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    MHCL_PTR(ctx, stats);
+    MHCL_DEVICE(ctx);
+    if (T == 0) return check_cuda(ctx, cudaMemsetAsync(stats, 0, 4 * sizeof(float), (cudaStream_t)stream), "memset stats");
+    MHCL_PTR(ctx, H_res);
+    launch_ds_gap_stats(ctx, T, H_res, stats, (cudaStream_t)stream);
+    MHCL_LAUNCH_CHECK(ctx, "ds_gap_stats");
+    return MHCLITE_OK;
+}
+
+int mhclite_log_inv_nu_histogram(mhclite_ctx* ctx, int64_t T, const float* X, int bins, float lo, float hi,
+                                 unsigned long long* hist, void* stream) {
+    MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
+    if (bins < 1 || bins > 4096 || !(hi > lo)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "bins must be in [1,4096] and hi > lo");
+    if (!hist || ((uintptr_t)hist & 7)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "hist null or not 8-byte aligned");
+    MHCL_DEVICE(ctx);
+    if (T == 0)
+        return check_cuda(ctx, cudaMemsetAsync(hist, 0, (size_t)(bins + 1) * 8, (cudaStream_t)stream), "memset hist");
+    MHCL_PTR(ctx, X);
+    launch_log_inv_nu_hist(ctx, T, X, bins, lo, hi, hist, (cudaStream_t)stream);
+    MHCL_LAUNCH_CHECK(ctx, "log_inv_nu_hist");
     return MHCLITE_OK;
 }
 

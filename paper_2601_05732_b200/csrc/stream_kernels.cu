@@ -317,6 +317,67 @@ __global__ void relative_range_k(int64_t T, int n, const float* __restrict__ X, 
     nu[t] = (hi > 0.f) ? lo / hi : 0.f;
 }
 
+// Population statistics of the doubly-stochastic gap over all tokens in one pass (the procedure behind the paper's
+// Fig. 3): stats = { max l1-error, sum of l1-errors, max column-sum deviation, sum of column-sum deviations }.
+// Non-negative floats order like their bit patterns, so the maxima are integer atomics.
+__global__ void __launch_bounds__(256) ds_gap_stats_k(int64_t T, int n, const float* __restrict__ H, float* stats) {
+    float l1m = 0.f, l1s = 0.f, cdm = 0.f, cds = 0.f;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < T; t += (int64_t)gridDim.x * blockDim.x) {
+        const float* h = H + t * n * n;
+        float err = 0.f, cmax = 0.f;
+        for (int i = 0; i < n; ++i) {
+            float rs = 0.f, cs = 0.f;
+            for (int j = 0; j < n; ++j) { rs += h[i * n + j]; cs += h[j * n + i]; }
+            err += fabsf(rs - 1.f) + fabsf(cs - 1.f);
+            cmax = fmaxf(cmax, fabsf(cs - 1.f));
+        }
+        l1m = fmaxf(l1m, err); l1s += err; cdm = fmaxf(cdm, cmax); cds += cmax;
+    }
+    l1m = warp_max(l1m); cdm = warp_max(cdm); l1s = warp_sum(l1s); cds = warp_sum(cds);
+    __shared__ float red[4][8];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane == 0) { red[0][w] = l1m; red[1][w] = l1s; red[2][w] = cdm; red[3][w] = cds; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int k = 1; k < 8; ++k) { red[0][0] = fmaxf(red[0][0], red[0][k]); red[1][0] += red[1][k];
+                                       red[2][0] = fmaxf(red[2][0], red[2][k]); red[3][0] += red[3][k]; }
+        atomicMax(reinterpret_cast<int*>(stats), __float_as_int(red[0][0]));
+        atomicAdd(stats + 1, red[1][0]);
+        atomicMax(reinterpret_cast<int*>(stats + 2), __float_as_int(red[2][0]));
+        atomicAdd(stats + 3, red[3][0]);
+    }
+}
+
+// Histogram over the tokens of log10(1 / nu), nu the relative range of Eq. (3) (the procedure behind the paper's
+// Fig. 4): `bins` equal bins on [lo, hi), values outside clamped to the end bins; hist[bins] counts matrices without a
+// positive entry (nu = 0).
+__global__ void __launch_bounds__(256) log_inv_nu_hist_k(int64_t T, int n, const float* __restrict__ X, int bins, float lo,
+                                                         float hi, unsigned long long* hist) {
+    extern __shared__ unsigned int sh[];
+    for (int b = threadIdx.x; b <= bins; b += blockDim.x) sh[b] = 0;
+    __syncthreads();
+    const float scale = (float)bins / (hi - lo);
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < T; t += (int64_t)gridDim.x * blockDim.x) {
+        const float* x = X + t * n * n;
+        float mn = 3.4e38f, mx = -3.4e38f;
+        for (int e = 0; e < n * n; ++e) {
+            const float v = x[e];
+            mx = fmaxf(mx, v);
+            if (v > 0.f) mn = fminf(mn, v);
+        }
+        int b = bins;
+        if (mx > 0.f) {
+            const float l = log10f(mx / mn);
+            b = (int)floorf((l - lo) * scale);
+            b = b < 0 ? 0 : (b >= bins ? bins - 1 : b);
+        }
+        atomicAdd(&sh[b], 1u);
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b <= bins; b += blockDim.x)
+        if (sh[b]) atomicAdd(hist + b, (unsigned long long)sh[b]);
+}
+
 // ---- launchers -----------------------------------------------------------------------------------
 static int grid_for(int64_t items, int sm_count, int per_sm) {
     int64_t blocks = (items + kThreads - 1) / kThreads;
@@ -380,6 +441,23 @@ void launch_ds_gap(const mhclite_ctx* c, int64_t T, const float* H_res, float* l
     c->launches += 1;
     const int grid = (int)((T + 127) / 128);
     ds_gap_k<<<grid, 128, 0, s>>>(T, c->n, H_res, l1, cdev);
+}
+
+void launch_ds_gap_stats(const mhclite_ctx* c, int64_t T, const float* H_res, float* stats, cudaStream_t s) {
+    c->launches += 1;
+    cudaMemsetAsync(stats, 0, 4 * sizeof(float), s);
+    int64_t blocks = (T + 255) / 256;
+    if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
+    ds_gap_stats_k<<<(unsigned)blocks, 256, 0, s>>>(T, c->n, H_res, stats);
+}
+
+void launch_log_inv_nu_hist(const mhclite_ctx* c, int64_t T, const float* X, int bins, float lo, float hi,
+                            unsigned long long* hist, cudaStream_t s) {
+    c->launches += 1;
+    cudaMemsetAsync(hist, 0, (size_t)(bins + 1) * sizeof(unsigned long long), s);
+    int64_t blocks = (T + 255) / 256;
+    if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
+    log_inv_nu_hist_k<<<(unsigned)blocks, 256, (size_t)(bins + 1) * sizeof(unsigned int), s>>>(T, c->n, X, bins, lo, hi, hist);
 }
 
 void launch_depth_product(const mhclite_ctx* c, int64_t T, const float* H_res, float* P, int first, cudaStream_t s) {

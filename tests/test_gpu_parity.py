@@ -145,6 +145,11 @@ def test_bad_arguments_are_rejected_without_launch():
     assert lib.mhclite_premix_fwd(h, T, None, G.B.H_pre.data_ptr(), G.B.u.data_ptr(), None) == ERR_BAD_ARG
     assert lib.mhclite_premix_fwd(h, T, x + 2, G.B.H_pre.data_ptr(), G.B.u.data_ptr(), None) == ERR_BAD_ARG
     assert b"aligned" in lib.mhclite_last_error(h)
+    # in-place use is refused (outputs must not alias inputs)
+    assert lib.mhclite_postres_fwd(h, T, x, G.y.data_ptr(), G.B.H_res.data_ptr(), G.B.H_post.data_ptr(), x, None) == ERR_BAD_ARG
+    assert b"alias" in lib.mhclite_last_error(h)
+    assert lib.mhclite_postres_bwd(h, T, x, G.y.data_ptr(), G.B.H_res.data_ptr(), G.B.H_post.data_ptr(), G.g.data_ptr(),
+                                   G.B.dy.data_ptr(), G.B.dH_res.data_ptr(), G.B.dH_post.data_ptr(), G.g.data_ptr(), 0, None) == ERR_BAD_ARG
     # a context without workspace refuses the calls that need one
     ctx2 = MhcLite(n, C)
     B = G.B
@@ -304,3 +309,34 @@ def test_depth_product_and_relative_range(n):
     ref_nu = O.relative_range(X[ok].astype(np.float64))
     np.testing.assert_allclose(host(nu)[ok], ref_nu, rtol=1e-6)
     assert float(nu[0]) == 0.0
+
+
+def test_gap_statistics_and_relative_range_histogram():
+    # Section 3.1's population figures in one pass each: gap statistics of an SK output (Fig. 3's procedure) and the
+    # histogram of log10(1/nu) of the SK input (Fig. 4's), against the oracle's per-token values
+    n, C, T = 4, 64, 5000
+    sk = synth.make_layer_inputs(n, C, T, seed=16, kind="sk", alpha=[1.0, 1.0, 1.0], w_std=0.3)
+    sk["b"][:16] = synth.normal(16, 99, (16,), 6.0).astype(np.float32)
+    G = GpuLayer(sk, kind="sk"); G.forward()
+    ref = oracle_fwd(sk, kind="sk")
+    stats = torch.empty(4, device=DEV)
+    G.ctx.ds_gap_stats(G.B.H_res, stats); torch.cuda.synchronize()
+    Hg = host(G.B.H_res)                                   # the statistics of the matrices the GPU produced
+    l1 = O.l1_error(Hg); cd = np.abs(O.column_sums(Hg) - 1).max(axis=1)
+    got = host(stats)
+    np.testing.assert_allclose(got, [l1.max(), l1.sum(), cd.max(), cd.sum()], rtol=2e-4, atol=1e-5)
+    assert abs(got[0] - O.l1_error(ref["H_res"]).max()) <= 1e-2 * O.l1_error(ref["H_res"]).max() + 1e-5
+    M0 = np.ascontiguousarray(ref["M0"], dtype=np.float32)
+    M0[7] = 0.0                                            # a matrix without a positive entry
+    bins, lo, hi = 20, 0.0, 10.0
+    hist = torch.empty(bins + 1, dtype=torch.int64, device=DEV)
+    G.ctx.log_inv_nu_histogram(torch.from_numpy(M0).to(DEV), bins, lo, hi, hist); torch.cuda.synchronize()
+    nu = O.relative_range(M0.astype(np.float64))
+    ok = nu > 0
+    l = np.log10(1.0 / nu[ok])
+    idx = np.clip(np.floor((l - lo) * bins / (hi - lo)).astype(int), 0, bins - 1)
+    expect = np.bincount(idx, minlength=bins + 1); expect[bins] = int((~ok).sum())
+    h = hist.cpu().numpy()
+    assert h.sum() == T and h[bins] == 1
+    # a value within rounding of a bin edge may fall either side: compare cumulative counts with a slack of a few
+    assert np.abs(np.cumsum(h) - np.cumsum(expect)).max() <= 3
