@@ -583,6 +583,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg5")
     ap.add_argument("--T", type=int, default=0, help="override the token count of the workload")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers of a stack workload (cfg3)")
     ap.add_argument("--cpu-sample", type=int, default=0, help="tokens of the oracle's timed sample (0: by workload)")
     ap.add_argument("--min-ms", type=float, default=500.0, help="least timed work of the headline (repeats of K steps)")
     ap.add_argument("--min-ms-table", type=float, default=100.0, help="least timed work of each row of the table")
@@ -598,6 +599,8 @@ def main():
     wl = synth.WORKLOADS[args.workload]
     if args.T:
         wl = dataclasses.replace(wl, T=args.T)
+    if args.layers:
+        wl = dataclasses.replace(wl, layers=args.layers)
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     if args.impl == "reference":
