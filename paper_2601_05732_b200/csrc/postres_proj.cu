@@ -208,7 +208,7 @@ postres_proj_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 if (ok) ok = mbar_wait(smem_u32(&ctl->full[s]), (it / a.stages) & 1, abort, 6, it);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                unsigned char* slot = smem + s * stage_bytes;
+                const uint32_t slot = smem_u32(smem + s * stage_bytes);
                 if (row < a.tm) {
 #pragma unroll
                     for (int pp = 0; pp < 4; ++pp) {
@@ -216,8 +216,8 @@ postres_proj_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                         const int po = row * 128 + ((pc ^ (row & 7)) << 4);
                         uint64_t xf[N_][4], yf[4];
 #pragma unroll
-                        for (int j = 0; j < N_; ++j) unpack8x2(*reinterpret_cast<const uint4*>(slot + j * kPpBox + po), xf[j]);
-                        unpack8x2(*reinterpret_cast<const uint4*>(slot + N_ * kPpBox + po), yf);
+                        for (int j = 0; j < N_; ++j) unpack8x2(lds128(slot + j * kPpBox + po), xf[j]);
+                        unpack8x2(lds128(slot + N_ * kPpBox + po), yf);
 #pragma unroll
                         for (int i = 0; i < N_; ++i) {
                             uint64_t o[4];
@@ -228,7 +228,7 @@ postres_proj_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
 #pragma unroll
                                 for (int k = 0; k < 4; ++k) o[k] = fma2(hr2[i][j], xf[j][k], o[k]);
                             const uint4 v = pack8x2(o);
-                            *reinterpret_cast<uint4*>(slot + i * kPpBox + po) = v;
+                            sts128(slot + i * kPpBox + po, v);
                             uint64_t r[4];                                       // the next layer normalises what is stored
                             unpack8x2(v, r);
 #pragma unroll

@@ -135,12 +135,12 @@ proj_fwd_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ C
 #pragma unroll
             for (int m = 0; m < 2; ++m) {
                 if (m < mt) {
-                    const unsigned char* xr = smem + s * stage_bytes + m * kTcXBytes + row * 128;
+                    const uint32_t xr = smem_u32(smem + s * stage_bytes + m * kTcXBytes + row * 128);
                     float part = 0.f;                       // per 64-element chunk, then added: short chains round less
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         float f[8];
-                        unpack8(*reinterpret_cast<const uint4*>(xr + ((c ^ (row & 7)) << 4)), f);
+                        unpack8(lds128(xr + ((c ^ (row & 7)) << 4)), f);
 #pragma unroll
                         for (int e = 0; e < 8; ++e) part = fmaf(f[e], f[e], part);
                     }

@@ -277,7 +277,7 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                         hr2[i][j] = pack2f(h, h);
                     }
             }
-            unsigned char* slot = slots + ((ti * 4 + quad) % kFSlots) * kSlot;
+            const uint32_t slot = smem_u32(slots + ((ti * 4 + quad) % kFSlots) * kSlot);
             ok = mbar_wait(smem_u32(&ctl->d_full[quad][ti & 1]), (ti >> 1) & 1, abort, 7, ti);
             // MODE 0 writes dx over x itself: the G MMAs must have read the boxes
             if (MODE == 0 && ok) ok = mbar_wait(smem_u32(&ctl->g_done[quad][ti & 1]), (ti >> 1) & 1, abort, 8, ti);
@@ -299,8 +299,8 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                     uint64_t gf[MODE == 1 ? N_ : 1][4], df[4];
                     if (MODE == 1) {
 #pragma unroll
-                        for (int i = 0; i < N_; ++i) unpack8x2(*reinterpret_cast<const uint4*>(slot + (N_ + i) * kFBox + po), gf[i]);
-                        unpack8x2(*reinterpret_cast<const uint4*>(slot + 2 * N_ * kFBox + po), df);
+                        for (int i = 0; i < N_; ++i) unpack8x2(lds128(slot + (N_ + i) * kFBox + po), gf[i]);
+                        unpack8x2(lds128(slot + 2 * N_ * kFBox + po), df);
                     }
                     ftc_ld_wait();
 #pragma unroll
@@ -308,7 +308,7 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
 #pragma unroll
                     for (int j = 0; j < N_; ++j) {
                         uint64_t xf[4], o[4];
-                        unpack8x2(*reinterpret_cast<const uint4*>(slot + j * kFBox + po), xf);
+                        unpack8x2(lds128(slot + j * kFBox + po), xf);
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
                             o[k] = fma2(xf[k], nkap2, pack2f(__uint_as_float(acc[j][2 * k]), __uint_as_float(acc[j][2 * k + 1])));
@@ -322,12 +322,12 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                         }
                         if (MODE == 2) {
                             uint64_t old[4];
-                            unpack8x2(*reinterpret_cast<const uint4*>(slot + (N_ + j) * kFBox + po), old);
+                            unpack8x2(lds128(slot + (N_ + j) * kFBox + po), old);
 #pragma unroll
                             for (int k = 0; k < 4; ++k) o[k] = fma2(old[k], pack2f(1.f, 1.f), o[k]);
                         }
                         // dx takes the place of g (of the old dx; of x itself in MODE 0) in the slot
-                        *reinterpret_cast<uint4*>(slot + (kOut + j) * kFBox + po) = pack8x2(o);
+                        sts128(slot + (kOut + j) * kFBox + po, pack8x2(o));
                     }
                 }
                 tc_fence_before();
@@ -345,7 +345,7 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                 // lane j stores box j once both warps of the quadrant have written their part
                 bool oks = lane >= N_ || mbar_wait(smem_u32(&ctl->q_done[quad]), ti & 1, abort, 10, ti);
                 if (oks && lane < N_ && row0 < a.T) {
-                    tma_store_2d(&tmdx, smem_u32(slot + (kOut + lane) * kFBox), lane * a.C + c0, (int)row0);
+                    tma_store_2d(&tmdx, slot + (kOut + lane) * kFBox, lane * a.C + c0, (int)row0);
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 }

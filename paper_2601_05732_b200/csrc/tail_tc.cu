@@ -370,7 +370,7 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const unsigned char* slot = d_s + ds * kDSlot;
+            const uint32_t slot = smem_u32(d_s + ds * kDSlot);
             const int rsw = (lane >> 1) & 3;                    // 64-byte swizzle: piece ^= (row / 2) % 4
             const uint32_t tbase = tmem + ((uint32_t)(quad * 32) << 16) + buf * kDW;
 #pragma unroll
@@ -383,8 +383,8 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
                 float gf[FUSED ? N_ : 1][8], df[8];
                 if (FUSED) {
 #pragma unroll
-                    for (int i = 0; i < N_; ++i) unpack8(*reinterpret_cast<const uint4*>(slot + (N_ + i) * kDBox + po), gf[i]);
-                    unpack8(*reinterpret_cast<const uint4*>(slot + 2 * N_ * kDBox + po), df);
+                    for (int i = 0; i < N_; ++i) unpack8(lds128(slot + (N_ + i) * kDBox + po), gf[i]);
+                    unpack8(lds128(slot + 2 * N_ * kDBox + po), df);
                 }
                 tc_ld_wait();
 #pragma unroll
@@ -393,7 +393,7 @@ tail_dx_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CU
 #pragma unroll
                 for (int j = 0; j < N_; ++j) {
                     float xf[8], o[8];
-                    unpack8(*reinterpret_cast<const uint4*>(slot + j * kDBox + po), xf);
+                    unpack8(lds128(slot + j * kDBox + po), xf);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) o[e] = fmaf(-xf[e], kap, __uint_as_float(acc[j][e]));
                     if (FUSED) {
