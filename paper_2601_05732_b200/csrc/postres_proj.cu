@@ -9,7 +9,7 @@
 // A CTA takes tiles of tm <= 128 tokens and walks the C / 64 channel blocks of a tile; per block ("stage"):
 //   * TMA (128-byte swizzle) brings the n boxes of x_l [tm tokens x 64 channels], the box of y, and the n tiles of
 //     W' (bf16 hi rows | lo rows, K-major) that belong to these channels of the n streams;
-//   * eight merge warps (thread = token, two threads per token splitting the row's eight 16-byte pieces) compute
+//   * sixteen merge warps (thread = token, four threads per token splitting the row's eight 16-byte pieces) compute
 //     the n output boxes with packed fp32 FMAs and write them OVER the x boxes, in the same swizzled layout (a
 //     thread has read every input of a piece before it writes there); they also add up the squares of the
 //     rounded outputs;
@@ -29,15 +29,15 @@ namespace mhcl {
 
 constexpr int kPpRows = 128;                      // UMMA M: rows of the accumulator
 constexpr int kPpBox = kPpRows * 128;             // bytes reserved per box: 128 rows x 64 channels of bf16
-constexpr int kPpMergeWarps = 8;
-constexpr int kPpThreads = 128 + 32 * kPpMergeWarps;   // warp 0 loads, 1 issues MMAs, 2 stores, 3 idles; 4..11 merge
+constexpr int kPpMergeWarps = 16;                 // four per lane quadrant: each takes two of a row's eight pieces
+constexpr int kPpThreads = 128 + 32 * kPpMergeWarps;   // warp 0 loads, 1 issues MMAs, 2 stores, 3 idles; 4.. merge
 constexpr int kPpMaxStages = 3;
 
 struct PpCtl {
     uint64_t full[kPpMaxStages], merged[kPpMaxStages], empty[kPpMaxStages], acc_full[2], acc_empty[2], sq_ready[2];
     uint32_t tmem_base;
     int abort[3];
-    float ssq_s[2][kPpRows];
+    float ssq_s[kPpMergeWarps / 4 - 1][kPpRows];   // the other warps' sums of squares of the tile that is being read out
 };
 
 struct PpArgs {
@@ -83,7 +83,7 @@ postres_proj_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[b]), 4);
-            mbar_init(smem_u32(&ctl->sq_ready[b]), 4);
+            mbar_init(smem_u32(&ctl->sq_ready[b]), kPpMergeWarps - 4);
         }
         ctl->abort[0] = ctl->abort[1] = ctl->abort[2] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -211,8 +211,8 @@ postres_proj_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 const uint32_t slot = smem_u32(smem + s * stage_bytes);
                 if (row < a.tm) {
 #pragma unroll
-                    for (int pp = 0; pp < 4; ++pp) {
-                        const int pc = half * 4 + pp;                          // 16-byte piece of the 128-byte row
+                    for (int pp = 0; pp < 32 / kPpMergeWarps; ++pp) {
+                        const int pc = half * (32 / kPpMergeWarps) + pp;       // 16-byte piece of the 128-byte row
                         const int po = row * 128 + ((pc ^ (row & 7)) << 4);
                         uint64_t xf[N_][4], yf[4];
 #pragma unroll
@@ -246,8 +246,12 @@ postres_proj_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             float sqa, sqb;
             unpack2f(sq2, sqa, sqb);
             const float sq = sqa + sqb;
-            if (half == 1) {
-                ctl->ssq_s[b][row] = sq;
+            if (half != 0) {
+                // the one buffer of partial sums is free once the tile before this one has been read out
+                if (tcount > 0) ok = mbar_wait(smem_u32(&ctl->acc_empty[(tcount - 1) & 1]), ((tcount - 1) >> 1) & 1, abort, 9, tcount);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                ctl->ssq_s[half - 1][row] = sq;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->sq_ready[b]));
             } else {
@@ -270,7 +274,12 @@ postres_proj_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                                     make_float4(hi[e] + lo[e], hi[e + 1] + lo[e + 1], hi[e + 2] + lo[e + 2], hi[e + 3] + lo[e + 3]);
                     }
                 }
-                if (live) a.ssq[t] = sq + ctl->ssq_s[b][row];
+                if (live) {
+                    float tot = sq;
+#pragma unroll
+                    for (int h = 0; h < kPpMergeWarps / 4 - 1; ++h) tot += ctl->ssq_s[h][row];
+                    a.ssq[t] = tot;
+                }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));

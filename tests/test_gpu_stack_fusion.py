@@ -47,11 +47,12 @@ def test_merge_with_next_projection(n, C, T):
     for k, got in (("H_res", B1.H_res), ("H_pre", B1.H_pre), ("H_post", B1.H_post), ("a_saved", B1.a_saved)):
         check_f32(k, host(got), co["a" if k == "a_saved" else k], 2e-4)
     check_bf16("u", host(B1.u), O.premix_fwd(xn, co["H_pre"]))
-    # same results as the un-fused sequence on the same x_next
+    # same results as the un-fused sequence on the same x_next, up to the summation order of the contraction (these
+    # logits are sharp: alpha = 1, so 1e-5 in a logit shows at that size in the mappings)
     B2 = L.LayerBuffers(ctx, T)
     L.pre_fwd(ctx, P1, B2, B0.x_next, eps, True)
     torch.cuda.synchronize()
-    assert float((B2.H_res - B1.H_res).abs().max()) < 2e-5 and float((B2.rstd - B1.rstd).abs().max()) < 1e-5 * float(B2.rstd.max())
+    assert float((B2.H_res - B1.H_res).abs().max()) < 5e-5 and float((B2.rstd - B1.rstd).abs().max()) < 1e-5 * float(B2.rstd.max())
 
 
 def test_resume_needs_pending_partials():
