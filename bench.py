@@ -82,6 +82,38 @@ def ncu_traffic(kernel: str, workload: str, T: int):
     return None
 
 
+_TRAFFIC_KERNELS = {"proj_fwd": ("proj_fwd_tc_k", "proj_tc.cu"), "act_premix": ("lite_act_premix_t_k", "act_kernels.cu"),
+                    "postres_fwd": ("postres_fwd_k", "stream_kernels.cu"), "postres_bwd": ("postres_bwd_k", "stream_kernels.cu"),
+                    "tail_pre": ("lite_tailpre_w_k", "act_kernels.cu"), "tail_dx": ("tail_ftc_k", "tail_ftc.cu")}
+
+
+def write_ncu_traffic(workload: str, T: int, csv_path: str) -> None:
+    """Writes profiles/dram_traffic_<workload>.txt from an `ncu --csv` log of one step of this workload at T tokens that
+    holds dram__bytes_read.sum and dram__bytes_write.sum (the first launch of each kernel counts), with the hash of
+    each kernel's source so that a later edit voids the figure.  Needs no GPU."""
+    import csv
+    import hashlib
+    rows = list(csv.reader(open(csv_path)))
+    head = next(r for r in rows if "Kernel Name" in r and "Metric Name" in r)
+    k_i, m_i, v_i = head.index("Kernel Name"), head.index("Metric Name"), head.index("Metric Value")
+    seen = {}
+    for r in rows:
+        if len(r) <= v_i or not r[0].isdigit():
+            continue
+        name = r[k_i].replace("void ", "").replace("mhcl::", "").split("<")[0].split("(")[0]
+        seen.setdefault(name, {}).setdefault(r[m_i], float(r[v_i].replace(",", "")))
+    lines = []
+    for key, (kname, src) in _TRAFFIC_KERNELS.items():
+        if kname not in seen:
+            continue
+        b = int(seen[kname]["dram__bytes_read.sum"] + seen[kname]["dram__bytes_write.sum"])
+        h = hashlib.sha256(open(os.path.join(ROOT, "paper_2601_05732_b200", "csrc", src), "rb").read()).hexdigest()
+        lines.append(f"{key} {T} {b} {src} {h}")
+    out = os.path.join(ROOT, "profiles", f"dram_traffic_{workload}.txt")
+    open(out, "w").write("\n".join(lines) + "\n")
+    print("\n".join(lines))
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -593,7 +625,12 @@ def main():
     ap.add_argument("--no-table", action="store_true", help="skip the table of the other workloads")
     ap.add_argument("--unfused", action="store_true", help="time the un-fused call sequence (six entry points)")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph of one step")
+    ap.add_argument("--traffic-from-ncu", default="", metavar="CSV",
+                    help="no run: write profiles/dram_traffic_<workload>.txt from an ncu --csv log of one step at --T tokens")
     args = ap.parse_args()
+    if args.traffic_from_ncu:
+        write_ncu_traffic(args.workload, args.T or synth.WORKLOADS[args.workload].T, args.traffic_from_ncu)
+        return
 
     from paper_2601_05732_b200 import synth
     wl = synth.WORKLOADS[args.workload]

@@ -126,5 +126,7 @@ __host__ __device__ constexpr uint32_t umma_idesc_mn(int m, int n, int a_mn, int
 bool tensor_maps_available();
 bool make_tensor_map_2d(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t pitch_elems,
                         uint32_t box_cols, uint32_t box_rows, int swizzle_bytes);
+bool make_tensor_map_3d(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t pitch1_elems,
+                        uint64_t pitch2_elems, uint32_t box0, uint32_t box1, uint32_t box2, int swizzle_bytes);
 
 }  // namespace mhcl
