@@ -20,6 +20,11 @@
 
 namespace mhcl {
 
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
 constexpr int kGTok = 64;                       // tokens per stage of the G kernel (4 k-steps of 16)
 constexpr int kGStages = 2;
 constexpr int kGXBox = kGTok * 128;             // one TMA box: 64 tokens x 64 channels of bf16
@@ -32,8 +37,8 @@ struct GCtl {
 
 template <int MT>
 __global__ void __launch_bounds__(192, 1)
-tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __nv_bfloat16* __restrict__ ehi,
-            const __nv_bfloat16* __restrict__ elo, int64_t T, int64_t tok_per_split, int nC, int Kp, int tmem_cols,
+tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmeh,
+            const __grid_constant__ CUtensorMap tmel, int64_t T, int64_t tok_per_split, int nC, int Kp, int tmem_cols,
             float* __restrict__ Gpart, int* __restrict__ status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -66,22 +71,26 @@ tail_g_tc_k(const __grid_constant__ CUtensorMap tmx, const __nv_bfloat16* __rest
     const uint32_t tmem = ctl->tmem_base;
 
     if (warp == 0) {
-        if (lane == 0) {
-            for (int i = 0; i < nblk; ++i) {
-                const int s = i % kGStages;
-                if (!mbar_wait(smem_u32(&ctl->empty[s]), ((i / kGStages) & 1) ^ 1, abort, 1, i)) break;
-                const uint32_t full = smem_u32(&ctl->full[s]);
-                mbar_expect_tx(full, stage_bytes);
-                const uint32_t dst = smem_u32(smem + s * stage_bytes);
-                const int64_t t0 = t_begin + (int64_t)i * kGTok;
-#pragma unroll
-                for (int b = 0; b < MT * 2; ++b) tma_load_2d(dst + b * kGXBox, &tmx, full, m0 + b * 64, (int)t0);
-                // the 64 tokens' pieces of every column group: 1 KB runs, 2 KB apart in the granule
-                const int64_t gran = (t0 >> 7) * ncg * 1024 + (t0 & 64) * 8;       // element offset
-                for (int cg = 0; cg < ncg; ++cg) {
-                    bulk_load(dst + x_bytes + cg * 1024, ehi + gran + (int64_t)cg * 1024, 1024, full);
-                    bulk_load(dst + x_bytes + e_bytes + cg * 1024, elo + gran + (int64_t)cg * 1024, 1024, full);
-                }
+        // Producer: lane b issues copy b of a stage (the x boxes, then the 64 tokens' pieces of every column group of e_hi
+        // and of e_lo as one box each: 1 KB runs, 2 KB apart in the granule); lane 0 waits for the stage and arms it.
+        // One thread issuing every copy in turn (forty-odd of them while e went by plain bulk copies) was what bound
+        // this kernel.
+        bool ok = true;
+        for (int i = 0; i < nblk && ok; ++i) {
+            const int s = i % kGStages;
+            if (lane == 0) ok = mbar_wait(smem_u32(&ctl->empty[s]), ((i / kGStages) & 1) ^ 1, abort, 1, i);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const uint32_t full = smem_u32(&ctl->full[s]);
+            if (lane == 0) mbar_expect_tx(full, stage_bytes);
+            __syncwarp();
+            const uint32_t dst = smem_u32(smem + s * stage_bytes);
+            const int64_t t0 = t_begin + (int64_t)i * kGTok;
+            if (lane < MT * 2) {
+                tma_load_2d(dst + lane * kGXBox, &tmx, full, m0 + lane * 64, (int)t0);
+            } else if (lane < MT * 2 + 2) {
+                const int lo = lane - MT * 2;
+                tma_load_3d(dst + x_bytes + lo * e_bytes, lo ? &tmel : &tmeh, full, 0, (int)((t0 & 64) >> 3), (int)((t0 >> 7) * ncg));
             }
         }
     } else if (warp == 1) {
@@ -192,10 +201,6 @@ struct DxArgs {
     int* status;
 };
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
-}
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
     asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
                  ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
@@ -485,7 +490,7 @@ __global__ void __launch_bounds__(256) pack_wb_k(int n, int C, int N, int Kp, in
 
 // ---- host side -------------------------------------------------------------------------------------
 template <int MT>
-static void launch_g_t(const TailPlan& p, const CUtensorMap& tmx, const void* ehi, const void* elo, int64_t T, int nC,
+static bool launch_g_t(const TailPlan& p, const CUtensorMap& tmx, const void* ehi, const void* elo, int64_t T, int nC,
                        float* Gpart, int* status, cudaStream_t s) {
     const int stage_bytes = MT * 2 * kGXBox + 2 * (p.Kp >> 3) * (kGTok * 16);
     const int smem = kGStages * stage_bytes + (int)sizeof(GCtl) + 1024;
@@ -493,8 +498,15 @@ static void launch_g_t(const TailPlan& p, const CUtensorMap& tmx, const void* eh
     while (tmem_cols < MT * p.Kp) tmem_cols *= 2;
     cudaFuncSetAttribute(tail_g_tc_k<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     dim3 grid(p.g_groups, p.g_splits);
-    tail_g_tc_k<MT><<<grid, 192, smem, s>>>(tmx, (const __nv_bfloat16*)ehi, (const __nv_bfloat16*)elo, T,
+    // e_hi / e_lo as [granule x column group][16 groups of 8 tokens][8 tokens x 8 columns]: a box takes half a granule's
+    // rows (64 tokens) of all column groups
+    const uint64_t erows = (uint64_t)((T + kEGranule - 1) / kEGranule) * (uint64_t)(p.Kp >> 3);
+    CUtensorMap tmeh, tmel;
+    if (!make_tensor_map_3d(&tmeh, ehi, 64, 16, erows, 64, 1024, 64, 8, (uint32_t)(p.Kp >> 3), 0)) return false;
+    if (!make_tensor_map_3d(&tmel, elo, 64, 16, erows, 64, 1024, 64, 8, (uint32_t)(p.Kp >> 3), 0)) return false;
+    tail_g_tc_k<MT><<<grid, 192, smem, s>>>(tmx, tmeh, tmel, T,
                                             p.g_tok_per_split, nC, p.Kp, tmem_cols, Gpart, status);
+    return true;
 }
 
 // G partials of every token range -> Gpart[g_splits][nC][Kp].  False when no tensor map could be made.
@@ -503,13 +515,14 @@ bool launch_tail_g_tc(const mhclite_ctx* c, int64_t T, const TailPlan& p, const 
     const int nC = c->n * c->C;
     CUtensorMap tmx;
     if (!make_tensor_map_2d(&tmx, x, (uint64_t)nC, (uint64_t)T, (uint64_t)nC, 64, kGTok, 128)) return false;
-    c->launches += 1;
+    bool ok;
     switch (p.g_mt) {
-        case 1: launch_g_t<1>(p, tmx, ehi, elo, T, nC, Gpart, status, s); break;
-        case 2: launch_g_t<2>(p, tmx, ehi, elo, T, nC, Gpart, status, s); break;
-        default: launch_g_t<3>(p, tmx, ehi, elo, T, nC, Gpart, status, s); break;
+        case 1: ok = launch_g_t<1>(p, tmx, ehi, elo, T, nC, Gpart, status, s); break;
+        case 2: ok = launch_g_t<2>(p, tmx, ehi, elo, T, nC, Gpart, status, s); break;
+        default: ok = launch_g_t<3>(p, tmx, ehi, elo, T, nC, Gpart, status, s); break;
     }
-    return true;
+    if (ok) c->launches += 1;
+    return ok;
 }
 
 size_t tail_wb_bytes(int n, int C, int Kp) { return (size_t)n * ((C + kDCh - 1) / kDCh) * Kp * kDCh * 2; }
