@@ -9,8 +9,9 @@ output y and its backward's du are inputs).  Rank r of an N-GPU run processes it
 tokens (weak scaling, no data-path collective).  Prints one JSON line on rank 0.
 
 The default workload is the largest single-GPU one (cfg5: n = 4, C = 4096, T = 131072).  On one GPU the
-line also carries a `workloads` table: cfg2, the 24-layer stack cfg3, cfg4a, cfg4b and the cfg5 token
-sweep, each with the mHC-lite step and the in-library SK-20 step timed the same way (CUDA-graph replay).
+line also carries a `workloads` table: cfg2, the 24-layer stack cfg3, cfg4a, cfg4b, the subset variant of the
+paper's Section 5 on the cfg4b shape (24 sampled permutations of 120) and the cfg5 token sweep, each with the
+mHC-lite step and (full tables) the in-library SK-20 step timed the same way (CUDA-graph replay).
 
 --impl reference times the fp64 CPU oracle on the host cores (rank 0 only) on a bounded sample.
 With --gpus N > 1 and no torchrun environment the script starts its own N ranks.
@@ -292,10 +293,13 @@ class Pool:
                 v(self.du, need_small, (T, C)))
 
 
-def time_layer_case(mods, timer, ctx, wl, T, kind, acts, dev, steps, min_total_ms, use_graph=True, fused=True):
-    """Times one single-layer workload (kind 'lite' or 'sk') on the given activations."""
+def time_layer_case(mods, timer, ctx, wl, T, kind, acts, dev, steps, min_total_ms, use_graph=True, fused=True,
+                    n_res=None):
+    """Times one single-layer workload (kind 'lite' or 'sk') on the given activations; n_res = K when the context
+    holds a subset of K permutations."""
     torch, L, synth = mods["torch"], mods["L"], mods["synth"]
-    p = synth.make_layer_params(wl.n, wl.C, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std, kind=kind)
+    p = synth.make_layer_params(wl.n, wl.C, wl.seed, bias_std=wl.bias_std, alpha=wl.alpha, w_std=wl.w_std, kind=kind,
+                                n_res=n_res)
     P = L.LayerParams(p["W"], p["b"], p["alpha"], p["gain"], dev)
     B = L.LayerBuffers(ctx, T, kind)
     x, y, g, du = acts
@@ -401,12 +405,16 @@ def run_ours(args, wl, rank, world):
     pool = Pool(torch, L, inp, dev, repeat=(T + T_draw - 1) // T_draw)
     ctxs = {}
 
-    def ctx_for(n_, C_):
-        if (n_, C_) not in ctxs:
-            ctxs[(n_, C_)] = MhcLite(n_, C_, local)
-        return ctxs[(n_, C_)]
+    def ctx_for(n_, C_, K_=None, seed_=0):
+        """One context per shape; K_: a context that holds a sampled subset of K_ permutations (paper Section 5)."""
+        if (n_, C_, K_) not in ctxs:
+            c_ = MhcLite(n_, C_, local)
+            if K_:
+                c_.set_perm_subset(torch.from_numpy(synth.sample_perm_table(n_, K_, seed_)).to(dev))
+            ctxs[(n_, C_, K_)] = c_
+        return ctxs[(n_, C_, K_)]
 
-    ctx = ctx_for(n, C)
+    ctx = ctx_for(n, C, args.permutations or None, wl.seed)
     timer = Timer(torch, D, world, dev)
     fused = not args.unfused
     steps = args.steps
@@ -440,7 +448,7 @@ def run_ours(args, wl, rank, world):
     sampler = ClockSampler(local) if rank == 0 else None
     # (the warm-up steps run inside time_layer_case: three plain, one counted, the capture, three replays)
     head, P, B, step, graph = time_layer_case(mods, timer, ctx, wl, T, "lite", acts, dev, steps, args.min_ms,
-                                              use_graph=not args.no_graph, fused=fused)
+                                              use_graph=not args.no_graph, fused=fused, n_res=args.permutations or None)
     clocks = sampler.stop() if sampler else None
     ms = head["ms_per_step"]
     launch_mode = head["launch"]
@@ -525,11 +533,26 @@ def run_ours(args, wl, rank, world):
         table = []
         del B, graph
         torch.cuda.empty_cache()
-        rows = [("cfg2", None), ("cfg3", None), ("cfg4a", None), ("cfg4b", None)] + \
-               [("cfg5", t) for t in (4096, 8192, 16384, 32768, 65536, 131072)]
-        for name, Tt in rows:
+        # (workload, T override, K): K = a sampled subset of K of the n! permutations (paper Section 5) on that shape
+        rows = [("cfg2", None, None), ("cfg3", None, None), ("cfg4a", None, None), ("cfg4b", None, None),
+                ("cfg4b", None, 24)] + [("cfg5", t, None) for t in (4096, 8192, 16384, 32768, 65536, 131072)]
+        for name, Tt, K in rows:
             w = synth.WORKLOADS[name]
             Tt = Tt or w.T
+            if K:
+                a = pool.views(Tt, w.n, w.C)
+                c = ctx_for(w.n, w.C, K, w.seed)
+                r, _, Bl, _, gr = time_layer_case(mods, timer, c, w, Tt, "lite", a, dev, steps, args.min_ms_table,
+                                                  not args.no_graph, n_res=K)
+                table.append({"workload": name, "n": w.n, "C": w.C, "T": Tt, "permutations": K,
+                              "ms_per_step": r["ms_per_step"], "ms_min": r["ms_min"], "ms_max": r["ms_max"],
+                              "repeats": r["repeats"], **rates(w.n, w.C, Tt, r["ms_per_step"], peak), "launch": r["launch"],
+                              "launches_per_step": r["launches_per_step"], "sk20": None,
+                              "note": "subset variant: Eq. (5) over %d sampled permutations of %d" % (K, math.factorial(w.n))})
+                del Bl, gr
+                c.device_status()
+                torch.cuda.empty_cache()
+                continue
             if name == wl.name and Tt == T:
                 row = {"workload": name, "n": n, "C": C, "T": T, "ms_per_step": ms, **rates(n, C, T, ms, peak),
                        "launch": launch_mode, "sk20": sk20, "note": "the headline row"}
@@ -589,6 +612,7 @@ def run_ours(args, wl, rank, world):
             "data": "synthetic" if world == 1 else f"synthetic ({T_draw} tokens drawn per rank, repeated to T)",
             "config": {"workload": wl.name, "n": n, "C": C, "T_per_gpu": T, "passes": "fwd+bwd" if wl.backward else "fwd",
                        "calls": "fused" if fused else "unfused", "launch": launch_mode, "note": wl.note,
+                       **({"permutations": args.permutations} if args.permutations else {}),
                        "l2": "inputs larger than L2 (working set %.0f MB)" % (total_bytes / 1e6)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": head["launches_per_step"] * steps * head["repeats"],
             "roofline": roofline, "cpu_baseline": cpu_baseline, "sk20_comparison": sk20, "workloads": table,
@@ -625,9 +649,14 @@ def main():
     ap.add_argument("--no-table", action="store_true", help="skip the table of the other workloads")
     ap.add_argument("--unfused", action="store_true", help="time the un-fused call sequence (six entry points)")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph of one step")
+    ap.add_argument("--permutations", type=int, default=0, metavar="K",
+                    help="headline on the subset variant (paper Section 5): K sampled permutations instead of n!; "
+                         "device-resident timing only")
     ap.add_argument("--traffic-from-ncu", default="", metavar="CSV",
                     help="no run: write profiles/dram_traffic_<workload>.txt from an ncu --csv log of one step at --T tokens")
     args = ap.parse_args()
+    if args.permutations:
+        args.no_e2e = args.no_cpu_baseline = args.no_sk = args.no_table = True
     if args.traffic_from_ncu:
         write_ncu_traffic(args.workload, args.T or synth.WORKLOADS[args.workload].T, args.traffic_from_ncu)
         return

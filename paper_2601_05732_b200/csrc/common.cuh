@@ -103,7 +103,7 @@ struct TailPlan {
     int Kp, KS;             // projection columns padded to 16, and Kp / 16
     int slices, splits;     // 64-channel slices x token ranges = the grid
     int64_t tok_per_split;  // multiple of 32
-    bool supported;         // KS <= 3 (N <= 48): the fused mma.sync kernel
+    bool supported;         // KS <= 3 (N <= 48) and n <= 4: the fused mma.sync kernel
     // wider projections: tcgen05 kernels (tail_tc.cu) when the shape allows, else the CUDA-core kernels
     bool tc;                // Kp <= 256 and rows of x a multiple of 16 bytes
     int g_mt;               // G kernel: 128-row accumulators per CTA (g_mt * Kp <= 512 tensor-memory columns)

@@ -341,7 +341,9 @@ TailPlan plan_tail(int n, int C, int64_t T, int N, int sm_count) {
     TailPlan p;
     p.Kp = round_up(N, 16);
     p.KS = p.Kp / 16;
-    p.supported = p.KS <= 3;
+    // n = 5 always takes the tcgen05 pair of tail_tc.cu, also with a narrow projection (a subset of the permutations):
+    // the fused tcgen05 kernel stops at n = 4, and the pair is about twice as fast as this file's mma.sync kernel
+    p.supported = p.KS <= 3 && n <= 4;
     p.slices = (C + kCS - 1) / kCS;
     if (sm_count > 148) sm_count = 148;                       // the workspace is sized for at most 2 x 148 CTAs
     int64_t splits = (2 * sm_count) / p.slices;
