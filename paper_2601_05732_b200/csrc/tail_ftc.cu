@@ -173,7 +173,10 @@ tail_ftc_k(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUte
                         tma_load_2d(smem_u32(slots + sl * kSlot) + b * kFBox, mp, full, col, row);
                         // the quadrant's next boxes start their way from HBM to L2 now: a slot is busy for a
                         // whole load + compute + store round, too long to hide the HBM latency with so few slots
-                        if (ti + 1 < nt) tma_prefetch_2d(mp, col, next_row);
+                        // (every other tile only: the tensor maps promote L2 fills to 256 bytes, so the neighbouring
+                        //  slice's CTA, which walks the same tiles at the same time, brings this slice's lines along
+                        //  on the tiles in between; a prefetch costs the TMA unit as much as the load itself)
+                        if (ti + 1 < nt && (((ti + (int)blockIdx.x) & 1) == 0)) tma_prefetch_2d(mp, col, next_row);
                     }
                 }
             }
