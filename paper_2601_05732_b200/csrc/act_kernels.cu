@@ -721,10 +721,16 @@ __global__ void __launch_bounds__(256, 4) lite_tailpre_w_k(
         float sdb = 0.f, sdal = 0.f;
 #pragma unroll
         for (int k = 0; k < 8; ++k) { sdb += red[0][k][lane]; sdal += red[1][k][lane]; }
-        if (c < D::kN) atomicAdd(db + c, sdb);
         const float s_res = warp_sum(is_res ? sdal : 0.f), s_pre = warp_sum(is_pre ? sdal : 0.f),
                     s_post = warp_sum(is_post ? sdal : 0.f);
-        if (lane == 0) { atomicAdd(dalpha, s_res); atomicAdd(dalpha + 1, s_pre); atomicAdd(dalpha + 2, s_post); }
+        if (dalpha) {
+            if (c < D::kN) atomicAdd(db + c, sdb);
+            if (lane == 0) { atomicAdd(dalpha, s_res); atomicAdd(dalpha + 1, s_pre); atomicAdd(dalpha + 2, s_post); }
+        } else {                                           // per-block partials, summed by tail_finish_k
+            float* part = db + (int64_t)blockIdx.x * kPartStride;
+            if (c < D::kN) part[c] = sdb;
+            if (lane == 0) { part[D::kN] = s_res; part[D::kN + 1] = s_pre; part[D::kN + 2] = s_post; }
+        }
     }
 }
 
@@ -1081,7 +1087,9 @@ __global__ void __launch_bounds__(kActThreads, 3) sk_tailpre_k(
         __syncthreads();
     }
     for (int c = tid; c < N + 3; c += kActThreads) {
-        if (c < N) atomicAdd(db + c, red[c]); else atomicAdd(dalpha + (c - N), red[c]);
+        if (!dalpha) db[(int64_t)blockIdx.x * kPartStride + c] = red[c];      // per-block partials (tail_finish_k adds them)
+        else if (c < N) atomicAdd(db + c, red[c]);
+        else atomicAdd(dalpha + (c - N), red[c]);
     }
 }
 
@@ -1154,10 +1162,12 @@ void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp,
 #undef MHCL_AP_T
 }
 
-void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const void* du, const float* a, const float* p,
-                         const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
-                         const float* dH_res, const float* dH_post, float* dH_pre_ws, float* e, int Npad, void* ehi,
-                         void* elo, int Kp, float* kappa, float* db, float* dalpha, cudaStream_t s) {
+// Returns the number of blocks launched (= partials written when dalpha is null; only the n <= 4 kernel of a context
+// without a permutation subset writes partials).
+int launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const void* du, const float* a, const float* p,
+                        const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
+                        const float* dH_res, const float* dH_post, float* dH_pre_ws, float* e, int Npad, void* ehi,
+                        void* elo, int Kp, float* kappa, float* db, float* dalpha, cudaStream_t s) {
     c->launches += 1;
     KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_PRE, s);
     const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
@@ -1185,6 +1195,7 @@ void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const v
     }
 #undef MHCL_TP_W
 #undef MHCL_TP_T
+    return blocks;
 }
 
 void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,
@@ -1227,10 +1238,10 @@ void launch_sk_act_premix(const mhclite_ctx* c, int64_t T, int iters, const Proj
                                                                           (const uint4*)x, (uint4*)u));
 }
 
-void launch_sk_tailpre(const mhclite_ctx* c, int64_t T, int iters, const void* x, const void* du, const float* p,
-                       const float* b, const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
-                       const float* dH_res, const float* dH_post, float* e, int Npad, void* ehi, void* elo, int Kp,
-                       float* kappa, float* db, float* dalpha, cudaStream_t s) {
+int launch_sk_tailpre(const mhclite_ctx* c, int64_t T, int iters, const void* x, const void* du, const float* p,
+                      const float* b, const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
+                      const float* dH_res, const float* dH_post, float* e, int Npad, void* ehi, void* elo, int Kp,
+                      float* kappa, float* db, float* dalpha, cudaStream_t s) {
     c->launches += 1;
     KernelTimer timer_(c, MHCLITE_KERNEL_TAIL_PRE, s);
     const EOut eo{e, Npad, (__nv_bfloat16*)ehi, (__nv_bfloat16*)elo, Kp};
@@ -1241,6 +1252,7 @@ void launch_sk_tailpre(const mhclite_ctx* c, int64_t T, int iters, const void* x
     MHCL_DISPATCH_N(c->n, sk_tailpre_k<N_><<<grid, kActThreads, 0, s>>>(T, C8, iters, inv, (const uint4*)x, (const uint4*)du, p,
                                                                        b, rstd, alpha, H_pre, H_post, dH_res, dH_post, eo,
                                                                        kappa, db, dalpha));
+    return grid;
 }
 
 }  // namespace mhcl

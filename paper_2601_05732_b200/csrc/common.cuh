@@ -53,6 +53,12 @@ inline int64_t round_up64(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 //   element (t, c)  ->  ((t / 128) * (Kp / 8) + c / 8) * 1024 + (t % 128) * 8 + c % 8.
 // A granule is then a ready-made shared-memory operand without swizzle (8 x 16-byte core matrices) both
 // with tokens as the M dimension and columns as K, and with columns as N and tokens as K.
+// db / dalpha as per-block partials (deterministic, and nothing has to be cleared first): a kernel that gets a null
+// dalpha writes its block's sums to db[block * kPartStride + c], c < N for db and N..N+2 for dalpha; tail_finish_k
+// adds the blocks up in a fixed order.
+constexpr int kPartStride = 136;
+constexpr int kMaxParts = 148 * 16;
+
 constexpr int kEGranule = 128;
 __host__ __device__ inline int64_t e_tiled_index(int Kp, int64_t t, int c) {
     return ((t >> 7) * (Kp >> 3) + (c >> 3)) * 1024 + (t & 127) * 8 + (c & 7);
@@ -129,6 +135,7 @@ struct Workspace {
     float* Gpart;    // [splits or g_splits][nC][Kp] partial G of each token range
     void* Wb;        // bf16 W' blocks of the tcgen05 dx kernels
     void* Wt;        // [2 nq][Kpad] bf16: W' hi rows then lo rows, K-major (tcgen05 projection)
+    float* dpart;    // [kMaxParts][kPartStride] per-block partials of db and dalpha
     int* status;     // device status word (0, or a negative mhclite_status raised by a kernel)
     size_t bytes;
     int Npad;

@@ -54,8 +54,13 @@ bool launch_tail_ftc(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, 
                      const void* du, const void* ehi, const void* elo, const float* kappa, const float* H_res,
                      const float* H_pre, const float* W, const float* gain, void* Wf, bool wf_packed, void* dx,
                      int acc_dx, float* Gpart, int* status, cudaStream_t s);
+// db[N], dalpha[3] (+)= the nparts per-block partials alone (for a backward that does not end in launch_tail_finish)
+void launch_dpart_sum(const mhclite_ctx* c, int N, const float* dpart, int nparts, float* db, float* dalpha, int acc_params,
+                      cudaStream_t s);
+// dpart (null: none): nparts per-block partials of db / dalpha, added up into db[N], dalpha[3] by the same launch
 void launch_tail_finish(const mhclite_ctx* c, int N, int Kp, int splits, const float* W, const float* gain,
-                        const float* Gpart, float* dW, float* dgain, int acc_params, cudaStream_t s);
+                        const float* Gpart, float* dW, float* dgain, int acc_params, cudaStream_t s,
+                        const float* dpart = nullptr, int nparts = 0, float* db = nullptr, float* dalpha = nullptr);
 bool proj_tc_supported(int n, int C, int N);
 int proj_tc_nq(int N);
 void launch_pack_wt(const mhclite_ctx* c, const ProjPlan& p, int N, const float* W, const float* gain, void* Wt,
@@ -81,18 +86,18 @@ void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float*
 void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, const float* qpart, const float* ssq,
                             float eps, const float* b, const float* alpha, float* H_res, float* H_pre, float* H_post,
                             float* a_saved, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s);
-void launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const void* du, const float* a, const float* p,
-                         const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
-                         const float* dH_res, const float* dH_post, float* dH_pre_ws, float* e, int Npad, void* ehi,
-                         void* elo, int Kp, float* kappa, float* db, float* dalpha, cudaStream_t s);
+int launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const void* du, const float* a, const float* p,
+                        const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
+                        const float* dH_res, const float* dH_post, float* dH_pre_ws, float* e, int Npad, void* ehi,
+                        void* elo, int Kp, float* kappa, float* db, float* dalpha, cudaStream_t s);
 // the SK path's counterparts of the two fused kernels above
 void launch_sk_act_premix(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,
                           const float* ssq, float eps, const float* b, const float* alpha, float* H_res, float* H_pre,
                           float* H_post, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s);
-void launch_sk_tailpre(const mhclite_ctx* c, int64_t T, int iters, const void* x, const void* du, const float* p,
-                       const float* b, const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
-                       const float* dH_res, const float* dH_post, float* e, int Npad, void* ehi, void* elo, int Kp,
-                       float* kappa, float* db, float* dalpha, cudaStream_t s);
+int launch_sk_tailpre(const mhclite_ctx* c, int64_t T, int iters, const void* x, const void* du, const float* p,
+                      const float* b, const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
+                      const float* dH_res, const float* dH_post, float* e, int Npad, void* ehi, void* elo, int Kp,
+                      float* kappa, float* db, float* dalpha, cudaStream_t s);
 void launch_sk_act_fwd(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,
                        const float* ssq, float eps, const float* b, const float* alpha, float* H_res, float* H_pre,
                        float* H_post, float* p_saved, float* rstd, cudaStream_t s);

@@ -46,6 +46,7 @@ Workspace plan_workspace(int n, int C, int64_t T, int N, void* base, int sm_coun
     w.Gpart = (float*)(p + off); off += align256((size_t)gparts * n * C * tp.Kp * sizeof(float));
     w.Wt = p + off;              off += align256((size_t)2 * proj_tc_nq(N) * pp.nchunks * 64 * 2);
     w.Wb = p + off;              off += align256((tp.tc || tp.ftc) ? tail_wb_bytes(n, C, tp.Kp) : 0);
+    w.dpart = (float*)(p + off); off += align256((size_t)kMaxParts * kPartStride * sizeof(float));
     w.status = (int*)(p + off);  off += 256;
     w.bytes = off;
     return w;
@@ -136,14 +137,21 @@ static bool tail_pair(const TailPlan& tp) { return tp.supported || (tp.tc && ten
 static int proj_backward(mhclite_ctx* ctx, int64_t T, int N, const Workspace& w, const TailPlan& tp,
                          const mhclite_bf16* x, const mhclite_bf16* g, const mhclite_bf16* du, const float* H_res,
                          const float* H_pre, const float* W, const float* gain, bool wf_packed, mhclite_bf16* dx,
-                         int accumulate_dx, float* dW, float* dgain, int accumulate_params, cudaStream_t s) {
+                         int accumulate_dx, float* dW, float* dgain, int accumulate_params, cudaStream_t s,
+                         const float* dpart = nullptr, int nparts = 0, float* db = nullptr, float* dalpha = nullptr) {
+    // dpart: db and dalpha were left as nparts per-block partials by the activation backward
     if (tp.ftc && launch_tail_ftc(ctx, T, N, tp, x, g, du, w.ehi, w.elo, w.kappa, H_res, H_pre, W, gain, w.Wb, wf_packed,
                                   dx, accumulate_dx, w.Gpart, w.status, s)) {
         MHCL_LAUNCH_CHECK(ctx, "tail_ftc");
         ctx->launches += 1;
-        launch_tail_finish(ctx, N, tp.Kp, tp.f_splits, W, gain, w.Gpart, dW, dgain, accumulate_params, s);
+        launch_tail_finish(ctx, N, tp.Kp, tp.f_splits, W, gain, w.Gpart, dW, dgain, accumulate_params, s, dpart, nparts, db,
+                           dalpha);
         MHCL_LAUNCH_CHECK(ctx, "tail_finish");
         return MHCLITE_OK;
+    }
+    if (dpart) {
+        launch_dpart_sum(ctx, N, dpart, nparts, db, dalpha, accumulate_params, s);
+        MHCL_LAUNCH_CHECK(ctx, "dpart_sum");
     }
     if (tp.supported) {
         launch_tail_mma(ctx, T, N, tp, x, g, du, w.ehi, w.elo, w.kappa, H_res, H_pre, W, gain, dx, accumulate_dx,
@@ -468,6 +476,16 @@ int mhclite_premix_bwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const
     return MHCLITE_OK;
 }
 
+// The fused backward tails that end in tail_ftc_k leave db and dalpha as per-block partials in their first kernel
+// (dH_pre + activation backward); tail_finish_k adds them up in a fixed order.  Nothing has to be cleared first,
+// and the sums do not depend on the order in which blocks finish.  True when that route is open: W' has then been
+// packed for tail_ftc_k.  (Packing on a second stream while the first kernel runs was measured: no gain.)
+static bool part_pack(mhclite_ctx* ctx, int N, const TailPlan& tp, const Workspace& w, const float* W, const float* gain,
+                      cudaStream_t s) {
+    if (!tp.ftc || !tensor_maps_available() || ctx->sm_count * 16 > kMaxParts) return false;
+    return launch_tail_ftc_prep(ctx, N, tp, W, gain, w.Wb, nullptr, nullptr, s);
+}
+
 // Zeroes the parameter-gradient accumulators that the kernels add into, unless the caller accumulates.  When
 // the backward ends in the fused tcgen05 tail, the kernel that packs W' for it does the zeroing as well
 // (*wf_packed tells proj_backward that W' is ready).
@@ -533,13 +551,20 @@ int mhclite_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, c
     const int N = ctx_cols(ctx, 0);
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
     bool wf_packed = false;
-    rc = prep_param_grads(ctx, N, tp, w, W, gain, db, dalpha, accumulate_params, s, &wf_packed);
-    if (rc) return rc;
-    launch_lite_tailpre(ctx, T, x, du, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_post, w.dH_pre,
-                        tp.supported ? nullptr : w.e, w.Npad, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db,
-                        dalpha, s);
+    // (the partials are written by the n <= 4 kernel of a context without a permutation subset)
+    const bool part = ctx->n <= 4 && !ctx->table_dev && part_pack(ctx, N, tp, w, W, gain, s);
+    if (part) {
+        wf_packed = true;
+    } else {
+        rc = prep_param_grads(ctx, N, tp, w, W, gain, db, dalpha, accumulate_params, s, &wf_packed);
+        if (rc) return rc;
+    }
+    const int nparts = launch_lite_tailpre(ctx, T, x, du, a_saved, p_saved, rstd, alpha, H_pre, H_post, dH_res, dH_post,
+                                           w.dH_pre, tp.supported ? nullptr : w.e, w.Npad, tail_pair(tp) ? w.ehi : nullptr,
+                                           w.elo, tp.Kp, w.kappa, part ? w.dpart : db, part ? nullptr : dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "lite_tailpre");
-    return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W, gain, wf_packed, dx, 0, dW, dgain, accumulate_params, s);
+    return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W, gain, wf_packed, dx, 0, dW, dgain, accumulate_params, s,
+                         part ? w.dpart : nullptr, nparts, db, dalpha);
 }
 
 // ---- SK comparison path --------------------------------------------------------------------------
@@ -642,13 +667,19 @@ int mhc_sk20_tail_bwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, 
     const int N = ctx_cols(ctx, 1);
     const TailPlan tp = plan_tail(ctx->n, ctx->C, T, N, ctx->sm_count);
     bool wf_packed = false;
-    rc = prep_param_grads(ctx, N, tp, w, W_sk, gain, db, dalpha, accumulate_params, s, &wf_packed);
-    if (rc) return rc;
-    launch_sk_tailpre(ctx, T, iters, x, du, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, dH_post,
-                      tp.supported ? nullptr : w.e, w.Npad, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp, w.kappa, db,
-                      dalpha, s);
+    const bool part = part_pack(ctx, N, tp, w, W_sk, gain, s);
+    if (part) {
+        wf_packed = true;
+    } else {
+        rc = prep_param_grads(ctx, N, tp, w, W_sk, gain, db, dalpha, accumulate_params, s, &wf_packed);
+        if (rc) return rc;
+    }
+    const int nparts = launch_sk_tailpre(ctx, T, iters, x, du, p_saved, b_sk, rstd, alpha, H_pre, H_post, dH_res, dH_post,
+                                         tp.supported ? nullptr : w.e, w.Npad, tail_pair(tp) ? w.ehi : nullptr, w.elo, tp.Kp,
+                                         w.kappa, part ? w.dpart : db, part ? nullptr : dalpha, s);
     MHCL_LAUNCH_CHECK(ctx, "sk_tailpre");
-    return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W_sk, gain, wf_packed, dx, 0, dW, dgain, accumulate_params, s);
+    return proj_backward(ctx, T, N, w, tp, x, g, du, H_res, H_pre, W_sk, gain, wf_packed, dx, 0, dW, dgain, accumulate_params, s,
+                         part ? w.dpart : nullptr, nparts, db, dalpha);
 }
 
 int mhclite_ds_gap(mhclite_ctx* ctx, int64_t T, const float* H_res, float* l1_err, float* colsum_dev, void* stream) {

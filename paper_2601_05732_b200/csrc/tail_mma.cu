@@ -312,9 +312,20 @@ __global__ void __launch_bounds__(256, 2) tail_mma_k(const TailArgs a) {
 template <bool ACC>
 __global__ void __launch_bounds__(256) tail_finish_k(int nC, int N, int Kp, int splits, const float* __restrict__ W,
                                                      const float* __restrict__ gain, const float* __restrict__ Gpart,
-                                                     float* dW, float* dgain) {
+                                                     float* dW, float* dgain, const float* __restrict__ dpart, int nparts,
+                                                     float* db, float* dalpha) {
     const int lane = threadIdx.x & 31;
     const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
+    // the first warps also add up the per-block partials of db and dalpha, one column each, in a fixed order
+    if (dpart && m < N + 3) {
+        float v = 0.f;
+        for (int p0 = lane; p0 < nparts; p0 += 32) v += __ldg(dpart + (int64_t)p0 * kPartStride + m);
+        v = warp_sum(v);
+        if (lane == 0) {
+            float* dst = m < N ? db + m : dalpha + (m - N);
+            *dst = ACC ? *dst + v : v;
+        }
+    }
     if (m >= nC) return;
     const float gm = __ldg(gain + m);
     float dg = 0.f;
@@ -336,7 +347,29 @@ __global__ void __launch_bounds__(256) tail_finish_k(int nC, int N, int Kp, int 
     if (lane == 0) dgain[m] = ACC ? dgain[m] + dg : dg;
 }
 
+template <bool ACC>
+__global__ void __launch_bounds__(256) dpart_sum_k(int N, const float* __restrict__ dpart, int nparts, float* db, float* dalpha) {
+    const int lane = threadIdx.x & 31;
+    const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (m >= N + 3) return;
+    float v = 0.f;
+    for (int p0 = lane; p0 < nparts; p0 += 32) v += __ldg(dpart + (int64_t)p0 * kPartStride + m);
+    v = warp_sum(v);
+    if (lane == 0) {
+        float* dst = m < N ? db + m : dalpha + (m - N);
+        *dst = ACC ? *dst + v : v;
+    }
+}
+
 // ---- host side -------------------------------------------------------------------------------------
+void launch_dpart_sum(const mhclite_ctx* c, int N, const float* dpart, int nparts, float* db, float* dalpha, int acc_params,
+                      cudaStream_t s) {
+    c->launches += 1;
+    const int grid = (N + 3 + 7) / 8;
+    if (acc_params) dpart_sum_k<true><<<grid, 256, 0, s>>>(N, dpart, nparts, db, dalpha);
+    else dpart_sum_k<false><<<grid, 256, 0, s>>>(N, dpart, nparts, db, dalpha);
+}
+
 TailPlan plan_tail(int n, int C, int64_t T, int N, int sm_count) {
     TailPlan p;
     p.Kp = round_up(N, 16);
@@ -415,11 +448,13 @@ void launch_tail_mma(const mhclite_ctx* c, int64_t T, int N, const TailPlan& p, 
 
 // Counted by the caller.
 void launch_tail_finish(const mhclite_ctx* c, int N, int Kp, int splits, const float* W, const float* gain,
-                        const float* Gpart, float* dW, float* dgain, int acc_params, cudaStream_t s) {
+                        const float* Gpart, float* dW, float* dgain, int acc_params, cudaStream_t s, const float* dpart,
+                        int nparts, float* db, float* dalpha) {
     const int nC = c->n * c->C;
-    const int fg = (nC + 7) / 8;
-    if (acc_params) tail_finish_k<true><<<fg, 256, 0, s>>>(nC, N, Kp, splits, W, gain, Gpart, dW, dgain);
-    else tail_finish_k<false><<<fg, 256, 0, s>>>(nC, N, Kp, splits, W, gain, Gpart, dW, dgain);
+    int fg = (nC + 7) / 8;
+    if (dpart && fg < (N + 3 + 7) / 8) fg = (N + 3 + 7) / 8;
+    if (acc_params) tail_finish_k<true><<<fg, 256, 0, s>>>(nC, N, Kp, splits, W, gain, Gpart, dW, dgain, dpart, nparts, db, dalpha);
+    else tail_finish_k<false><<<fg, 256, 0, s>>>(nC, N, Kp, splits, W, gain, Gpart, dW, dgain, dpart, nparts, db, dalpha);
 }
 
 }  // namespace mhcl

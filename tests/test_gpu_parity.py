@@ -340,3 +340,58 @@ def test_gap_statistics_and_relative_range_histogram():
     assert h.sum() == T and h[bins] == 1
     # a value within rounding of a bin edge may fall either side: compare cumulative counts with a slack of a few
     assert np.abs(np.cumsum(h) - np.cumsum(expect)).max() <= 3
+
+
+@pytest.mark.parametrize("kind", ["lite", "sk"])
+def test_fused_tail_partials_accumulate_and_survive_a_graph(kind):
+    """The fused backward tail on the tcgen05 path sums db / dalpha from per-block partials in a fixed order (no
+    atomics on the lite path, nothing cleared beforehand): two runs give the same db, dalpha and dx bit for
+    bit (dW and dgain agree to rounding: the order in which tensor memory accumulates a tile's four token quadrants
+    follows the arrival of their data), an accumulating call doubles the parameter gradients, and the call sequence can
+    be captured in a CUDA graph and replayed."""
+    n, C, T = 4, 512, 1500
+    inp = synth.make_layer_inputs(n, C, T, seed=77, bias_std=0.1, gain_std=0.1, kind=kind)
+    G = GpuLayer(inp, kind=kind)
+    G.forward(True)
+    G.backward(True)
+    torch.cuda.synchronize()
+    names = ("db", "dalpha", "dW", "dgain", "dx")
+    first = {k: getattr(G.B, k).clone() for k in names}
+    ref = oracle_bwd(inp, kind=kind)
+    check_f32(f"{kind} db from partials", host(first["db"]), ref["db"], 1e-3)
+    check_f32(f"{kind} dalpha from partials", host(first["dalpha"]), ref["dalpha"], 1e-3)
+    exact = ("db", "dalpha", "dx") if kind == "lite" else ("dx",)      # the SK kernel adds within a block by atomics
+
+    def same_as_first(what):
+        for k, v in first.items():
+            got = getattr(G.B, k)
+            if k in exact:
+                assert torch.equal(got, v), f"{k} differs {what}"
+            else:
+                scale = v.float().pow(2).mean().sqrt()
+                assert (got.float() - v.float()).abs().max() <= 1e-5 * scale, f"{k} differs {what}"
+
+    G.backward(True)
+    torch.cuda.synchronize()
+    same_as_first("between two runs")
+    G.backward(True, accumulate_params=True)
+    torch.cuda.synchronize()
+    for k in ("db", "dalpha", "dW", "dgain"):
+        v = first[k]
+        scale = v.float().pow(2).mean().sqrt()
+        assert (getattr(G.B, k) - 2 * v).abs().max() <= 2e-5 * scale, f"{k} is not doubled by an accumulating call"
+    # capture and replay
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        G.backward(True)
+        st.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=st):
+            L.post_bwd(G.ctx, G.B, G.x, G.y, G.g, True)
+            L.tail_bwd(G.ctx, G.P, G.B, G.x, G.g, G.du, G.eps, True, G.iters, False)
+        for k in names:
+            getattr(G.B, k).zero_()
+        graph.replay()
+        st.synchronize()
+    same_as_first("after a graph replay")
+    G.ctx.device_status()
