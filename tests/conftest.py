@@ -31,7 +31,8 @@ def pytest_collection_modifyitems(config, items):
 
 def pytest_sessionfinish(session, exitstatus):
     """Writes the raw error figures that the parity helpers collected (one JSON object per comparison) to
-    gpurun_out/parity_errors.jsonl at the repository root; tests/parity_report.py turns them into a table."""
+    parity_errors.jsonl in the report folder (PARITY_REPORT_DIR, default parity_report/ at the repository root);
+    tests/parity_report.py turns them into a table."""
     try:
         import json
         import parity_utils
@@ -39,7 +40,7 @@ def pytest_sessionfinish(session, exitstatus):
         return
     if not parity_utils.RECORDS:
         return
-    out = os.path.join(ROOT, "gpurun_out")
+    out = os.environ.get("PARITY_REPORT_DIR") or os.path.join(ROOT, "parity_report")
     os.makedirs(out, exist_ok=True)
     with open(os.path.join(out, "parity_errors.jsonl"), "w") as f:
         for r in parity_utils.RECORDS:

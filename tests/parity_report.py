@@ -1,4 +1,5 @@
-"""Summarises gpurun_out/parity_errors.jsonl (written by a `-m gpu` test session) as a markdown table:
+"""Summarises parity_errors.jsonl (written by a `-m gpu` test session into PARITY_REPORT_DIR, default parity_report/
+at the repository root) as a markdown table:
 per tensor, the worst raw figures over all comparisons of that tensor in the chosen tests.
 
     python tests/parity_report.py [substring of the test id ...]
@@ -12,7 +13,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def main(argv):
-    path = os.path.join(ROOT, "gpurun_out", "parity_errors.jsonl")
+    path = os.path.join(os.environ.get("PARITY_REPORT_DIR") or os.path.join(ROOT, "parity_report"), "parity_errors.jsonl")
     recs = [json.loads(l) for l in open(path)]
     if argv:
         recs = [r for r in recs if any(a in r["test"] for a in argv)]
