@@ -197,7 +197,10 @@ __global__ void __launch_bounds__(kActThreads) lite_act_fwd_k(int64_t T, int n, 
 //      (one round of coalesced loads, so the per-token math below waits on no global load);
 //   A: one warp per token: gates, softmax, H_res;
 //   P: all threads stream the group's tokens: u[t,:] = sum_j H_pre[t,j] x[t,j,:]   (Eq. (1), inner term).
-constexpr int kGroupTok = 32;
+// Eight tokens (one per warp) and a grid of resident blocks only: a block then walks many groups, so that the blocks of
+// an SM drift apart and one block's mappings run under the others' streaming.  (With 32-token groups and one or two
+// groups per block, all blocks of a wave went through their phases together and HBM idled during L and A.)
+constexpr int kGroupTok = 8;
 
 template <int N_>
 __global__ void __launch_bounds__(kActThreads, 4) lite_act_premix_k(
@@ -248,23 +251,41 @@ __global__ void __launch_bounds__(kActThreads, 4) lite_act_premix_k(
             if (lane < N_) hg[tl][lane] = gate;
         }
         __syncthreads();
-        // P
-        for (int i = tid; i < nt * C8; i += kActThreads) {
-            const int tl = i / C8, cv = i - tl * C8;
-            const int64_t t = t0 + tl;
-            uint4 v[N_];
+        // P (two vectors per thread in flight: the loads of the second are issued before the first is used)
+        for (int i0 = tid; i0 < nt * C8; i0 += 2 * kActThreads) {
+            const int i1 = i0 + kActThreads;
+            const bool has1 = i1 < nt * C8;
+            const int tl0 = i0 / C8, cv0 = i0 - tl0 * C8;
+            const int tl1 = has1 ? i1 / C8 : tl0, cv1 = has1 ? i1 - tl1 * C8 : cv0;
+            uint4 v0[N_], v1[N_];
 #pragma unroll
-            for (int j = 0; j < N_; ++j) v[j] = ld_stream(x + (t * N_ + j) * C8 + cv);
-            float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            for (int j = 0; j < N_; ++j) v0[j] = ld_stream(x + ((t0 + tl0) * N_ + j) * C8 + cv0);
 #pragma unroll
-            for (int j = 0; j < N_; ++j) {
-                const float h = hg[tl][j];
-                float f[8];
-                unpack8(v[j], f);
+            for (int j = 0; j < N_; ++j) v1[j] = ld_stream(x + ((t0 + tl1) * N_ + j) * C8 + cv1);
+            {
+                float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] = fmaf(h, f[e], acc[e]);
+                for (int j = 0; j < N_; ++j) {
+                    const float h = hg[tl0][j];
+                    float f[8];
+                    unpack8(v0[j], f);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[e] = fmaf(h, f[e], acc[e]);
+                }
+                st_stream(u + (t0 + tl0) * C8 + cv0, pack8(acc));
             }
-            st_stream(u + t * C8 + cv, pack8(acc));
+            if (has1) {
+                float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+                for (int j = 0; j < N_; ++j) {
+                    const float h = hg[tl1][j];
+                    float f[8];
+                    unpack8(v1[j], f);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[e] = fmaf(h, f[e], acc[e]);
+                }
+                st_stream(u + (t0 + tl1) * C8 + cv1, pack8(acc));
+            }
         }
         __syncthreads();
     }
@@ -385,7 +406,7 @@ __global__ void __launch_bounds__(kActThreads, 4) lite_tailpre_k(
     constexpr int NN = N_ * N_;
     constexpr int kFact = (N_ == 2) ? 2 : (N_ == 3) ? 6 : (N_ == 4) ? 24 : 120;
     constexpr int kStride = kFact + (kFact + 2 * N_) + NN + 3 * N_ + 1 + 1;
-    constexpr int kGroupTok = (N_ == 5) ? 16 : 32;              // keeps the staging under the static shared-memory limit
+    constexpr int kGroupTok = 8;                               // one token per warp; see lite_act_premix_k
     __shared__ float in_s[kGroupTok][kStride];
     __shared__ float dhp_s[kGroupTok][kMaxN];
     load_tables(sh, N_, nf, table);
@@ -1101,6 +1122,12 @@ static int warp_grid(int64_t T, int sm_count) {
     return (int)(blocks < 1 ? 1 : blocks);
 }
 
+// One block per group, at most `resident` of them (the blocks that fit the GPU at once).
+static int resident_grid(int64_t T, int group, int resident) {
+    const int64_t blocks = (T + group - 1) / group;
+    return (int)(blocks < 1 ? 1 : (blocks > resident ? resident : blocks));
+}
+
 static int group_grid(int64_t T, int group, int sm_count) {
     int64_t blocks = (T + group - 1) / group;
     const int64_t cap = (int64_t)sm_count * 16;
@@ -1145,7 +1172,7 @@ void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp,
         (const uint4*)x, (uint4*)u)
     // one warp per token: n = 5 (120 logits do not fit a thread's registers) and every context that holds a
     // subset of the permutations (its table is data, not a compile-time constant)
-#define MHCL_AP_W(N_) lite_act_premix_k<N_><<<group_grid(T, kGroupTok, c->sm_count), kActThreads, 0, s>>>( \
+#define MHCL_AP_W(N_) lite_act_premix_k<N_><<<resident_grid(T, kGroupTok, c->sm_count * 4), kActThreads, 0, s>>>( \
         T, C8, c->nfact, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b, alpha, H_res, H_pre, H_post, a_saved, \
         p_saved, rstd, (const uint4*)x, (uint4*)u, c->table_dev)
     if (c->table_dev) {
@@ -1180,7 +1207,7 @@ int launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const vo
 #define MHCL_TP_T(N_) lite_tailpre_w_k<N_><<<blocks, 256, 0, s>>>( \
         T, C8, inv, (const uint4*)x, (const uint4*)du, a, p, rstd, alpha, H_pre, H_post, dH_res, dH_post, eo, kappa, \
         db, dalpha)
-#define MHCL_TP_W(N_) lite_tailpre_k<N_><<<group_grid(T, (N_ == 5) ? 16 : 32, c->sm_count), kActThreads, 0, s>>>( \
+#define MHCL_TP_W(N_) lite_tailpre_k<N_><<<resident_grid(T, 8, c->sm_count * 4), kActThreads, 0, s>>>( \
         T, C8, c->nfact, inv, (const uint4*)x, (const uint4*)du, a, p, rstd, alpha, H_pre, H_post, dH_res, \
         dH_post, eo, kappa, db, dalpha, c->table_dev)
     if (c->table_dev) {
