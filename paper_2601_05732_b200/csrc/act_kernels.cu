@@ -544,28 +544,30 @@ __device__ __forceinline__ void lite_thread_fwd(const float* prow, float* orow, 
 
 constexpr int kTokGroup = 32;    // tokens per block iteration of the thread-per-token kernels
 
-template <int N_>
+template <int N_, int GT>
 __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
     int64_t T, int C8, int Npad, int ksplit, float inv_nC, float eps, const float* __restrict__ qpart,
     const float* __restrict__ ssq, const float* __restrict__ b, const float* __restrict__ alpha,
     float* __restrict__ H_res, float* __restrict__ H_pre, float* __restrict__ H_post, float* __restrict__ a_saved,
     float* __restrict__ p_saved, float* __restrict__ rstd, const uint4* __restrict__ x, uint4* __restrict__ u) {
+    // GT <= kTokGroup tokens per group: small when there are few tokens, so that every block walks several groups
+    constexpr int gtok = GT;
     using D = LiteDims<N_>;
     __shared__ uint8_t klist_s[D::kNN * D::kPer];
     __shared__ float b_s[D::kN];
-    __shared__ float pg[kTokGroup][D::kN + 1];
-    __shared__ float og[kTokGroup][D::kOut + 1];
-    __shared__ float rg[kTokGroup];
+    __shared__ float pg[GT][D::kN + 1];
+    __shared__ float og[GT][D::kOut + 1];
+    __shared__ float rg[GT];
     const int tid = threadIdx.x;
     for (int i = tid; i < D::kNN * D::kPer; i += kActThreads) klist_s[i] = c_perm[N_].klist[i];
     for (int i = tid; i < D::kN; i += kActThreads) b_s[i] = __ldg(b + i);
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
     __syncthreads();
-    const int64_t ngroups = (T + kTokGroup - 1) / kTokGroup;
+    const int64_t ngroups = (T + gtok - 1) / gtok;
     for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
         // descending: the projection kernel before this one read x in ascending order and left its last lines in L2
-        const int64_t t0 = (ngroups - 1 - grp) * kTokGroup;
-        const int nt = (T - t0 < kTokGroup) ? (int)(T - t0) : kTokGroup;
+        const int64_t t0 = (ngroups - 1 - grp) * gtok;
+        const int nt = (T - t0 < gtok) ? (int)(T - t0) : gtok;
         // L: partials -> normalised projection rows in shared memory (and p_saved, rstd)
         if (tid < nt) {
             float ss = 0.f;
@@ -574,9 +576,9 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
             rg[tid] = r;
             rstd[t0 + tid] = r;
         }
-        float qv[(kTokGroup * D::kN + kActThreads - 1) / kActThreads];
+        float qv[(GT * D::kN + kActThreads - 1) / kActThreads];
 #pragma unroll
-        for (int it = 0; it < (kTokGroup * D::kN + kActThreads - 1) / kActThreads; ++it) {
+        for (int it = 0; it < (GT * D::kN + kActThreads - 1) / kActThreads; ++it) {
             const int i = tid + it * kActThreads;
             qv[it] = 0.f;
             if (i < nt * D::kN) {
@@ -586,7 +588,7 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
         }
         __syncthreads();
 #pragma unroll
-        for (int it = 0; it < (kTokGroup * D::kN + kActThreads - 1) / kActThreads; ++it) {
+        for (int it = 0; it < (GT * D::kN + kActThreads - 1) / kActThreads; ++it) {
             const int i = tid + it * kActThreads;
             if (i < nt * D::kN) {
                 const int tl = i / D::kN, c = i - tl * D::kN;
@@ -1167,9 +1169,19 @@ void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp,
     KernelTimer timer_(c, MHCLITE_KERNEL_ACT_PREMIX, s);
     const int C8 = c->C / 8;
     const float inv = 1.f / (float)(c->n * c->C);
-#define MHCL_AP_T(N_) lite_act_premix_t_k<N_><<<group_grid(T, kTokGroup, c->sm_count), kActThreads, 0, s>>>( \
+    // groups of 32 tokens unless that leaves resident block slots (three per SM) empty: then 16 or 8
+    const int resident_t = c->sm_count * 3;
+    // (but never groups of less than 256 KB of x: below that the phases' barriers cost more than the parallelism gains;
+    //  measured at C = 1024 and 1536)
+    int gmin = 8;
+    while (gmin < kTokGroup && (int64_t)gmin * c->n * c->C * 2 < 256 * 1024) gmin <<= 1;
+    int gtok = kTokGroup;
+    while (gtok > gmin && (T + gtok - 1) / gtok < (int64_t)resident_t) gtok >>= 1;
+    const int grid_t = group_grid(T, gtok, c->sm_count);
+#define MHCL_AP_TG(N_, G_) lite_act_premix_t_k<N_, G_><<<grid_t, kActThreads, 0, s>>>( \
         T, C8, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, \
         (const uint4*)x, (uint4*)u)
+#define MHCL_AP_T(N_) do { if (gtok == 8) MHCL_AP_TG(N_, 8); else if (gtok == 16) MHCL_AP_TG(N_, 16); else MHCL_AP_TG(N_, 32); } while (0)
     // one warp per token: n = 5 (120 logits do not fit a thread's registers) and every context that holds a
     // subset of the permutations (its table is data, not a compile-time constant)
 #define MHCL_AP_W(N_) lite_act_premix_k<N_><<<resident_grid(T, kGroupTok, c->sm_count * 4), kActThreads, 0, s>>>( \
@@ -1187,6 +1199,7 @@ void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp,
     }
 #undef MHCL_AP_W
 #undef MHCL_AP_T
+#undef MHCL_AP_TG
 }
 
 // Returns the number of blocks launched (= partials written when dalpha is null; only the n <= 4 kernel of a context
