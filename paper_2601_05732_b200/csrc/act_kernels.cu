@@ -941,25 +941,25 @@ __global__ void __launch_bounds__(128) sk_act_bwd_k(
 // sk_act_premix_k = SK activation + stream pre-mix (one thread per token for the 20 iterations, then all threads
 // stream the group's tokens); sk_tailpre_k = dH_pre stream (one warp per token) + SK backward (one thread per token).
 // ------------------------------------------------------------------------------------------------
-constexpr int kSkGroup = 64;     // tokens per block iteration
+constexpr int kSkGroup = 64;     // tokens per block iteration (GS below: 64, or 32 / 16 when there are few tokens)
 
-template <int N_>
+template <int N_, int GS>
 __global__ void __launch_bounds__(kActThreads, 3) sk_act_premix_k(
     int64_t T, int C8, int iters, int Npad, int ksplit, float inv_nC, float eps, const float* __restrict__ qpart,
     const float* __restrict__ ssq, const float* __restrict__ b, const float* __restrict__ alpha,
     float* __restrict__ H_res, float* __restrict__ H_pre, float* __restrict__ H_post, float* __restrict__ p_saved,
     float* __restrict__ rstd, const uint4* __restrict__ x, uint4* __restrict__ u) {
     constexpr int NN = N_ * N_, N = NN + 2 * N_;
-    __shared__ float pg[kSkGroup][N + 1];
-    __shared__ float og[kSkGroup][N + 1];          // H_res | H_pre | H_post
-    __shared__ float rg[kSkGroup];
+    __shared__ float pg[GS][N + 1];
+    __shared__ float og[GS][N + 1];          // H_res | H_pre | H_post
+    __shared__ float rg[GS];
     const int tid = threadIdx.x;
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
-    const int64_t ngroups = (T + kSkGroup - 1) / kSkGroup;
+    const int64_t ngroups = (T + GS - 1) / GS;
     for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
         // descending: the projection kernel before this one read x in ascending order and left its last lines in L2
-        const int64_t t0 = (ngroups - 1 - grp) * kSkGroup;
-        const int nt = (T - t0 < kSkGroup) ? (int)(T - t0) : kSkGroup;
+        const int64_t t0 = (ngroups - 1 - grp) * GS;
+        const int nt = (T - t0 < GS) ? (int)(T - t0) : GS;
         if (tid < nt) {
             float ss = 0.f;
             for (int s = 0; s < ksplit; ++s) ss += __ldg(ssq + (int64_t)s * T + t0 + tid);
@@ -1028,7 +1028,7 @@ __global__ void __launch_bounds__(kActThreads, 3) sk_act_premix_k(
     }
 }
 
-template <int N_>
+template <int N_, int GS>
 __global__ void __launch_bounds__(kActThreads, 3) sk_tailpre_k(
     int64_t T, int C8, int iters, float inv_nC, const uint4* __restrict__ x, const uint4* __restrict__ du,
     const float* __restrict__ p, const float* __restrict__ b, const float* __restrict__ rstd,
@@ -1038,17 +1038,17 @@ __global__ void __launch_bounds__(kActThreads, 3) sk_tailpre_k(
     constexpr int NN = N_ * N_, N = NN + 2 * N_;
     constexpr int o_dhres = N, o_hpre = o_dhres + NN, o_hpost = o_hpre + N_, o_dhpost = o_hpost + N_, o_rstd = o_dhpost + N_,
                   nin = o_rstd + 1;
-    __shared__ float in_s[kSkGroup][nin];          // p | dH_res | H_pre | H_post | dH_post | rstd of the group's tokens
-    __shared__ float dhp_s[kSkGroup][kMaxN];
+    __shared__ float in_s[GS][nin];          // p | dH_res | H_pre | H_post | dH_post | rstd of the group's tokens
+    __shared__ float dhp_s[GS][kMaxN];
     __shared__ float red[N + 3];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     for (int c = tid; c < N + 3; c += kActThreads) red[c] = 0.f;
     __syncthreads();
     const float a_res = __ldg(alpha), a_pre = __ldg(alpha + 1), a_post = __ldg(alpha + 2);
-    const int64_t ngroups = (T + kSkGroup - 1) / kSkGroup;
+    const int64_t ngroups = (T + GS - 1) / GS;
     for (int64_t grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
-        const int64_t t0 = grp * kSkGroup;
-        const int nt = (T - t0 < kSkGroup) ? (int)(T - t0) : kSkGroup;
+        const int64_t t0 = grp * GS;
+        const int nt = (T - t0 < GS) ? (int)(T - t0) : GS;
         // the per-token inputs of the SK backward travel to shared memory while the warps stream x and du
         for (int i = tid; i < nt * nin; i += kActThreads) {
             const int tl = i / nin, c = i - tl * nin;
@@ -1265,6 +1265,17 @@ void launch_sk_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, int iters, con
 
 namespace mhcl {
 
+// Tokens per group of the SK path's fused kernels: as for the lite path's thread-per-token kernel, smaller groups when
+// the full ones would leave resident block slots (three per SM) empty, but no group of less than 512 KB of x (the 20
+// iterations per token make its per-group phase longer: at C = 1024 groups of 32 were slower than groups of 64).
+static int sk_group_tokens(const mhclite_ctx* c, int64_t T) {
+    int gmin = 16;
+    while (gmin < kSkGroup && (int64_t)gmin * c->n * c->C * 2 < 512 * 1024) gmin <<= 1;
+    int gs = kSkGroup;
+    while (gs > gmin && 2 * ((T + gs - 1) / gs) <= (int64_t)c->sm_count * 3) gs >>= 1;   // halved groups still fit one wave
+    return gs;
+}
+
 void launch_sk_act_premix(const mhclite_ctx* c, int64_t T, int iters, const ProjPlan& pp, const float* qpart,
                           const float* ssq, float eps, const float* b, const float* alpha, float* H_res, float* H_pre,
                           float* H_post, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s) {
@@ -1272,10 +1283,13 @@ void launch_sk_act_premix(const mhclite_ctx* c, int64_t T, int iters, const Proj
     KernelTimer timer_(c, MHCLITE_KERNEL_ACT_PREMIX, s);
     const int C8 = c->C / 8;
     const float inv = 1.f / (float)(c->n * c->C);
-    const int grid = group_grid(T, kSkGroup, c->sm_count);
-    MHCL_DISPATCH_N(c->n, sk_act_premix_k<N_><<<grid, kActThreads, 0, s>>>(T, C8, iters, pp.Npad, pp.ksplit, inv, eps, qpart,
-                                                                          ssq, b, alpha, H_res, H_pre, H_post, p_saved, rstd,
-                                                                          (const uint4*)x, (uint4*)u));
+    const int gs = sk_group_tokens(c, T);
+    const int grid = group_grid(T, gs, c->sm_count);
+#define MHCL_SKAP(G_) MHCL_DISPATCH_N(c->n, (sk_act_premix_k<N_, G_><<<grid, kActThreads, 0, s>>>(                       \
+        T, C8, iters, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b, alpha, H_res, H_pre, H_post, p_saved, rstd,           \
+        (const uint4*)x, (uint4*)u)))
+    if (gs == 16) { MHCL_SKAP(16); } else if (gs == 32) { MHCL_SKAP(32); } else { MHCL_SKAP(64); }
+#undef MHCL_SKAP
 }
 
 int launch_sk_tailpre(const mhclite_ctx* c, int64_t T, int iters, const void* x, const void* du, const float* p,
@@ -1288,10 +1302,13 @@ int launch_sk_tailpre(const mhclite_ctx* c, int64_t T, int iters, const void* x,
     clear_e_tail(T, ehi, elo, Kp, s);
     const int C8 = c->C / 8;
     const float inv = 1.f / (float)(c->n * c->C);
-    const int grid = group_grid(T, kSkGroup, c->sm_count);
-    MHCL_DISPATCH_N(c->n, sk_tailpre_k<N_><<<grid, kActThreads, 0, s>>>(T, C8, iters, inv, (const uint4*)x, (const uint4*)du, p,
-                                                                       b, rstd, alpha, H_pre, H_post, dH_res, dH_post, eo,
-                                                                       kappa, db, dalpha));
+    const int gs = sk_group_tokens(c, T);
+    const int grid = group_grid(T, gs, c->sm_count);
+#define MHCL_SKTP(G_) MHCL_DISPATCH_N(c->n, (sk_tailpre_k<N_, G_><<<grid, kActThreads, 0, s>>>(                         \
+        T, C8, iters, inv, (const uint4*)x, (const uint4*)du, p, b, rstd, alpha, H_pre, H_post, dH_res, dH_post, eo,     \
+        kappa, db, dalpha)))
+    if (gs == 16) { MHCL_SKTP(16); } else if (gs == 32) { MHCL_SKTP(32); } else { MHCL_SKTP(64); }
+#undef MHCL_SKTP
     return grid;
 }
 
