@@ -9,7 +9,7 @@ output y and its backward's du are inputs).  Rank r of an N-GPU run processes it
 tokens (weak scaling, no data-path collective).  Prints one JSON line on rank 0.
 
 The default workload is the largest single-GPU one (cfg5: n = 4, C = 4096, T = 131072).  On one GPU the
-line also carries a `workloads` table: cfg2, the 24-layer stack cfg3, cfg4a, cfg4b, the subset variant of the
+line also carries a `workloads` table: cfg1 (forward only), cfg2, the 24-layer stack cfg3, cfg4a, cfg4b, the subset variant of the
 paper's Section 5 on the cfg4b shape (24 sampled permutations of 120) and the cfg5 token sweep, each with the
 mHC-lite step and (full tables) the in-library SK-20 step timed the same way (CUDA-graph replay).
 
@@ -534,7 +534,7 @@ def run_ours(args, wl, rank, world):
         del B, graph
         torch.cuda.empty_cache()
         # (workload, T override, K): K = a sampled subset of K of the n! permutations (paper Section 5) on that shape
-        rows = [("cfg2", None, None), ("cfg3", None, None), ("cfg4a", None, None), ("cfg4b", None, None),
+        rows = [("cfg1", None, None), ("cfg2", None, None), ("cfg3", None, None), ("cfg4a", None, None), ("cfg4b", None, None),
                 ("cfg4b", None, 24)] + [("cfg5", t, None) for t in (4096, 8192, 16384, 32768, 65536, 131072)]
         for name, Tt, K in rows:
             w = synth.WORKLOADS[name]
@@ -575,8 +575,10 @@ def run_ours(args, wl, rank, world):
                                                   not args.no_graph)
                 row = {"workload": name, "n": w.n, "C": w.C, "T": Tt, "ms_per_step": r["ms_per_step"],
                        "ms_min": r["ms_min"], "ms_max": r["ms_max"], "repeats": r["repeats"],
-                       **rates(w.n, w.C, Tt, r["ms_per_step"], peak), "launch": r["launch"],
+                       **rates(w.n, w.C, Tt, r["ms_per_step"], peak, backward=w.backward), "launch": r["launch"],
                        "launches_per_step": r["launches_per_step"]}
+                if not w.backward:
+                    row["note"] = "forward only; 29 MB of tensors: fits L2, launch-bound (reported, not a roofline case)"
                 row["sk20"] = sk_compare(c, w, Tt, a, r["ms_per_step"], Bl)
                 del Bl, gr
             c.device_status()
