@@ -405,6 +405,14 @@ def standin_sublayer_fwd(u, eps: float = 1e-6):
     return u * r
 
 
+def premix_row_rstd(u_stored, eps: float = 1e-6):
+    """Row statistic of an RMSNorm applied to the stored pre-mix output u = H_pre x_l (inner term of Eq. (1)):
+    (mean_c u[t,c]^2 + eps)^(-1/2) per token, over the values as stored (the caller passes the bf16-rounded u).
+    The stand-in sublayer above is u times this."""
+    u = np.asarray(u_stored, dtype=F64)
+    return 1.0 / np.sqrt(np.mean(u * u, axis=-1) + eps)
+
+
 def standin_sublayer_bwd(u, dy, eps: float = 1e-6):
     u = np.asarray(u, dtype=F64); dy = np.asarray(dy, dtype=F64)
     C = u.shape[-1]

@@ -43,6 +43,7 @@ SIGNATURES = {
     "mhclite_premix_fwd": (_i, [_p, _i64, _p, _p, _p, _p]),
     "mhclite_postres_fwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p]),
     "mhclite_pre_fwd_fused": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p]),
+    "mhclite_pre_fwd_fused_ustat": (_i, [_p, _i64, _p, _p, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p, _f, _p]),
     "mhclite_postres_fwd_next_proj": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p, _p, _p]),
     "mhclite_pre_fwd_resume": (_i, [_p, _i64, _p, _p, _p, _f, _p, _p, _p, _p, _p, _p, _p, _p]),
     "mhclite_postres_bwd": (_i, [_p, _i64, _p, _p, _p, _p, _p, _p, _p, _p, _p, _i, _p]),
@@ -214,6 +215,15 @@ class MhcLite:
             self._ptr(gain, f), float(eps), self._ptr(H_res, f), self._ptr(H_pre, f), self._ptr(H_post, f),
             self._ptr(a_saved, f), self._ptr(p_saved, f), self._ptr(rstd, f), self._ptr(u, h), self._stream()),
             "mhclite_pre_fwd_fused")
+
+    def pre_fwd_fused_ustat(self, x, W, b, alpha, gain, eps, H_res, H_pre, H_post, a_saved, p_saved, rstd, u, u_rstd,
+                            eps_u):
+        f, h = self._torch.float32, self._torch.bfloat16
+        self._check(self.lib.mhclite_pre_fwd_fused_ustat(
+            self._h, x.shape[0], self._ptr(x, h), self._ptr(W, f), self._ptr(b, f), self._ptr(alpha, f),
+            self._ptr(gain, f), float(eps), self._ptr(H_res, f), self._ptr(H_pre, f), self._ptr(H_post, f),
+            self._ptr(a_saved, f), self._ptr(p_saved, f), self._ptr(rstd, f), self._ptr(u, h), self._ptr(u_rstd, f),
+            float(eps_u), self._stream()), "mhclite_pre_fwd_fused_ustat")
 
     def postres_fwd_next_proj(self, x, y, H_res, H_post, x_next, W_next, gain_next):
         f, h = self._torch.float32, self._torch.bfloat16

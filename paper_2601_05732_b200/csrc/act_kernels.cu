@@ -544,12 +544,14 @@ __device__ __forceinline__ void lite_thread_fwd(const float* prow, float* orow, 
 
 constexpr int kTokGroup = 32;    // tokens per block iteration of the thread-per-token kernels
 
-template <int N_, int GT>
+template <int N_, int GT, bool USTAT>
 __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
     int64_t T, int C8, int Npad, int ksplit, float inv_nC, float eps, const float* __restrict__ qpart,
     const float* __restrict__ ssq, const float* __restrict__ b, const float* __restrict__ alpha,
     float* __restrict__ H_res, float* __restrict__ H_pre, float* __restrict__ H_post, float* __restrict__ a_saved,
-    float* __restrict__ p_saved, float* __restrict__ rstd, const uint4* __restrict__ x, uint4* __restrict__ u) {
+    float* __restrict__ p_saved, float* __restrict__ rstd, const uint4* __restrict__ x, uint4* __restrict__ u, float* __restrict__ u_rstd, float eps_u) {
+    // USTAT: also u_rstd[t] = (mean_c u[t,c]^2 + eps_u)^-1/2 of the stored (rounded) u: the statistic of the RMSNorm that
+    // usually opens the sublayer, so that the caller applies it as a row scale without another pass over u.
     // GT <= kTokGroup tokens per group: small when there are few tokens, so that every block walks several groups
     constexpr int gtok = GT;
     using D = LiteDims<N_>;
@@ -558,6 +560,7 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
     __shared__ float pg[GT][D::kN + 1];
     __shared__ float og[GT][D::kOut + 1];
     __shared__ float rg[GT];
+    __shared__ float usq[USTAT ? GT : 1];
     const int tid = threadIdx.x;
     for (int i = tid; i < D::kNN * D::kPer; i += kActThreads) klist_s[i] = c_perm[N_].klist[i];
     for (int i = tid; i < D::kN; i += kActThreads) b_s[i] = __ldg(b + i);
@@ -575,6 +578,7 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
             const float r = 1.f / sqrtf(ss * inv_nC + eps);
             rg[tid] = r;
             rstd[t0 + tid] = r;
+            if (USTAT) usq[tid] = 0.f;
         }
         float qv[(GT * D::kN + kActThreads - 1) / kActThreads];
 #pragma unroll
@@ -612,10 +616,15 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
             else H_post[t * N_ + (c - D::kFact - D::kNN - N_)] = v;
         }
         // P: u[t,:] = sum_j H_pre[t,j] x[t,j,:]  (two vectors per thread in flight)
-        for (int i0 = tid; i0 < nt * C8; i0 += 2 * kActThreads) {
+        // (with USTAT the warps stay whole through the loop, for the warp-wide sums below: a lane past the end repeats
+        //  the group's last vector and neither stores nor counts it)
+        const int total = nt * C8;
+        for (int i0 = tid; (USTAT ? i0 - (tid & 31) : i0) < total; i0 += 2 * kActThreads) {
+            const bool has0 = !USTAT || i0 < total;
+            const int i0c = has0 ? i0 : total - 1;
             const int i1 = i0 + kActThreads;
-            const bool has1 = i1 < nt * C8;
-            const int tl0 = i0 / C8, cv0 = i0 - tl0 * C8;
+            const bool has1 = i1 < total;
+            const int tl0 = i0c / C8, cv0 = i0c - tl0 * C8;
             const int tl1 = has1 ? i1 / C8 : tl0, cv1 = has1 ? i1 - tl1 * C8 : cv0;
             uint4 v0[N_], v1[N_];
 #pragma unroll
@@ -632,10 +641,26 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
 #pragma unroll
                 for (int e = 0; e < 8; ++e) { acc0[e] = fmaf(h0, f0[e], acc0[e]); acc1[e] = fmaf(h1, f1[e], acc1[e]); }
             }
-            st_stream(u + (t0 + tl0) * C8 + cv0, pack8(acc0));
-            if (has1) st_stream(u + (t0 + tl1) * C8 + cv1, pack8(acc1));
+            const uint4 pk0 = pack8(acc0), pk1 = pack8(acc1);
+            if (has0) st_stream(u + (t0 + tl0) * C8 + cv0, pk0);
+            if (has1) st_stream(u + (t0 + tl1) * C8 + cv1, pk1);
+            if (USTAT) {
+                float r0[8], r1[8], s0 = 0.f, s1 = 0.f;
+                unpack8(pk0, r0);
+                unpack8(pk1, r1);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { s0 = fmaf(r0[e], r0[e], s0); s1 = fmaf(r1[e], r1[e], s1); }
+                if (!has0) s0 = 0.f;
+                if (!has1) s1 = 0.f;
+                // the lanes of a warp mostly share a token: one shared-memory add per warp then
+                const bool same0 = __all_sync(0xffffffffu, tl0 == __shfl_sync(0xffffffffu, tl0, 0));
+                const bool same1 = __all_sync(0xffffffffu, tl1 == __shfl_sync(0xffffffffu, tl1, 0));
+                if (same0) { s0 = warp_sum(s0); if ((tid & 31) == 0) atomicAdd(&usq[tl0], s0); } else atomicAdd(&usq[tl0], s0);
+                if (same1) { s1 = warp_sum(s1); if ((tid & 31) == 0) atomicAdd(&usq[tl1], s1); } else atomicAdd(&usq[tl1], s1);
+            }
         }
         __syncthreads();
+        if (USTAT && tid < nt) u_rstd[t0 + tid] = 1.f / sqrtf(usq[tid] / (float)(C8 * 8) + eps_u);
     }
 }
 
@@ -1116,6 +1141,24 @@ __global__ void __launch_bounds__(kActThreads, 3) sk_tailpre_k(
     }
 }
 
+// u_rstd[t] = (mean_c u[t,c]^2 + eps)^-1/2, one warp per token: for the paths whose pre-mix kernel does not produce it.
+__global__ void __launch_bounds__(kActThreads) row_rstd_k(int64_t T, int C8, const uint4* __restrict__ u, float eps,
+                                                         float* __restrict__ u_rstd) {
+    const int lane = threadIdx.x & 31;
+    const int64_t nwarps = (int64_t)gridDim.x * kActWarps;
+    for (int64_t t = (int64_t)blockIdx.x * kActWarps + (threadIdx.x >> 5); t < T; t += nwarps) {
+        float s = 0.f;
+        for (int cv = lane; cv < C8; cv += 32) {
+            float f[8];
+            unpack8(ld_stream(u + t * C8 + cv), f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s = fmaf(f[e], f[e], s);
+        }
+        s = warp_sum(s);
+        if (lane == 0) u_rstd[t] = 1.f / sqrtf(s / (float)(C8 * 8) + eps);
+    }
+}
+
 // ---- launchers -----------------------------------------------------------------------------------
 static int warp_grid(int64_t T, int sm_count) {
     int64_t blocks = (T + kActWarps - 1) / kActWarps;
@@ -1164,7 +1207,8 @@ void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float*
 
 void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, const float* qpart, const float* ssq,
                             float eps, const float* b, const float* alpha, float* H_res, float* H_pre, float* H_post,
-                            float* a_saved, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s) {
+                            float* a_saved, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s, float* u_rstd,
+                            float eps_u) {
     c->launches += 1;
     KernelTimer timer_(c, MHCLITE_KERNEL_ACT_PREMIX, s);
     const int C8 = c->C / 8;
@@ -1178,15 +1222,17 @@ void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp,
     int gtok = kTokGroup;
     while (gtok > gmin && (T + gtok - 1) / gtok < (int64_t)resident_t) gtok >>= 1;
     const int grid_t = group_grid(T, gtok, c->sm_count);
-#define MHCL_AP_TG(N_, G_) lite_act_premix_t_k<N_, G_><<<grid_t, kActThreads, 0, s>>>( \
+#define MHCL_AP_TGS(N_, G_, S_) lite_act_premix_t_k<N_, G_, S_><<<grid_t, kActThreads, 0, s>>>( \
         T, C8, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, \
-        (const uint4*)x, (uint4*)u)
+        (const uint4*)x, (uint4*)u, u_rstd, eps_u)
+#define MHCL_AP_TG(N_, G_) do { if (u_rstd) MHCL_AP_TGS(N_, G_, true); else MHCL_AP_TGS(N_, G_, false); } while (0)
 #define MHCL_AP_T(N_) do { if (gtok == 8) MHCL_AP_TG(N_, 8); else if (gtok == 16) MHCL_AP_TG(N_, 16); else MHCL_AP_TG(N_, 32); } while (0)
     // one warp per token: n = 5 (120 logits do not fit a thread's registers) and every context that holds a
     // subset of the permutations (its table is data, not a compile-time constant)
 #define MHCL_AP_W(N_) lite_act_premix_k<N_><<<resident_grid(T, kGroupTok, c->sm_count * 4), kActThreads, 0, s>>>( \
         T, C8, c->nfact, pp.Npad, pp.ksplit, inv, eps, qpart, ssq, b, alpha, H_res, H_pre, H_post, a_saved, \
         p_saved, rstd, (const uint4*)x, (uint4*)u, c->table_dev)
+    const bool warp_kernel = c->table_dev || c->n > 4;
     if (c->table_dev) {
         MHCL_DISPATCH_N(c->n, MHCL_AP_W(N_));
     } else {
@@ -1197,9 +1243,19 @@ void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp,
             default: MHCL_AP_W(5);
         }
     }
+    if (u_rstd && warp_kernel) {                       // the warp-per-token kernel does not produce the statistic
+        c->launches += 1;
+        row_rstd_k<<<warp_grid(T, c->sm_count), kActThreads, 0, s>>>(T, C8, (const uint4*)u, eps_u, u_rstd);
+    }
 #undef MHCL_AP_W
 #undef MHCL_AP_T
 #undef MHCL_AP_TG
+#undef MHCL_AP_TGS
+}
+
+void launch_row_rstd(const mhclite_ctx* c, int64_t T, const void* u, float eps, float* u_rstd, cudaStream_t s) {
+    c->launches += 1;
+    row_rstd_k<<<warp_grid(T, c->sm_count), kActThreads, 0, s>>>(T, c->C / 8, (const uint4*)u, eps, u_rstd);
 }
 
 // Returns the number of blocks launched (= partials written when dalpha is null; only the n <= 4 kernel of a context

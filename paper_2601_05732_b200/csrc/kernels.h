@@ -85,7 +85,10 @@ void launch_lite_act_bwd(const mhclite_ctx* c, int64_t T, int Npad, const float*
 // mappings + pre-mix in one kernel; dH_pre + activation backward in one kernel (the fused call sequences)
 void launch_lite_act_premix(const mhclite_ctx* c, int64_t T, const ProjPlan& pp, const float* qpart, const float* ssq,
                             float eps, const float* b, const float* alpha, float* H_res, float* H_pre, float* H_post,
-                            float* a_saved, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s);
+                            float* a_saved, float* p_saved, float* rstd, const void* x, void* u, cudaStream_t s,
+                            float* u_rstd = nullptr, float eps_u = 0.f);
+// u_rstd[t] = (mean_c u[t,c]^2 + eps)^-1/2 of a stored u [T][C] (bf16), one warp per token
+void launch_row_rstd(const mhclite_ctx* c, int64_t T, const void* u, float eps, float* u_rstd, cudaStream_t s);
 int launch_lite_tailpre(const mhclite_ctx* c, int64_t T, const void* x, const void* du, const float* a, const float* p,
                         const float* rstd, const float* alpha, const float* H_pre, const float* H_post,
                         const float* dH_res, const float* dH_post, float* dH_pre_ws, float* e, int Npad, void* ehi,

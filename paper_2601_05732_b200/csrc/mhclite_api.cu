@@ -355,9 +355,10 @@ int mhclite_postres_fwd(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, cons
     return MHCLITE_OK;
 }
 
-int mhclite_pre_fwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W, const float* b,
-                          const float* alpha, const float* gain, float eps, float* H_res, float* H_pre, float* H_post,
-                          float* a_saved, float* p_saved, float* rstd, mhclite_bf16* u, void* stream) {
+static int pre_fwd_fused_impl(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W, const float* b,
+                              const float* alpha, const float* gain, float eps, float* H_res, float* H_pre, float* H_post,
+                              float* a_saved, float* p_saved, float* rstd, mhclite_bf16* u, float* u_rstd, float eps_u,
+                              void* stream) {
     MHCL_REQUIRE_CTX(ctx); MHCL_REQUIRE_T(ctx, T);
     if (T == 0) return MHCLITE_OK;
     MHCL_PTR(ctx, x); MHCL_PTR(ctx, W); MHCL_PTR(ctx, b); MHCL_PTR(ctx, alpha); MHCL_PTR(ctx, gain);
@@ -374,9 +375,28 @@ int mhclite_pre_fwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, co
     const ProjPlan pp = plan_proj(ctx->n, ctx->C, T, N, ctx->sm_count);
     rc = proj_forward(ctx, T, N, w, pp, x, W, gain, s);
     if (rc) return rc;
-    launch_lite_act_premix(ctx, T, pp, w.qpart, w.ssq, eps, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, x, u, s);
+    launch_lite_act_premix(ctx, T, pp, w.qpart, w.ssq, eps, b, alpha, H_res, H_pre, H_post, a_saved, p_saved, rstd, x, u, s,
+                           u_rstd, eps_u);
     MHCL_LAUNCH_CHECK(ctx, "lite_act_premix");
     return MHCLITE_OK;
+}
+
+int mhclite_pre_fwd_fused(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W, const float* b,
+                          const float* alpha, const float* gain, float eps, float* H_res, float* H_pre, float* H_post,
+                          float* a_saved, float* p_saved, float* rstd, mhclite_bf16* u, void* stream) {
+    return pre_fwd_fused_impl(ctx, T, x, W, b, alpha, gain, eps, H_res, H_pre, H_post, a_saved, p_saved, rstd, u, nullptr,
+                              0.f, stream);
+}
+
+int mhclite_pre_fwd_fused_ustat(mhclite_ctx* ctx, int64_t T, const mhclite_bf16* x, const float* W, const float* b,
+                                const float* alpha, const float* gain, float eps, float* H_res, float* H_pre,
+                                float* H_post, float* a_saved, float* p_saved, float* rstd, mhclite_bf16* u,
+                                float* u_rstd, float eps_u, void* stream) {
+    if (!ctx) return MHCLITE_ERR_BAD_ARG;
+    if (!u_rstd || ((uintptr_t)u_rstd & 15) != 0) return fail(ctx, MHCLITE_ERR_BAD_ARG, "u_rstd: null or not 16-byte aligned");
+    if (!(eps_u >= 0.f)) return fail(ctx, MHCLITE_ERR_BAD_ARG, "eps_u must be >= 0");
+    return pre_fwd_fused_impl(ctx, T, x, W, b, alpha, gain, eps, H_res, H_pre, H_post, a_saved, p_saved, rstd, u, u_rstd,
+                              eps_u, stream);
 }
 
 // One K slice covering all of n*C: the plan of projection partials that a single kernel produced per token tile.

@@ -49,8 +49,15 @@ class LayerBuffers:
         ctx.ensure_workspace(T, 0 if kind == "lite" else 1)
 
 
-def pre_fwd(ctx: MhcLite, P: LayerParams, B: LayerBuffers, x, eps=1e-6, fused=True, iters=20):
-    """Mappings + stream pre-mix: everything before the sublayer. Result: B.u (and the coefficients)."""
+def pre_fwd(ctx: MhcLite, P: LayerParams, B: LayerBuffers, x, eps=1e-6, fused=True, iters=20, u_rstd=None, eps_u=1e-6):
+    """Mappings + stream pre-mix: everything before the sublayer. Result: B.u (and the coefficients).  With u_rstd
+    (fp32 [T], fused lite path only) the call also leaves the RMSNorm row statistic of the stored u there."""
+    if u_rstd is not None:
+        if B.kind != "lite" or not fused:
+            raise ValueError("u_rstd is produced by the fused mHC-lite call only")
+        ctx.pre_fwd_fused_ustat(x, P.W, P.b, P.alpha, P.gain, eps, B.H_res, B.H_pre, B.H_post, B.a_saved, B.p_saved,
+                                B.rstd, B.u, u_rstd, eps_u)
+        return
     if B.kind == "sk" and fused:
         ctx.sk20_pre_fwd_fused(x, P.W, P.b, P.alpha, P.gain, eps, iters, B.H_res, B.H_pre, B.H_post, B.p_saved, B.rstd,
                                B.u)

@@ -395,3 +395,28 @@ def test_fused_tail_partials_accumulate_and_survive_a_graph(kind):
         st.synchronize()
     same_as_first("after a graph replay")
     G.ctx.device_status()
+
+
+@pytest.mark.parametrize("n,C,T", [(4, 1024, 300), (4, 4096, 70), (3, 264, 257), (2, 64, 100), (5, 320, 130)])
+def test_pre_fwd_with_the_row_statistic_of_u(n, C, T):
+    """mhclite_pre_fwd_fused_ustat: the same outputs as mhclite_pre_fwd_fused, and u_rstd = the oracle's RMSNorm row
+    statistic of the stored u (fused into the pre-mix kernel for n <= 4, a separate kernel for n = 5)."""
+    inp = synth.make_layer_inputs(n, C, T, seed=40 + n, bias_std=0.1, gain_std=0.1)
+    G = GpuLayer(inp)
+    G.forward(True)
+    torch.cuda.synchronize()
+    base = {k: getattr(G.B, k).clone() for k in ("u", "H_res", "H_pre", "H_post", "a_saved", "p_saved", "rstd")}
+    u_rstd = torch.full((T,), float("nan"), device=DEV)
+    eps_u = 1e-5
+    G.ctx.pre_fwd_fused_ustat(G.x, G.P.W, G.P.b, G.P.alpha, G.P.gain, G.eps, G.B.H_res, G.B.H_pre, G.B.H_post, G.B.a_saved,
+                              G.B.p_saved, G.B.rstd, G.B.u, u_rstd, eps_u)
+    torch.cuda.synchronize()
+    for k, v in base.items():
+        assert torch.equal(getattr(G.B, k), v), k
+    ref = O.premix_row_rstd(host(G.B.u), eps_u)          # over the stored (rounded) u, as the header says
+    check_f32("u_rstd", host(u_rstd), ref, 1e-5)
+    # and against the oracle's own u: the statistic inherits only u's bf16 rounding
+    ref_u = oracle_fwd(inp)["u"]
+    assert np.abs(host(u_rstd) / O.premix_row_rstd(ref_u, eps_u) - 1.0).max() < 4e-3
+    G.ctx.device_status()
+

@@ -358,6 +358,23 @@ def test_standin_sublayer_hand_case_and_gradient():
     assert np.abs((u * du0).sum(axis=1)).max() < 1e-13
 
 
+def test_premix_row_rstd_hand_cases():
+    # closed forms: u = (3, 4), eps = 0 -> mean square 12.5; u = (1,-1,1,-1), eps = 3 -> 1/sqrt(4); u = 0 -> eps^-1/2
+    assert abs(O.premix_row_rstd(np.array([[3.0, 4.0]]), 0.0)[0] - 1.0 / math.sqrt(12.5)) < 1e-16
+    assert abs(O.premix_row_rstd(np.array([[1.0, -1.0, 1.0, -1.0]]), 3.0)[0] - 0.5) < 1e-16
+    assert abs(O.premix_row_rstd(np.zeros((1, 8)), 0.25)[0] - 2.0) < 1e-16
+    # one value per token, each from its own row only; a row scaled by s has its statistic divided by s at eps = 0
+    r = np.random.default_rng(11)
+    u = r.standard_normal((5, 12))
+    got = O.premix_row_rstd(u, 0.0)
+    assert got.shape == (5,)
+    u2 = u.copy(); u2[3] *= 4.0
+    got2 = O.premix_row_rstd(u2, 0.0)
+    assert np.abs(got2[[0, 1, 2, 4]] - got[[0, 1, 2, 4]]).max() == 0.0 and abs(got2[3] - got[3] / 4.0) < 1e-15
+    # the normalised row has unit mean square
+    assert np.abs(np.mean((u * got[:, None]) ** 2, axis=1) - 1.0).max() < 1e-14
+
+
 def _stack_params(Ld, n, C, seed):
     r = np.random.default_rng(seed)
     N = math.factorial(n) + 2 * n
