@@ -560,7 +560,6 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
     __shared__ float pg[GT][D::kN + 1];
     __shared__ float og[GT][D::kOut + 1];
     __shared__ float rg[GT];
-    __shared__ float usq[USTAT ? GT : 1];
     const int tid = threadIdx.x;
     for (int i = tid; i < D::kNN * D::kPer; i += kActThreads) klist_s[i] = c_perm[N_].klist[i];
     for (int i = tid; i < D::kN; i += kActThreads) b_s[i] = __ldg(b + i);
@@ -578,7 +577,6 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
             const float r = 1.f / sqrtf(ss * inv_nC + eps);
             rg[tid] = r;
             rstd[t0 + tid] = r;
-            if (USTAT) usq[tid] = 0.f;
         }
         float qv[(GT * D::kN + kActThreads - 1) / kActThreads];
 #pragma unroll
@@ -616,15 +614,52 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
             else H_post[t * N_ + (c - D::kFact - D::kNN - N_)] = v;
         }
         // P: u[t,:] = sum_j H_pre[t,j] x[t,j,:]  (two vectors per thread in flight)
-        // (with USTAT the warps stay whole through the loop, for the warp-wide sums below: a lane past the end repeats
-        //  the group's last vector and neither stores nor counts it)
-        const int total = nt * C8;
-        for (int i0 = tid; (USTAT ? i0 - (tid & 31) : i0) < total; i0 += 2 * kActThreads) {
-            const bool has0 = !USTAT || i0 < total;
-            const int i0c = has0 ? i0 : total - 1;
+        if (USTAT) {
+            // one warp per token here, so that a lane sums the squares of its own vectors in a register and the warp adds
+            // them up once per token (warp-wide sums per vector, or shared-memory atomics, cost far more)
+            const int lane = tid & 31;
+            for (int tl = tid >> 5; tl < nt; tl += kActWarps) {
+                const int64_t t = t0 + tl;
+                float h[N_];
+#pragma unroll
+                for (int j = 0; j < N_; ++j) h[j] = og[tl][D::kFact + D::kNN + j];
+                float sq = 0.f;
+                for (int cv0 = lane; cv0 < C8; cv0 += 64) {
+                    const bool has1 = cv0 + 32 < C8;
+                    const int cv1 = has1 ? cv0 + 32 : cv0;
+                    uint4 v0[N_], v1[N_];
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) v0[j] = ld_stream(x + (t * N_ + j) * C8 + cv0);
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) v1[j] = ld_stream(x + (t * N_ + j) * C8 + cv1);
+                    float acc0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, acc1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+                    for (int j = 0; j < N_; ++j) {
+                        float f0[8], f1[8];
+                        unpack8(v0[j], f0);
+                        unpack8(v1[j], f1);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) { acc0[e] = fmaf(h[j], f0[e], acc0[e]); acc1[e] = fmaf(h[j], f1[e], acc1[e]); }
+                    }
+                    const uint4 pk0 = pack8(acc0), pk1 = pack8(acc1);
+                    st_stream(u + t * C8 + cv0, pk0);
+                    if (has1) st_stream(u + t * C8 + cv1, pk1);
+                    float r0[8], r1[8], s1 = 0.f;
+                    unpack8(pk0, r0);                          // the statistic is over the values as stored
+                    unpack8(pk1, r1);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) { sq = fmaf(r0[e], r0[e], sq); s1 = fmaf(r1[e], r1[e], s1); }
+                    if (has1) sq += s1;
+                }
+                sq = warp_sum(sq);                             // every lane of the warp is here: the token loop is warp-uniform
+                if (lane == 0) u_rstd[t] = 1.f / sqrtf(sq / (float)(C8 * 8) + eps_u);
+            }
+        }
+        const int total = USTAT ? 0 : nt * C8;
+        for (int i0 = tid; i0 < total; i0 += 2 * kActThreads) {
             const int i1 = i0 + kActThreads;
             const bool has1 = i1 < total;
-            const int tl0 = i0c / C8, cv0 = i0c - tl0 * C8;
+            const int tl0 = i0 / C8, cv0 = i0 - tl0 * C8;
             const int tl1 = has1 ? i1 / C8 : tl0, cv1 = has1 ? i1 - tl1 * C8 : cv0;
             uint4 v0[N_], v1[N_];
 #pragma unroll
@@ -641,26 +676,10 @@ __global__ void __launch_bounds__(kActThreads, 3) lite_act_premix_t_k(
 #pragma unroll
                 for (int e = 0; e < 8; ++e) { acc0[e] = fmaf(h0, f0[e], acc0[e]); acc1[e] = fmaf(h1, f1[e], acc1[e]); }
             }
-            const uint4 pk0 = pack8(acc0), pk1 = pack8(acc1);
-            if (has0) st_stream(u + (t0 + tl0) * C8 + cv0, pk0);
-            if (has1) st_stream(u + (t0 + tl1) * C8 + cv1, pk1);
-            if (USTAT) {
-                float r0[8], r1[8], s0 = 0.f, s1 = 0.f;
-                unpack8(pk0, r0);
-                unpack8(pk1, r1);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) { s0 = fmaf(r0[e], r0[e], s0); s1 = fmaf(r1[e], r1[e], s1); }
-                if (!has0) s0 = 0.f;
-                if (!has1) s1 = 0.f;
-                // the lanes of a warp mostly share a token: one shared-memory add per warp then
-                const bool same0 = __all_sync(0xffffffffu, tl0 == __shfl_sync(0xffffffffu, tl0, 0));
-                const bool same1 = __all_sync(0xffffffffu, tl1 == __shfl_sync(0xffffffffu, tl1, 0));
-                if (same0) { s0 = warp_sum(s0); if ((tid & 31) == 0) atomicAdd(&usq[tl0], s0); } else atomicAdd(&usq[tl0], s0);
-                if (same1) { s1 = warp_sum(s1); if ((tid & 31) == 0) atomicAdd(&usq[tl1], s1); } else atomicAdd(&usq[tl1], s1);
-            }
+            st_stream(u + (t0 + tl0) * C8 + cv0, pack8(acc0));
+            if (has1) st_stream(u + (t0 + tl1) * C8 + cv1, pack8(acc1));
         }
         __syncthreads();
-        if (USTAT && tid < nt) u_rstd[t0 + tid] = 1.f / sqrtf(usq[tid] / (float)(C8 * 8) + eps_u);
     }
 }
 
